@@ -1,0 +1,243 @@
+/*
+ * calidrop.h -- C ABI of the B200 (sm_100a) CaliDrop hot path.
+ *
+ * Two operations, after "CaliDrop: KV Cache Compression with Calibration":
+ *
+ *   calidrop_compress  end of prefill (Algorithm 1, lines 3-8): score the prompt's keys
+ *                      with an observation window of recent queries, pool the scores, keep
+ *                      a per-kv-head top-k budget of KV rows, compact them, and precompute
+ *                      the calibration term (O_c, LSE_c, C_q) over the evicted rows.
+ *   calidrop_decode    one decode step (Algorithm 2, lines 1-2 and 9-14): attention of the
+ *                      new query over the retained cache, cosine similarity with the stored
+ *                      calibration queries, threshold gate, and the merge of Eq. 1-2.
+ *
+ * Conventions
+ *   - Unless a comment says HOST, every tensor pointer is a DEVICE pointer to a contiguous,
+ *     16-byte aligned buffer on the current device.  "bf16" buffers hold bfloat16 values.
+ *   - The library allocates nothing, owns nothing and keeps no pointer between calls.  All
+ *     buffers, including the workspaces, belong to the caller.
+ *   - Every call validates its arguments on the host BEFORE enqueueing anything; a call that
+ *     returns a non-zero status has had no effect.  Work is enqueued on `stream`
+ *     (a cudaStream_t passed as void*; NULL is the default stream) and the call returns
+ *     without synchronising.
+ *   - Status codes: 0 = CALIDROP_OK, negative = error (see below).  No exceptions, no abort,
+ *     no device trap.
+ *   - Logits are q.k * softmax_scale with softmax_scale = 1/sqrt(D) when the field is 0.
+ *     (Algorithm 1 prints the exponent of C_weight divided by d_k; Eq. 1-2 only hold with
+ *     the attention's own 1/sqrt(d_k), which is what is used everywhere here.)
+ *   - C_weight of Algorithm 1 is stored as its logarithm LSE_c; A_weight of Algorithm 2
+ *     likewise as LSE_a.  alpha_i = exp(LSE_a - logaddexp(LSE_a, LSE_c)), which is Eq. 2.
+ */
+#ifndef CALIDROP_H_
+#define CALIDROP_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define CALIDROP_OK 0
+#define CALIDROP_INVALID_ARG (-1)         /* null/misaligned pointer, inconsistent sizes      */
+#define CALIDROP_UNSUPPORTED (-2)         /* D != 128, Hq/Hkv > 8, device is not sm_100       */
+#define CALIDROP_WORKSPACE_TOO_SMALL (-3)
+#define CALIDROP_CUDA_ERROR (-4)          /* a launch or runtime call failed                  */
+
+#define CALIDROP_MAX_LAYERS 32            /* layers per calidrop_decode_batched call          */
+
+typedef struct calidrop_params {
+  int32_t B, Hq, Hkv, D;        /* D must be 128; Hq % Hkv == 0; G = Hq/Hkv <= 8              */
+  int32_t L;                    /* prompt length; K, V are [B, Hkv, L, D]                      */
+  int32_t window;               /* W >= 1: observation window = the last W prompt positions    */
+  int32_t pool;                 /* odd >= 1: average-pool kernel over the votes                */
+  int32_t budget;               /* retained prompt rows per kv head, INCLUDING the W window    */
+                                /* rows; budget >= L keeps everything                          */
+  int32_t n_cal;                /* 1..W calibration queries = the last n_cal window rows;      */
+                                /* 1 is Algorithm 1 as printed (the last query only)           */
+  int32_t cap;                  /* row capacity of K_kept/V_kept: >= min(budget,L) + appended  */
+  float   softmax_scale;        /* 0 => 1/sqrt(D)                                              */
+  float   theta1, theta2;       /* decode: rho < theta1 raises needs_recompute; rho > theta2   */
+                                /* applies the calibration; theta2 <= -1 always applies it     */
+} calidrop_params;
+
+/*
+ * Bytes of scratch calidrop_compress needs for these parameters (0 if they are invalid).
+ */
+size_t calidrop_compress_workspace_bytes(const calidrop_params* p);
+
+/*
+ * Compress-and-calibrate (Algorithm 1, lines 3-8, with the SnapKV eviction rule the paper's
+ * Sections 1 and 4.1.3 describe: observation window + pooled accumulated attention).
+ *
+ * Per (batch b, kv head h), with G query heads per kv head and candidates t in [0, L-W):
+ *   a[g][j][t]  softmax row of window query j of head h*G+g (prompt position L-W+j) over
+ *               the keys t <= L-W+j it can see;
+ *   vote[t]   = sum_g sum_j a[g][j][t];
+ *   pooled[t] = (1/pool) sum_{|d| <= pool/2} vote[t+d]   (zero padding, constant divisor);
+ *   kept      = the budget-W candidates with the largest pooled[t] (ties: lowest index),
+ *               in ascending order, followed by the window rows L-W .. L-1;
+ *   E         = [0, L-W) \ kept, the evicted rows;
+ *   for c < n_cal, q_c = Q_obs[b, h*G+g, W-n_cal+c]:
+ *     LSE_c[c] = log sum_{t in E} exp(q_c.k_t * scale),  O_c[c] = Att(q_c, K_E, V_E),
+ *     C_q[c] = q_c.                                       (lines 5-8 of Algorithm 1)
+ * budget >= L keeps all L rows (n_kept = L), LSE_c = -inf, O_c = 0.
+ *
+ *   Q_obs   in  [B, Hq, W, D] bf16   the last W prompt queries, as the attention sees them
+ *   K, V    in  [B, Hkv, L, D] bf16
+ *   lse_obs in  [B, Hq, W] f32 or NULL: natural-log softmax denominators of those W rows of
+ *               the prefill attention (over keys t <= L-W+j, same scale).  Supplying them
+ *               skips the pass that recomputes them.  Not validated.
+ *   kept_idx out [B, Hkv, n_kept] i32, n_kept = min(budget, L)
+ *   K_kept, V_kept out [B, Hkv, cap, D] bf16; rows 0..n_kept-1 are written (bit copies)
+ *   O_c     out [B, Hq, n_cal, D] f32
+ *   LSE_c   out [B, Hq, n_cal] f32
+ *   C_q     out [B, Hq, n_cal, D] bf16
+ *   workspace   scratch of at least calidrop_compress_workspace_bytes(p) bytes, 256-byte
+ *               aligned; contents are undefined afterwards.  Two calls that overlap on the
+ *               device must not share a workspace.
+ *
+ * Errors: INVALID_ARG for a null or misaligned pointer, Hq % Hkv != 0, window < 1,
+ * even or non-positive pool, n_cal outside 1..W, budget <= window while budget < L,
+ * L < window while budget < L, cap < n_kept; UNSUPPORTED for D != 128 or G > 8 or a device
+ * that is not compute capability 10.x; WORKSPACE_TOO_SMALL; CUDA_ERROR.
+ */
+int calidrop_compress(const calidrop_params* p,
+                      const void* Q_obs, const void* K, const void* V, const float* lse_obs,
+                      int32_t* kept_idx, void* K_kept, void* V_kept,
+                      float* O_c, float* LSE_c, void* C_q,
+                      void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * Offsets (bytes from the workspace base) of intermediate arrays of the last
+ * calidrop_compress call that used this workspace, for diagnostics and tests:
+ *   vote   [B, Hkv, L-W] f32, pooled [B, Hkv, L-W] f32, row_lse [B, Hq, W] f32 (natural log).
+ * Returns CALIDROP_OK, or INVALID_ARG if the parameters are invalid.
+ */
+typedef struct calidrop_compress_layout {
+  size_t vote_offset, pooled_offset, row_lse_offset;
+} calidrop_compress_layout;
+int calidrop_compress_workspace_layout(const calidrop_params* p, calidrop_compress_layout* out);
+
+/*
+ * Bytes of scratch calidrop_decode needs when the retained cache holds at most kv_len_max
+ * rows after the append (0 if the parameters are invalid).  For calidrop_decode_batched
+ * multiply by the number of layers.
+ */
+size_t calidrop_decode_workspace_bytes(const calidrop_params* p, int32_t kv_len_max);
+
+/*
+ * Zero a decode workspace (asynchronously on `stream`).  A decode workspace must be zeroed
+ * once before its first use; every decode call leaves it ready for the next one.  Calls
+ * that overlap on the device must not share a workspace.
+ */
+int calidrop_decode_workspace_init(void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * One decode step for one layer (Algorithm 2, lines 1-2 and 9-14).
+ *
+ * Per (b, query head hq of kv head h):
+ *   if k_new != NULL the step's key/value rows are first stored at row kv_len of the cache;
+ *   (O_a, LSE_a) = attention of q over cache rows [0, n_kv), n_kv = kv_len + (k_new ? 1 : 0),
+ *                  with the log of its softmax denominator;            (line 1)
+ *   rho_c = cos(q, C_q[c]) (0 if either norm is 0); c* = argmax_c rho_c, ties to the
+ *           largest c; rho = rho_{c*};                                  (line 2)
+ *   needs_recompute = rho < theta1  (lines 3-8, the reload of the evicted KV, are the
+ *           caller's business: this call only raises the flag);
+ *   if (rho > theta2 or theta2 <= -1) and LSE_c[c*] > -inf:             (lines 9-12, Eq. 1-2)
+ *        LSE = logaddexp(LSE_a, LSE_c[c*]);
+ *        out = exp(LSE_a - LSE) O_a + exp(LSE_c[c*] - LSE) O_c[c*];
+ *   else out = O_a, LSE = LSE_a.                                        (lines 13-14)
+ *
+ *   q        in  [B, Hq, D] bf16
+ *   k_new, v_new in [B, Hkv, D] bf16, or both NULL (no append)
+ *   K_kept, V_kept in/out [B, Hkv, cap, D] bf16; row kv_len is written when k_new != NULL.
+ *            The caller advances kv_len by one after an appending call.
+ *   kv_len   rows valid before this call; kv_len + (k_new ? 1 : 0) must be in 1..cap
+ *   O_c, LSE_c, C_q in: as written by calidrop_compress
+ *   out      out [B, Hq, D] bf16
+ *   lse_out  out [B, Hq] f32 or NULL: the log-denominator that `out` corresponds to
+ *   flags    out [B, Hq] u8 or NULL: bit 0 calibration applied, bit 1 needs_recompute,
+ *            bits 2..7 c* (only when n_cal <= 64)
+ *   workspace    zero-initialised scratch (see calidrop_decode_workspace_init) of at least
+ *            calidrop_decode_workspace_bytes(p, kv_len + 1) bytes, 256-byte aligned
+ *
+ * Only B, Hq, Hkv, D, n_cal, cap, softmax_scale, theta1, theta2 of `p` are read.
+ * Errors as for calidrop_compress.
+ */
+int calidrop_decode(const calidrop_params* p,
+                    const void* q, const void* k_new, const void* v_new,
+                    void* K_kept, void* V_kept, int32_t kv_len,
+                    const float* O_c, const float* LSE_c, const void* C_q,
+                    void* out, float* lse_out, uint8_t* flags,
+                    void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * The same decode step for n_layers independent layers of identical shape in ONE launch
+ * (the attention layers of a model stack do not depend on each other inside this path once
+ * their queries are known; a stack of small retained caches is otherwise launch-bound).
+ * `layers` is a HOST array of n_layers entries whose members are the device pointers of
+ * calidrop_decode, per layer.  n_layers must be in 1..CALIDROP_MAX_LAYERS.  The workspace
+ * must hold n_layers * calidrop_decode_workspace_bytes(p, kv_len + 1) bytes.
+ */
+typedef struct calidrop_decode_layer {
+  const void* q;
+  const void* k_new;
+  const void* v_new;
+  void* K_kept;
+  void* V_kept;
+  const float* O_c;
+  const float* LSE_c;
+  const void* C_q;
+  void* out;
+  float* lse_out;
+  uint8_t* flags;
+} calidrop_decode_layer;
+
+int calidrop_decode_batched(const calidrop_params* p, int32_t n_layers,
+                            const calidrop_decode_layer* layers /* HOST */, int32_t kv_len,
+                            void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * End-to-end variants for callers whose tensors live in HOST memory (pinned memory makes the
+ * copies asynchronous).  Inputs are copied to the caller's device buffers, the device
+ * operation runs, and the results are copied back, all on `stream`; the call returns without
+ * synchronising.  Arguments with the suffix _h are HOST pointers with the layouts of their
+ * device counterparts; the device buffers and workspaces are as above.
+ *
+ * calidrop_compress_host copies Q_obs, K, V (and lse_obs_h if not NULL) in, and kept_idx,
+ * O_c, LSE_c out; the compacted cache and C_q stay on the device for the decode steps.
+ * calidrop_decode_host copies q, k_new, v_new in and out (and lse_out/flags if not NULL) out.
+ */
+int calidrop_compress_host(const calidrop_params* p,
+                           const void* Q_obs_h, const void* K_h, const void* V_h,
+                           const float* lse_obs_h,
+                           int32_t* kept_idx_h, float* O_c_h, float* LSE_c_h,
+                           void* Q_obs, void* K, void* V, float* lse_obs,
+                           int32_t* kept_idx, void* K_kept, void* V_kept,
+                           float* O_c, float* LSE_c, void* C_q,
+                           void* workspace, size_t workspace_bytes, void* stream);
+
+int calidrop_decode_host(const calidrop_params* p,
+                         const void* q_h, const void* k_new_h, const void* v_new_h,
+                         void* out_h, float* lse_out_h, uint8_t* flags_h,
+                         void* q, void* k_new, void* v_new,
+                         void* K_kept, void* V_kept, int32_t kv_len,
+                         const float* O_c, const float* LSE_c, const void* C_q,
+                         void* out, float* lse_out, uint8_t* flags,
+                         void* workspace, size_t workspace_bytes, void* stream);
+
+/* Human-readable text for a status code; for CALIDROP_CUDA_ERROR includes the last CUDA
+ * error string seen by the calling thread. */
+const char* calidrop_status_string(int status);
+
+/* Library version: major * 10000 + minor * 100 + patch. */
+int calidrop_version(void);
+
+/* Number of kernels the library has launched from the calling process so far. */
+uint64_t calidrop_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* CALIDROP_H_ */

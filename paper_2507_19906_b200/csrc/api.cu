@@ -1,0 +1,334 @@
+// C-ABI layer: argument validation, workspace carving and launch sequencing.
+// Everything that computes lives in the kernels; this file only marshals.
+#include <atomic>
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+
+#include "../../include/calidrop.h"
+#include "common.cuh"
+#include "internal.h"
+
+namespace calidrop {
+
+namespace {
+
+std::atomic<uint64_t> g_launches{0};
+thread_local char g_err_text[256] = "";
+
+size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+int cuda_fail(cudaError_t e) {
+  snprintf(g_err_text, sizeof g_err_text, "CUDA error: %s", cudaGetErrorString(e));
+  return CALIDROP_CUDA_ERROR;
+}
+
+// Parameter checks shared by every entry point that reads the full struct.
+int check_common(const calidrop_params* p) {
+  if (!p) return CALIDROP_INVALID_ARG;
+  if (p->B < 1 || p->Hq < 1 || p->Hkv < 1 || p->Hq % p->Hkv != 0) return CALIDROP_INVALID_ARG;
+  if (p->D != kD) return CALIDROP_UNSUPPORTED;
+  if (p->Hq / p->Hkv > kMaxG) return CALIDROP_UNSUPPORTED;
+  if (p->n_cal < 1 || p->cap < 1) return CALIDROP_INVALID_ARG;
+  if (!(p->softmax_scale >= 0.f) || !std::isfinite(p->softmax_scale)) return CALIDROP_INVALID_ARG;
+  return CALIDROP_OK;
+}
+
+int check_compress(const calidrop_params* p) {
+  int rc = check_common(p);
+  if (rc != CALIDROP_OK) return rc;
+  if (p->L < 1 || p->window < 1 || p->budget < 1) return CALIDROP_INVALID_ARG;
+  if (p->pool < 1 || p->pool % 2 == 0) return CALIDROP_INVALID_ARG;
+  if (p->n_cal > p->window) return CALIDROP_INVALID_ARG;
+  if (p->budget < p->L && (p->budget <= p->window || p->L < p->window)) return CALIDROP_INVALID_ARG;
+  const int n_kept = p->budget < p->L ? p->budget : p->L;
+  if (p->cap < n_kept) return CALIDROP_INVALID_ARG;
+  return CALIDROP_OK;
+}
+
+float scale2_of(const calidrop_params* p) {
+  const float s = p->softmax_scale > 0.f ? p->softmax_scale : 1.0f / sqrtf((float)p->D);
+  return s * kLog2e;
+}
+
+CompressGeom make_geom(const calidrop_params* p) {
+  CompressGeom g{};
+  g.B = p->B; g.Hq = p->Hq; g.Hkv = p->Hkv; g.G = p->Hq / p->Hkv;
+  g.L = p->L; g.W = p->window; g.pool = p->pool; g.budget = p->budget; g.n_cal = p->n_cal; g.cap = p->cap;
+  g.keep_all = p->budget >= p->L;
+  g.n_cand = g.keep_all ? 0 : p->L - p->window;
+  g.k_sel = g.keep_all ? 0 : p->budget - p->window;
+  g.n_kept = g.keep_all ? p->L : p->budget;
+  g.units = p->B * p->Hkv;
+  g.bitmap_words = (p->L + 31) / 32;
+  g.scale2 = scale2_of(p);
+  return g;
+}
+
+CompressWs make_ws(const CompressGeom& g) {
+  CompressWs w{};
+  size_t off = 0;
+  const size_t n_cand = (size_t)(g.L > g.W ? g.L - g.W : 0);
+  w.vote = off;    off = align_up(off + (size_t)g.units * n_cand * 4, 256);
+  w.pooled = off;  off = align_up(off + (size_t)g.units * n_cand * 4, 256);
+  w.row_lse = off; off = align_up(off + (size_t)g.B * g.Hq * g.W * 4, 256);
+  w.bitmap = off;  off = align_up(off + (size_t)g.units * g.bitmap_words * 4, 256);
+  w.n_tiles = (g.L + 127) / 128;
+  w.stat_part = off; off = align_up(off + (size_t)g.B * g.Hq * g.W * w.n_tiles * 8, 256);
+  w.total = off;
+  return w;
+}
+
+int device_supported() {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return 0;
+  static int major_of[64];
+  if (dev < 0 || dev >= 64) return 0;
+  if (major_of[dev] == 0) {
+    int major = 0;
+    if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return 0;
+    major_of[dev] = major;
+  }
+  return major_of[dev] == 10;
+}
+
+// Split-K factor of the decode launch: enough CTAs to fill the machine twice over, never
+// fewer than 32 rows per split.
+int decode_nsplit(int units_total, int n_kv) {
+  int ns = kDecodeTargetCtas / units_total;
+  if (ns < 1) ns = 1;
+  if (ns > kDecodeMaxSplit) ns = kDecodeMaxSplit;
+  const int by_rows = (n_kv + 31) / 32;
+  if (ns > by_rows) ns = by_rows;
+  return ns < 1 ? 1 : ns;
+}
+
+struct DecodeWs {
+  size_t part_o, part_ml, rho, counters, per_layer;
+  int max_split;
+};
+
+DecodeWs make_decode_ws(const calidrop_params* p) {
+  DecodeWs w{};
+  const int units = p->B * p->Hkv;
+  w.max_split = decode_nsplit(units, 1 << 30);
+  size_t off = 0;
+  w.counters = off; off = align_up(off + (size_t)units * 4 * kDecodeMaxLayers, 256);
+  w.part_ml = off;  off = align_up(off + (size_t)units * w.max_split * kMaxG * 2 * 4, 256);
+  w.rho = off;      off = align_up(off + (size_t)units * kMaxG * p->n_cal * 4, 256);
+  w.part_o = off;   off = align_up(off + (size_t)units * w.max_split * kMaxG * kD * 4, 256);
+  w.per_layer = off;
+  return w;
+}
+
+}  // namespace
+
+void count_launch(int n) { g_launches.fetch_add((uint64_t)n, std::memory_order_relaxed); }
+
+}  // namespace calidrop
+
+using namespace calidrop;
+
+extern "C" {
+
+size_t calidrop_compress_workspace_bytes(const calidrop_params* p) {
+  if (check_compress(p) != CALIDROP_OK) return 0;
+  return make_ws(make_geom(p)).total;
+}
+
+int calidrop_compress_workspace_layout(const calidrop_params* p, calidrop_compress_layout* out) {
+  int rc = check_compress(p);
+  if (rc != CALIDROP_OK || !out) return rc != CALIDROP_OK ? rc : CALIDROP_INVALID_ARG;
+  CompressWs w = make_ws(make_geom(p));
+  out->vote_offset = w.vote;
+  out->pooled_offset = w.pooled;
+  out->row_lse_offset = w.row_lse;
+  return CALIDROP_OK;
+}
+
+int calidrop_compress(const calidrop_params* p, const void* Q_obs, const void* K, const void* V,
+                      const float* lse_obs, int32_t* kept_idx, void* K_kept, void* V_kept, float* O_c,
+                      float* LSE_c, void* C_q, void* workspace, size_t workspace_bytes, void* stream) {
+  int rc = check_compress(p);
+  if (rc != CALIDROP_OK) return rc;
+  const void* ptrs[] = {Q_obs, K, V, kept_idx, K_kept, V_kept, O_c, LSE_c, C_q, workspace};
+  for (const void* q : ptrs)
+    if (!q || !aligned16(q)) return CALIDROP_INVALID_ARG;
+  if (lse_obs && !aligned16(lse_obs)) return CALIDROP_INVALID_ARG;
+  if (reinterpret_cast<uintptr_t>(workspace) & 255u) return CALIDROP_INVALID_ARG;
+  const CompressGeom g = make_geom(p);
+  const CompressWs ws = make_ws(g);
+  if (workspace_bytes < ws.total) return CALIDROP_WORKSPACE_TOO_SMALL;
+  if (!device_supported()) return CALIDROP_UNSUPPORTED;
+
+  cudaStream_t st = (cudaStream_t)stream;
+  char* wsp = (char*)workspace;
+  cudaError_t e = cudaSuccess;
+  if (!g.keep_all) {
+    const float* row_lse = lse_obs;
+    if (!row_lse) {
+      e = launch_row_stats(g, ws, Q_obs, K, wsp, st);
+      if (e != cudaSuccess) return cuda_fail(e);
+      row_lse = (const float*)(wsp + ws.row_lse);
+    }
+    e = launch_votes(g, ws, Q_obs, K, row_lse, wsp, st);
+    if (e != cudaSuccess) return cuda_fail(e);
+  }
+  e = launch_pool_select(g, ws, wsp, kept_idx, st);
+  if (e != cudaSuccess) return cuda_fail(e);
+  e = launch_gather(g, K, V, kept_idx, K_kept, V_kept, st);
+  if (e != cudaSuccess) return cuda_fail(e);
+  e = launch_calib_direct(g, ws, Q_obs, K, V, wsp, O_c, LSE_c, C_q, st);
+  if (e != cudaSuccess) return cuda_fail(e);
+  return CALIDROP_OK;
+}
+
+size_t calidrop_decode_workspace_bytes(const calidrop_params* p, int32_t kv_len_max) {
+  if (check_common(p) != CALIDROP_OK || kv_len_max < 1) return 0;
+  return make_decode_ws(p).per_layer;
+}
+
+int calidrop_decode_workspace_init(void* workspace, size_t workspace_bytes, void* stream) {
+  if (!workspace) return CALIDROP_INVALID_ARG;
+  cudaError_t e = cudaMemsetAsync(workspace, 0, workspace_bytes, (cudaStream_t)stream);
+  return e == cudaSuccess ? CALIDROP_OK : cuda_fail(e);
+}
+
+int calidrop_decode_batched(const calidrop_params* p, int32_t n_layers, const calidrop_decode_layer* layers,
+                            int32_t kv_len, void* workspace, size_t workspace_bytes, void* stream) {
+  int rc = check_common(p);
+  if (rc != CALIDROP_OK) return rc;
+  if (!layers || n_layers < 1 || n_layers > CALIDROP_MAX_LAYERS) return CALIDROP_INVALID_ARG;
+  if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u)) return CALIDROP_INVALID_ARG;
+  if (kv_len < 0) return CALIDROP_INVALID_ARG;
+  const bool has_new = layers[0].k_new != nullptr;
+  const int n_kv = kv_len + (has_new ? 1 : 0);
+  if (n_kv < 1 || n_kv > p->cap) return CALIDROP_INVALID_ARG;
+  for (int i = 0; i < n_layers; ++i) {
+    const calidrop_decode_layer& L = layers[i];
+    const void* req[] = {L.q, L.K_kept, L.V_kept, L.O_c, L.LSE_c, L.C_q, L.out};
+    for (const void* q : req)
+      if (!q || !aligned16(q)) return CALIDROP_INVALID_ARG;
+    if ((L.k_new != nullptr) != has_new || (L.v_new != nullptr) != has_new) return CALIDROP_INVALID_ARG;
+    if (has_new && (!aligned16(L.k_new) || !aligned16(L.v_new))) return CALIDROP_INVALID_ARG;
+  }
+  const DecodeWs w = make_decode_ws(p);
+  if (workspace_bytes < w.per_layer * (size_t)n_layers) return CALIDROP_WORKSPACE_TOO_SMALL;
+  if (!device_supported()) return CALIDROP_UNSUPPORTED;
+
+  DecodeArgs a{};
+  a.B = p->B; a.Hq = p->Hq; a.Hkv = p->Hkv; a.G = p->Hq / p->Hkv; a.n_cal = p->n_cal; a.cap = p->cap;
+  a.kv_len = kv_len; a.n_kv = n_kv; a.has_new = has_new ? 1 : 0;
+  a.units = p->B * p->Hkv; a.n_layers = n_layers;
+  a.nsplit = decode_nsplit(a.units * n_layers, n_kv);
+  if (a.nsplit > w.max_split) a.nsplit = w.max_split;
+  a.rows_per_split = (n_kv + a.nsplit - 1) / a.nsplit;
+  a.nsplit = (n_kv + a.rows_per_split - 1) / a.rows_per_split;
+  a.scale2 = scale2_of(p);
+  a.theta1 = p->theta1; a.theta2 = p->theta2; a.always_apply = p->theta2 <= -1.0f;
+  // The workspace is laid out array by array with the layer index outermost inside each
+  // array, so it is carved for n_layers at once.
+  char* base = (char*)workspace;
+  const size_t nl = (size_t)n_layers;
+  size_t off = 0;
+  a.counters = (unsigned*)(base + off); off += align_up((size_t)a.units * 4 * kDecodeMaxLayers, 256);
+  a.part_ml = (float*)(base + off);     off += align_up((size_t)a.units * a.nsplit * kMaxG * 2 * 4 * nl, 256);
+  a.rho = (float*)(base + off);         off += align_up((size_t)a.units * kMaxG * p->n_cal * 4 * nl, 256);
+  a.part_o = (float*)(base + off);
+  for (int i = 0; i < n_layers; ++i) {
+    const calidrop_decode_layer& L = layers[i];
+    a.layer[i] = DecodeLayerPtrs{L.q, L.k_new, L.v_new, L.K_kept, L.V_kept, L.O_c, L.LSE_c, L.C_q,
+                                 L.out, L.lse_out, L.flags};
+  }
+  cudaError_t e = launch_decode(a, (cudaStream_t)stream);
+  return e == cudaSuccess ? CALIDROP_OK : cuda_fail(e);
+}
+
+int calidrop_decode(const calidrop_params* p, const void* q, const void* k_new, const void* v_new,
+                    void* K_kept, void* V_kept, int32_t kv_len, const float* O_c, const float* LSE_c,
+                    const void* C_q, void* out, float* lse_out, uint8_t* flags, void* workspace,
+                    size_t workspace_bytes, void* stream) {
+  calidrop_decode_layer L{q, k_new, v_new, K_kept, V_kept, O_c, LSE_c, C_q, out, lse_out, flags};
+  return calidrop_decode_batched(p, 1, &L, kv_len, workspace, workspace_bytes, stream);
+}
+
+int calidrop_compress_host(const calidrop_params* p, const void* Q_obs_h, const void* K_h, const void* V_h,
+                           const float* lse_obs_h, int32_t* kept_idx_h, float* O_c_h, float* LSE_c_h,
+                           void* Q_obs, void* K, void* V, float* lse_obs, int32_t* kept_idx, void* K_kept,
+                           void* V_kept, float* O_c, float* LSE_c, void* C_q, void* workspace,
+                           size_t workspace_bytes, void* stream) {
+  int rc = check_compress(p);
+  if (rc != CALIDROP_OK) return rc;
+  if (!Q_obs_h || !K_h || !V_h || !kept_idx_h || !O_c_h || !LSE_c_h) return CALIDROP_INVALID_ARG;
+  if (!Q_obs || !K || !V || !kept_idx || !K_kept || !V_kept || !O_c || !LSE_c || !C_q || !workspace)
+    return CALIDROP_INVALID_ARG;
+  if (lse_obs_h && !lse_obs) return CALIDROP_INVALID_ARG;
+  if (workspace_bytes < calidrop_compress_workspace_bytes(p)) return CALIDROP_WORKSPACE_TOO_SMALL;
+  cudaStream_t st = (cudaStream_t)stream;
+  const size_t q_bytes = (size_t)p->B * p->Hq * p->window * kD * 2;
+  const size_t kv_bytes = (size_t)p->B * p->Hkv * p->L * kD * 2;
+  const size_t n_kept = p->budget < p->L ? p->budget : p->L;
+  cudaError_t e;
+  if ((e = cudaMemcpyAsync(Q_obs, Q_obs_h, q_bytes, cudaMemcpyHostToDevice, st)) != cudaSuccess) return cuda_fail(e);
+  if ((e = cudaMemcpyAsync(K, K_h, kv_bytes, cudaMemcpyHostToDevice, st)) != cudaSuccess) return cuda_fail(e);
+  if ((e = cudaMemcpyAsync(V, V_h, kv_bytes, cudaMemcpyHostToDevice, st)) != cudaSuccess) return cuda_fail(e);
+  if (lse_obs_h) {
+    e = cudaMemcpyAsync(lse_obs, lse_obs_h, (size_t)p->B * p->Hq * p->window * 4, cudaMemcpyHostToDevice, st);
+    if (e != cudaSuccess) return cuda_fail(e);
+  }
+  rc = calidrop_compress(p, Q_obs, K, V, lse_obs_h ? lse_obs : nullptr, kept_idx, K_kept, V_kept, O_c, LSE_c,
+                         C_q, workspace, workspace_bytes, stream);
+  if (rc != CALIDROP_OK) return rc;
+  if ((e = cudaMemcpyAsync(kept_idx_h, kept_idx, (size_t)p->B * p->Hkv * n_kept * 4, cudaMemcpyDeviceToHost, st)) != cudaSuccess) return cuda_fail(e);
+  if ((e = cudaMemcpyAsync(O_c_h, O_c, (size_t)p->B * p->Hq * p->n_cal * kD * 4, cudaMemcpyDeviceToHost, st)) != cudaSuccess) return cuda_fail(e);
+  if ((e = cudaMemcpyAsync(LSE_c_h, LSE_c, (size_t)p->B * p->Hq * p->n_cal * 4, cudaMemcpyDeviceToHost, st)) != cudaSuccess) return cuda_fail(e);
+  return CALIDROP_OK;
+}
+
+int calidrop_decode_host(const calidrop_params* p, const void* q_h, const void* k_new_h, const void* v_new_h,
+                         void* out_h, float* lse_out_h, uint8_t* flags_h, void* q, void* k_new, void* v_new,
+                         void* K_kept, void* V_kept, int32_t kv_len, const float* O_c, const float* LSE_c,
+                         const void* C_q, void* out, float* lse_out, uint8_t* flags, void* workspace,
+                         size_t workspace_bytes, void* stream) {
+  int rc = check_common(p);
+  if (rc != CALIDROP_OK) return rc;
+  if (!q_h || !out_h || !q || !out) return CALIDROP_INVALID_ARG;
+  if ((k_new_h != nullptr) != (v_new_h != nullptr)) return CALIDROP_INVALID_ARG;
+  if (k_new_h && (!k_new || !v_new)) return CALIDROP_INVALID_ARG;
+  if ((lse_out_h && !lse_out) || (flags_h && !flags)) return CALIDROP_INVALID_ARG;
+  cudaStream_t st = (cudaStream_t)stream;
+  const size_t q_bytes = (size_t)p->B * p->Hq * kD * 2;
+  const size_t kv_bytes = (size_t)p->B * p->Hkv * kD * 2;
+  cudaError_t e;
+  if ((e = cudaMemcpyAsync(q, q_h, q_bytes, cudaMemcpyHostToDevice, st)) != cudaSuccess) return cuda_fail(e);
+  if (k_new_h) {
+    if ((e = cudaMemcpyAsync(k_new, k_new_h, kv_bytes, cudaMemcpyHostToDevice, st)) != cudaSuccess) return cuda_fail(e);
+    if ((e = cudaMemcpyAsync(v_new, v_new_h, kv_bytes, cudaMemcpyHostToDevice, st)) != cudaSuccess) return cuda_fail(e);
+  }
+  rc = calidrop_decode(p, q, k_new_h ? k_new : nullptr, k_new_h ? v_new : nullptr, K_kept, V_kept, kv_len, O_c,
+                       LSE_c, C_q, out, lse_out, flags, workspace, workspace_bytes, stream);
+  if (rc != CALIDROP_OK) return rc;
+  if ((e = cudaMemcpyAsync(out_h, out, q_bytes, cudaMemcpyDeviceToHost, st)) != cudaSuccess) return cuda_fail(e);
+  if (lse_out_h && (e = cudaMemcpyAsync(lse_out_h, lse_out, (size_t)p->B * p->Hq * 4, cudaMemcpyDeviceToHost, st)) != cudaSuccess) return cuda_fail(e);
+  if (flags_h && (e = cudaMemcpyAsync(flags_h, flags, (size_t)p->B * p->Hq, cudaMemcpyDeviceToHost, st)) != cudaSuccess) return cuda_fail(e);
+  return CALIDROP_OK;
+}
+
+const char* calidrop_status_string(int status) {
+  switch (status) {
+    case CALIDROP_OK: return "ok";
+    case CALIDROP_INVALID_ARG: return "invalid argument";
+    case CALIDROP_UNSUPPORTED: return "unsupported configuration or device";
+    case CALIDROP_WORKSPACE_TOO_SMALL: return "workspace too small";
+    case CALIDROP_CUDA_ERROR: return g_err_text[0] ? g_err_text : "CUDA error";
+    default: return "unknown status";
+  }
+}
+
+int calidrop_version(void) { return 100; }
+
+uint64_t calidrop_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+}  // extern "C"

@@ -1,0 +1,310 @@
+// Decode-time attention over the compacted retained cache, merged with the calibration term.
+//
+// One launch covers: the append of the step's new K/V row, a split-K flash-decode over the
+// retained rows with the G query heads of a kv group packed into one MMA tile (so every K/V
+// byte is read once for all of them), the cosine similarity of the query with the stored
+// calibration queries, the threshold gate, and the merge of Eq. 1-2.  The work is bound by
+// HBM traffic (about 2G flop per byte), so the contraction uses the warp-level mma.sync path
+// with G <= 8 rows of a 16-row tile; tcgen05 tiles (64 rows minimum) would add nothing here.
+//
+// Grid: (split, batch*kv-head, layer).  Each CTA streams its slice of rows through
+// shared memory with 16-byte cp.async copies (XOR-swizzled so ldmatrix is conflict-free),
+// four warps each running an independent online softmax over interleaved 16-row blocks.
+// Per-split partial results go to the workspace; the CTA that arrives last at a per-unit
+// ticket counter combines them and applies gate and merge.  No CTA ever waits on another.
+#include "common.cuh"
+#include "internal.h"
+
+namespace calidrop {
+
+namespace {
+
+constexpr int kWarps = 4;
+constexpr int kThreads = kWarps * 32;
+constexpr int kBlkRows = 16;                         // rows per pipeline stage of one warp
+constexpr int kStages = 3;
+constexpr int kStageBytes = 2 * kBlkRows * kRowBytes;  // K block then V block
+constexpr int kWarpSmem = kStages * kStageBytes;       // 24 KB
+constexpr int kSmemBytes = kWarps * kWarpSmem;         // 96 KB -> two CTAs per SM
+
+__device__ __forceinline__ uint32_t swz(int row, int chunk) {
+  return (uint32_t)(row * kRowBytes + ((chunk ^ (row & 7)) << 4));
+}
+
+__global__ void __launch_bounds__(kThreads, 2) decode_kernel(const __grid_constant__ DecodeArgs a) {
+  extern __shared__ __align__(128) unsigned char smem[];
+  __shared__ int s_ticket;
+  __shared__ int s_cstar[kMaxG];
+  __shared__ float s_rho[kMaxG];
+
+  const int split = blockIdx.x, unit = blockIdx.y, layer = blockIdx.z;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int gq = lane >> 2, tq = lane & 3;  // MMA fragment coordinates
+  const DecodeLayerPtrs& P = a.layer[layer];
+  const int b = unit / a.Hkv, h = unit % a.Hkv;
+  const int hq0 = b * a.Hq + h * a.G;  // first query head of this kv group
+  const size_t lu = (size_t)layer * a.units + unit;
+
+  const __nv_bfloat16* q = (const __nv_bfloat16*)P.q;
+  const unsigned char* Kc = (const unsigned char*)P.K + (size_t)unit * a.cap * kRowBytes;
+  const unsigned char* Vc = (const unsigned char*)P.V + (size_t)unit * a.cap * kRowBytes;
+  const unsigned char* k_new = (const unsigned char*)P.k_new + (size_t)unit * kRowBytes;
+  const unsigned char* v_new = (const unsigned char*)P.v_new + (size_t)unit * kRowBytes;
+
+  const int r0 = split * a.rows_per_split;
+  const int r1 = min(a.n_kv, r0 + a.rows_per_split);
+  const int nblk = r1 > r0 ? (r1 - r0 + kBlkRows - 1) / kBlkRows : 0;
+  const int my_blocks = nblk > warp ? (nblk - warp + kWarps - 1) / kWarps : 0;
+
+  unsigned char* wsm = smem + warp * kWarpSmem;
+  const uint32_t wsm_u32 = smem_u32(wsm);
+
+  // ---- issue one 16-row block (K and V) of this warp into a stage
+  auto issue = [&](int i, int stage) {
+    const int row_base = r0 + (warp + i * kWarps) * kBlkRows;
+    const uint32_t dstK = wsm_u32 + stage * kStageBytes;
+    const uint32_t dstV = dstK + kBlkRows * kRowBytes;
+#pragma unroll
+    for (int it = 0; it < 8; ++it) {
+      const int idx = it * 32 + lane;
+      const int row = idx >> 4, chunk = idx & 15;
+      const int rg = row_base + row;
+      const bool valid = rg < r1;
+      const bool fresh = a.has_new && rg == a.kv_len;
+      const unsigned char* sk = fresh ? k_new + chunk * 16 : Kc + (size_t)(valid ? rg : 0) * kRowBytes + chunk * 16;
+      const unsigned char* sv = fresh ? v_new + chunk * 16 : Vc + (size_t)(valid ? rg : 0) * kRowBytes + chunk * 16;
+      cp_async_16(dstK + swz(row, chunk), sk, valid ? 16 : 0);
+      cp_async_16(dstV + swz(row, chunk), sv, valid ? 16 : 0);
+    }
+  };
+
+#pragma unroll
+  for (int s = 0; s < kStages - 1; ++s) {
+    if (s < my_blocks) issue(s, s);
+    cp_async_commit();
+  }
+
+  // ---- append: the CTA whose slice holds row kv_len stores the new K/V row into the cache
+  if (a.has_new && a.kv_len >= r0 && a.kv_len < r1 && warp == 0) {
+    const int chunk = lane & 15;
+    const unsigned char* src = (lane < 16 ? k_new : v_new) + chunk * 16;
+    unsigned char* dst = (unsigned char*)(lane < 16 ? P.K : P.V) +
+                         ((size_t)unit * a.cap + a.kv_len) * kRowBytes + chunk * 16;
+    *reinterpret_cast<uint4*>(dst) = *reinterpret_cast<const uint4*>(src);
+  }
+
+  // ---- cosine similarity of q with the calibration queries c = split, split + nsplit, ...
+  {
+    const __nv_bfloat16* Cq = (const __nv_bfloat16*)P.C_q;
+    const int n_c = a.n_cal > split ? (a.n_cal - split + a.nsplit - 1) / a.nsplit : 0;
+    const int pairs = n_c * a.G;
+    for (int pi = warp; pi < pairs; pi += kWarps) {
+      const int g = pi % a.G, c = split + (pi / a.G) * a.nsplit;
+      const uint2 qv = reinterpret_cast<const uint2*>(q + (size_t)(hq0 + g) * kD)[lane];
+      const uint2 cv = reinterpret_cast<const uint2*>(Cq + ((size_t)(hq0 + g) * a.n_cal + c) * kD)[lane];
+      const float q0 = bf16_lo(qv.x), q1 = bf16_hi(qv.x), q2 = bf16_lo(qv.y), q3 = bf16_hi(qv.y);
+      const float c0 = bf16_lo(cv.x), c1 = bf16_hi(cv.x), c2 = bf16_lo(cv.y), c3 = bf16_hi(cv.y);
+      float dot = q0 * c0 + q1 * c1 + q2 * c2 + q3 * c3;
+      float qq = q0 * q0 + q1 * q1 + q2 * q2 + q3 * q3;
+      float cc = c0 * c0 + c1 * c1 + c2 * c2 + c3 * c3;
+      dot = warp_sum(dot); qq = warp_sum(qq); cc = warp_sum(cc);
+      if (lane == 0)
+        a.rho[(lu * kMaxG + g) * a.n_cal + c] = (qq > 0.f && cc > 0.f) ? dot / (sqrtf(qq) * sqrtf(cc)) : 0.f;
+    }
+  }
+
+  // ---- query fragments: rows 0..G-1 of a 16-row A tile, the rest zero
+  uint32_t qa[kD / 16][2];
+#pragma unroll
+  for (int kk = 0; kk < kD / 16; ++kk) {
+    qa[kk][0] = 0u; qa[kk][1] = 0u;
+    if (gq < a.G) {
+      const uint32_t* qr = reinterpret_cast<const uint32_t*>(q + (size_t)(hq0 + gq) * kD + kk * 16);
+      qa[kk][0] = qr[tq];
+      qa[kk][1] = qr[4 + tq];
+    }
+  }
+
+  float o[kD / 8][4];
+#pragma unroll
+  for (int n = 0; n < kD / 8; ++n) { o[n][0] = o[n][1] = o[n][2] = o[n][3] = 0.f; }
+  float m = -INFINITY, l = 0.f;
+
+  for (int i = 0; i < my_blocks; ++i) {
+    const int nxt = i + kStages - 1;
+    if (nxt < my_blocks) issue(nxt, nxt % kStages);
+    cp_async_commit();
+    cp_async_wait<kStages - 1>();
+    __syncwarp();
+
+    const uint32_t sK = wsm_u32 + (i % kStages) * kStageBytes;
+    const uint32_t sV = sK + kBlkRows * kRowBytes;
+    const int row_base = r0 + (warp + i * kWarps) * kBlkRows;
+
+    // S = Q K^T for 16 keys: two n8 tiles
+    float s0[4] = {0.f, 0.f, 0.f, 0.f}, s1[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+    for (int kk = 0; kk < kD / 16; ++kk) {
+      const int mid = lane >> 3;
+      const int row = (lane & 7) + (mid >> 1) * 8;
+      const int chunk = kk * 2 + (mid & 1);
+      uint32_t b0, b1, b2, b3;
+      ldmatrix_x4(sK + swz(row, chunk), b0, b1, b2, b3);
+      mma_bf16_16816(s0, qa[kk][0], 0u, qa[kk][1], 0u, b0, b1);
+      mma_bf16_16816(s1, qa[kk][0], 0u, qa[kk][1], 0u, b2, b3);
+    }
+    // online softmax on row gq (keys 2tq, 2tq+1, 8+2tq, 9+2tq of this block)
+    const int kb = row_base + 2 * tq;
+    float x0 = kb < r1 ? s0[0] * a.scale2 : -INFINITY;
+    float x1 = kb + 1 < r1 ? s0[1] * a.scale2 : -INFINITY;
+    float x2 = kb + 8 < r1 ? s1[0] * a.scale2 : -INFINITY;
+    float x3 = kb + 9 < r1 ? s1[1] * a.scale2 : -INFINITY;
+    float bm = fmaxf(fmaxf(x0, x1), fmaxf(x2, x3));
+    bm = fmaxf(bm, __shfl_xor_sync(0xffffffffu, bm, 1));
+    bm = fmaxf(bm, __shfl_xor_sync(0xffffffffu, bm, 2));
+    const float m_new = fmaxf(m, bm);  // finite: every processed block has a valid first row
+    const float corr = ex2_approx(m - m_new);
+    const float p0 = ex2_approx(x0 - m_new), p1 = ex2_approx(x1 - m_new);
+    const float p2 = ex2_approx(x2 - m_new), p3 = ex2_approx(x3 - m_new);
+    l = l * corr + (p0 + p1) + (p2 + p3);
+    m = m_new;
+#pragma unroll
+    for (int n = 0; n < kD / 8; ++n) { o[n][0] *= corr; o[n][1] *= corr; }
+    const uint32_t pa0 = pack_bf16(p0, p1), pa2 = pack_bf16(p2, p3);
+    // O += P V
+#pragma unroll
+    for (int n = 0; n < kD / 8; n += 2) {
+      const int mid = lane >> 3;
+      const int row = (lane & 7) + (mid & 1) * 8;
+      const int chunk = n + (mid >> 1);
+      uint32_t b0, b1, b2, b3;
+      ldmatrix_x4_trans(sV + swz(row, chunk), b0, b1, b2, b3);
+      mma_bf16_16816(o[n], pa0, 0u, pa2, 0u, b0, b1);
+      mma_bf16_16816(o[n + 1], pa0, 0u, pa2, 0u, b2, b3);
+    }
+    __syncwarp();  // the stage is refilled by the next iteration's cp.async
+  }
+  cp_async_wait<0>();
+  l += __shfl_xor_sync(0xffffffffu, l, 1);
+  l += __shfl_xor_sync(0xffffffffu, l, 2);
+  __syncthreads();  // all warps are done with their stages: reuse them for the combine
+
+  // ---- CTA combine of the four warps
+  float* wo = reinterpret_cast<float*>(smem);                 // [warp][8][128]
+  float* wml = wo + kWarps * kMaxG * kD;                       // [warp][8][2]
+  if (gq < kMaxG) {
+#pragma unroll
+    for (int n = 0; n < kD / 8; ++n) {
+      float2 v = make_float2(o[n][0], o[n][1]);
+      *reinterpret_cast<float2*>(wo + ((warp * kMaxG + gq) * kD + n * 8 + 2 * tq)) = v;
+    }
+    if (tq == 0) { wml[(warp * kMaxG + gq) * 2] = m; wml[(warp * kMaxG + gq) * 2 + 1] = l; }
+  }
+  __syncthreads();
+  const int d = tid;  // one output dimension per thread
+  float* part_o = a.part_o + ((lu * a.nsplit + split) * kMaxG) * kD;
+  float* part_ml = a.part_ml + ((lu * a.nsplit + split) * kMaxG) * 2;
+  for (int g = 0; g < a.G; ++g) {
+    float M = -INFINITY;
+#pragma unroll
+    for (int w = 0; w < kWarps; ++w) M = fmaxf(M, wml[(w * kMaxG + g) * 2]);
+    float Lsum = 0.f, acc = 0.f;
+#pragma unroll
+    for (int w = 0; w < kWarps; ++w) {
+      const float mw = wml[(w * kMaxG + g) * 2];
+      const float sc = mw > -INFINITY ? ex2_approx(mw - M) : 0.f;
+      Lsum += wml[(w * kMaxG + g) * 2 + 1] * sc;
+      acc += wo[(w * kMaxG + g) * kD + d] * sc;
+    }
+    __stcg(part_o + g * kD + d, acc);
+    if (d == 0) { __stcg(part_ml + g * 2, M); __stcg(part_ml + g * 2 + 1, Lsum); }
+  }
+
+  // ---- ticket: the CTA that arrives last for this (layer, unit) finishes the job
+  __threadfence();
+  __syncthreads();
+  if (tid == 0) s_ticket = (int)atomicAdd(a.counters + lu, 1u);
+  __syncthreads();
+  if (s_ticket != a.nsplit - 1) return;
+  __threadfence();
+
+  // choice of the calibration row: highest cosine similarity, ties to the largest c
+  for (int g = warp; g < a.G; g += kWarps) {
+    float best = -INFINITY;
+    int bc = 0;
+    for (int c = lane; c < a.n_cal; c += 32) {
+      const float r = __ldcg(a.rho + (lu * kMaxG + g) * a.n_cal + c);
+      if (r >= best) { best = r; bc = c; }
+    }
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) {
+      const float ob = __shfl_xor_sync(0xffffffffu, best, off);
+      const int oc = __shfl_xor_sync(0xffffffffu, bc, off);
+      if (ob > best || (ob == best && oc > bc)) { best = ob; bc = oc; }
+    }
+    if (lane == 0) { s_cstar[g] = bc; s_rho[g] = best; }
+  }
+  __syncthreads();
+
+  // stage every split's (max, sum) pair in shared memory, then accumulate the partial outputs
+  const float* po = a.part_o + (lu * a.nsplit) * kMaxG * kD;
+  const float* pml = a.part_ml + (lu * a.nsplit) * kMaxG * 2;
+  float* ml_s = reinterpret_cast<float*>(smem) + kWarps * kMaxG * kD + kWarps * kMaxG * 2;  // [split][8][2]
+  for (int i = tid; i < a.nsplit * kMaxG * 2; i += kThreads) ml_s[i] = __ldcg(pml + i);
+  __syncthreads();
+  for (int g = 0; g < a.G; ++g) {
+    float M = -INFINITY;
+    for (int s = 0; s < a.nsplit; ++s) M = fmaxf(M, ml_s[(s * kMaxG + g) * 2]);
+    float Lsum = 0.f, acc = 0.f;
+#pragma unroll 4
+    for (int s = 0; s < a.nsplit; ++s) {
+      const float ms = ml_s[(s * kMaxG + g) * 2];
+      const float sc = ms > -INFINITY ? ex2_approx(ms - M) : 0.f;
+      Lsum += ml_s[(s * kMaxG + g) * 2 + 1] * sc;
+      acc += __ldcg(po + (s * kMaxG + g) * kD + d) * sc;
+    }
+    float outv = acc / Lsum;             // O_a
+    float lse2 = M + log2f(Lsum);        // LSE_a in the log2 domain
+    const int hq = hq0 + g;
+    const int cs = s_cstar[g];
+    const float rho = s_rho[g];
+    const float lse_c = P.LSE_c[(size_t)hq * a.n_cal + cs];
+    bool apply = (a.always_apply || rho > a.theta2) && (lse_c > -INFINITY);
+    if (apply) {
+      const float lc2 = lse_c * kLog2e;
+      const float mx = fmaxf(lse2, lc2);
+      const float ea = exp2f(lse2 - mx), ec = exp2f(lc2 - mx);
+      const float tot = ea + ec;
+      const float oc = P.O_c[((size_t)hq * a.n_cal + cs) * kD + d];
+      outv = (ea * outv + ec * oc) / tot;   // alpha_i O_a + alpha_j O_c   (Eq. 1-2)
+      lse2 = mx + log2f(tot);
+    }
+    reinterpret_cast<__nv_bfloat16*>(P.out)[(size_t)hq * kD + d] = __float2bfloat16_rn(outv);
+    if (d == 0) {
+      if (P.lse_out) P.lse_out[hq] = lse2 * kLn2;
+      if (P.flags)
+        P.flags[hq] = (uint8_t)((apply ? 1 : 0) | (rho < a.theta1 ? 2 : 0) | (a.n_cal <= 64 ? (cs << 2) : 0));
+    }
+  }
+  if (tid == 0) a.counters[lu] = 0u;  // ready for the next call
+}
+
+}  // namespace
+
+cudaError_t launch_decode(const DecodeArgs& a, cudaStream_t st) {
+  static bool attr_set[64] = {};
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  if (dev < 0 || dev >= 64 || !attr_set[dev]) {
+    e = cudaFuncSetAttribute(decode_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+    if (e != cudaSuccess) return e;
+    if (dev >= 0 && dev < 64) attr_set[dev] = true;
+  }
+  dim3 grid(a.nsplit, a.units, a.n_layers);
+  decode_kernel<<<grid, kThreads, kSmemBytes, st>>>(a);
+  count_launch(1);
+  return cudaGetLastError();
+}
+
+}  // namespace calidrop

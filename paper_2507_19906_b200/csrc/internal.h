@@ -1,0 +1,77 @@
+// Internal launcher interface between the C-ABI layer (api.cu) and the kernels.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+namespace calidrop {
+
+// Geometry of one compress call, derived from calidrop_params on the host.
+struct CompressGeom {
+  int B, Hq, Hkv, G, L, W, pool, budget, n_cal, cap;
+  int n_cand;   // L - W candidates per unit (0 when everything is kept)
+  int k_sel;    // budget - W selected candidates
+  int n_kept;   // min(budget, L)
+  int keep_all; // budget >= L
+  int units;    // B * Hkv
+  int bitmap_words;  // ceil(L / 32) per unit
+  float scale2;      // softmax scale * log2(e)
+};
+
+// Workspace carving of compress (byte offsets, all 256-byte aligned).
+struct CompressWs {
+  size_t vote, pooled, row_lse, bitmap, stat_part, total;
+  int n_tiles;  // 128-key tiles per unit for the partial row statistics
+};
+
+struct DecodeLayerPtrs {
+  const void* q;
+  const void* k_new;
+  const void* v_new;
+  void* K;
+  void* V;
+  const float* O_c;
+  const float* LSE_c;
+  const void* C_q;
+  void* out;
+  float* lse_out;
+  uint8_t* flags;
+};
+
+constexpr int kDecodeMaxLayers = 32;
+constexpr int kDecodeMaxSplit = 64;
+constexpr int kDecodeTargetCtas = 296;  // two resident CTAs on each of the 148 SMs
+
+struct DecodeArgs {
+  int B, Hq, Hkv, G, n_cal, cap, kv_len, n_kv, has_new;
+  int units, n_layers, nsplit, rows_per_split;
+  float scale2, theta1, theta2;
+  int always_apply;
+  // per-layer workspace arrays (element strides are implied by units / nsplit / n_cal)
+  float* part_o;       // [layer][unit][nsplit][8][128]
+  float* part_ml;      // [layer][unit][nsplit][8][2]
+  float* rho;          // [layer][unit][8][n_cal]
+  unsigned* counters;  // [layer][unit]
+  DecodeLayerPtrs layer[kDecodeMaxLayers];
+};
+
+// compress_simt.cu
+cudaError_t launch_row_stats(const CompressGeom& g, const CompressWs& ws, const void* Q_obs,
+                             const void* K, char* wsp, cudaStream_t st);
+cudaError_t launch_votes(const CompressGeom& g, const CompressWs& ws, const void* Q_obs, const void* K,
+                         const float* row_lse, char* wsp, cudaStream_t st);
+cudaError_t launch_calib_direct(const CompressGeom& g, const CompressWs& ws, const void* Q_obs,
+                                const void* K, const void* V, char* wsp, float* O_c, float* LSE_c,
+                                void* C_q, cudaStream_t st);
+// select.cu
+cudaError_t launch_pool_select(const CompressGeom& g, const CompressWs& ws, char* wsp,
+                               int32_t* kept_idx, cudaStream_t st);
+cudaError_t launch_gather(const CompressGeom& g, const void* K, const void* V, const int32_t* kept_idx,
+                          void* K_kept, void* V_kept, cudaStream_t st);
+// decode.cu
+cudaError_t launch_decode(const DecodeArgs& a, cudaStream_t st);
+
+void count_launch(int n = 1);
+
+}  // namespace calidrop

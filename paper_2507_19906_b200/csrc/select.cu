@@ -1,0 +1,205 @@
+// Pooling of the votes, per-(batch, kv-head) top-k selection with a deterministic
+// lowest-index tie rule, and gather-compaction of the kept K/V rows.
+//
+// Selection is an exact radix select on the fp32 bit patterns of the pooled votes (they are
+// non-negative, so unsigned order equals numeric order): four 8-bit histogram passes find the
+// value T of the k-th largest candidate and how many candidates equal to T still fit; one
+// ordered compaction pass then emits, in ascending position, every candidate above T plus the
+// first `need_eq` candidates equal to T.  No sort is needed because ascending position is
+// the storage order of the kept rows.
+#include "common.cuh"
+#include "internal.h"
+
+namespace calidrop {
+
+namespace {
+
+constexpr int kSelThreads = 1024;
+constexpr int kSelWarps = kSelThreads / 32;
+
+__global__ void __launch_bounds__(kSelThreads)
+pool_select_kernel(const float* __restrict__ vote, float* __restrict__ pooled,
+                   uint32_t* __restrict__ bitmap, int32_t* __restrict__ kept_idx, int n_cand, int L,
+                   int pool, int k_sel, int n_kept, int bitmap_words) {
+  __shared__ unsigned hist[kSelWarps][256];
+  __shared__ unsigned total[256];
+  __shared__ unsigned sel_bin, sel_k;
+  __shared__ unsigned warp_gt[kSelWarps], warp_eq[kSelWarps];
+
+  const int unit = blockIdx.x;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const float* v = vote + (size_t)unit * n_cand;
+  float* pl = pooled + (size_t)unit * n_cand;
+  uint32_t* bm = bitmap + (size_t)unit * bitmap_words;
+  int32_t* kept = kept_idx + (size_t)unit * n_kept;
+
+  // 1. zero-padded average pool with a constant divisor
+  const int half = pool >> 1;
+  const float fpool = (float)pool;
+  for (int t = tid; t < n_cand; t += kSelThreads) {
+    float acc = 0.f;
+    for (int d = -half; d <= half; ++d) {
+      int u = t + d;
+      if (u >= 0 && u < n_cand) acc += v[u];
+    }
+    pl[t] = acc / fpool;
+  }
+  __syncthreads();
+  const uint32_t* keys = reinterpret_cast<const uint32_t*>(pl);
+
+  // 2. radix select, most significant byte first
+  unsigned prefix = 0, k = (unsigned)k_sel;
+  for (int pass = 0; pass < 4; ++pass) {
+    const int shift = 24 - 8 * pass;
+    for (int i = tid; i < kSelWarps * 256; i += kSelThreads) (&hist[0][0])[i] = 0;
+    __syncthreads();
+    for (int t = tid; t < n_cand; t += kSelThreads) {
+      const unsigned key = keys[t];
+      const bool in = (pass == 0) || ((key >> (shift + 8)) == prefix);
+      if (in) atomicAdd(&hist[warp][(key >> shift) & 255u], 1u);
+    }
+    __syncthreads();
+    if (tid < 256) {
+      unsigned s = 0;
+#pragma unroll 8
+      for (int w = 0; w < kSelWarps; ++w) s += hist[w][tid];
+      total[tid] = s;
+    }
+    __syncthreads();
+    if (warp == 0) {
+      // lane 0 owns the 8 highest bins; walk bins downwards until k candidates are covered
+      const int base = 255 - 8 * lane;
+      unsigned c[8], s = 0;
+#pragma unroll
+      for (int j = 0; j < 8; ++j) { c[j] = total[base - j]; s += c[j]; }
+      unsigned incl = s;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        unsigned n = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += n;
+      }
+      const unsigned ball = __ballot_sync(0xffffffffu, incl >= k);
+      const int target = __ffs(ball) - 1;  // always found: the candidates number at least k
+      if (lane == target) {
+        unsigned run = incl - s;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+          if (run + c[j] >= k) { sel_bin = (unsigned)(base - j); sel_k = k - run; break; }
+          run += c[j];
+        }
+      }
+    }
+    __syncthreads();
+    prefix = (prefix << 8) | sel_bin;
+    k = sel_k;
+    __syncthreads();
+  }
+  const unsigned T = prefix;     // bit pattern of the k-th largest pooled vote
+  const unsigned need_eq = k;    // how many candidates equal to T are taken (lowest positions)
+
+  // 3. ordered compaction: thread i owns positions [i*per, (i+1)*per), per a multiple of 32
+  int per = (L + kSelThreads - 1) / kSelThreads;
+  per = (per + 31) & ~31;
+  const int t_begin = tid * per;
+  unsigned cnt_gt = 0, cnt_eq = 0;
+  for (int i = 0; i < per; ++i) {
+    const int t = t_begin + i;
+    if (t < n_cand) {
+      const unsigned key = keys[t];
+      cnt_gt += key > T;
+      cnt_eq += key == T;
+    }
+  }
+  unsigned inc_gt = cnt_gt, inc_eq = cnt_eq;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    unsigned a = __shfl_up_sync(0xffffffffu, inc_gt, o);
+    unsigned b = __shfl_up_sync(0xffffffffu, inc_eq, o);
+    if (lane >= o) { inc_gt += a; inc_eq += b; }
+  }
+  if (lane == 31) { warp_gt[warp] = inc_gt; warp_eq[warp] = inc_eq; }
+  __syncthreads();
+  unsigned before_gt = inc_gt - cnt_gt, before_eq = inc_eq - cnt_eq;
+  for (int w = 0; w < warp; ++w) { before_gt += warp_gt[w]; before_eq += warp_eq[w]; }
+
+  unsigned pos = before_gt + min(before_eq, need_eq);
+  unsigned eq_seen = before_eq;
+  for (int i0 = 0; i0 < per; i0 += 32) {
+    const int tw = t_begin + i0;
+    if (tw >= L) break;
+    uint32_t word = 0;
+    for (int i = 0; i < 32; ++i) {
+      const int t = tw + i;
+      bool take = false;
+      if (t < n_cand) {
+        const unsigned key = keys[t];
+        if (key > T) {
+          take = true;
+        } else if (key == T) {
+          take = eq_seen < need_eq;
+          ++eq_seen;
+        }
+        if (take) kept[pos++] = t;
+      } else if (t < L) {
+        take = true;  // observation-window rows are always kept
+      }
+      word |= (take ? 1u : 0u) << i;
+    }
+    bm[tw >> 5] = word;
+  }
+  // the window rows close the kept list
+  for (int j = tid; j < L - n_cand; j += kSelThreads) kept[k_sel + j] = n_cand + j;
+}
+
+// budget >= L: every row is kept.
+__global__ void keep_all_kernel(uint32_t* __restrict__ bitmap, int32_t* __restrict__ kept_idx, int L,
+                                int bitmap_words) {
+  const int unit = blockIdx.y;
+  const int t = blockIdx.x * blockDim.x + threadIdx.x;
+  if (t < L) kept_idx[(size_t)unit * L + t] = t;
+  if (t < bitmap_words) bitmap[(size_t)unit * bitmap_words + t] = 0xffffffffu;
+}
+
+// K_kept[u, i, :] = K[u, kept_idx[u, i], :], same for V; 16 lanes x 16 bytes per row.
+__global__ void __launch_bounds__(256)
+gather_kernel(const uint4* __restrict__ K, const uint4* __restrict__ V,
+              const int32_t* __restrict__ kept_idx, uint4* __restrict__ K_kept,
+              uint4* __restrict__ V_kept, int L, int n_kept, int cap) {
+  const int unit = blockIdx.y;
+  const int i = blockIdx.x * 16 + (threadIdx.x >> 4);
+  const int chunk = threadIdx.x & 15;
+  if (i >= n_kept) return;
+  const int t = kept_idx[(size_t)unit * n_kept + i];
+  const size_t src = ((size_t)unit * L + t) * 16 + chunk;
+  const size_t dst = ((size_t)unit * cap + i) * 16 + chunk;
+  K_kept[dst] = __ldg(K + src);
+  V_kept[dst] = __ldg(V + src);
+}
+
+}  // namespace
+
+cudaError_t launch_pool_select(const CompressGeom& g, const CompressWs& ws, char* wsp,
+                               int32_t* kept_idx, cudaStream_t st) {
+  if (g.keep_all) {
+    const int n = g.L > g.bitmap_words ? g.L : g.bitmap_words;
+    dim3 grid((n + 255) / 256, g.units);
+    keep_all_kernel<<<grid, 256, 0, st>>>((uint32_t*)(wsp + ws.bitmap), kept_idx, g.L, g.bitmap_words);
+  } else {
+    pool_select_kernel<<<g.units, kSelThreads, 0, st>>>(
+        (const float*)(wsp + ws.vote), (float*)(wsp + ws.pooled), (uint32_t*)(wsp + ws.bitmap), kept_idx,
+        g.n_cand, g.L, g.pool, g.k_sel, g.n_kept, g.bitmap_words);
+  }
+  count_launch(1);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_gather(const CompressGeom& g, const void* K, const void* V, const int32_t* kept_idx,
+                          void* K_kept, void* V_kept, cudaStream_t st) {
+  dim3 grid((g.n_kept + 15) / 16, g.units);
+  gather_kernel<<<grid, 256, 0, st>>>((const uint4*)K, (const uint4*)V, kept_idx, (uint4*)K_kept,
+                                      (uint4*)V_kept, g.L, g.n_kept, g.cap);
+  count_launch(1);
+  return cudaGetLastError();
+}
+
+}  // namespace calidrop

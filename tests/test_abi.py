@@ -1,0 +1,67 @@
+"""Host-side checks that need no GPU: the C-ABI library loads and exports what the header declares,
+and the size queries and status strings behave."""
+import ctypes
+import os
+import re
+
+import pytest
+
+from paper_2507_19906_b200 import binding as cd
+from paper_2507_19906_b200 import build as cdbuild
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def lib():
+    cdbuild.build()          # nvcc cross-compiles for sm_100a without a GPU
+    return cd.load()
+
+
+def declared_functions():
+    text = open(os.path.join(ROOT, "include", "calidrop.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(calidrop_[a-z_]+)\s*\(", text)))
+
+
+def test_library_exports_every_declared_symbol(lib):
+    names = declared_functions()
+    assert len(names) >= 12
+    for n in names:
+        assert hasattr(lib, n), f"{n} is declared in calidrop.h but not exported"
+    assert sorted(cd.EXPORTS) == names
+
+
+def test_binding_has_the_same_names():
+    for n in declared_functions():
+        if n == "calidrop_status_string":
+            assert hasattr(cd, "status_string")
+        else:
+            assert hasattr(cd, n), n
+
+
+def test_size_queries_and_status_strings(lib):
+    p = cd.make_params(B=4, Hq=32, Hkv=8, L=32768, window=64, pool=7, budget=2048, n_cal=64, cap=2176)
+    ws = cd.calidrop_compress_workspace_bytes(p)
+    assert ws >= 2 * 4 * 8 * (32768 - 64) * 4          # votes and pooled votes at least
+    assert ws % 256 == 0
+    assert cd.calidrop_decode_workspace_bytes(p, 2176) > 0
+    lay = cd.calidrop_compress_workspace_layout(p)
+    assert lay.vote_offset % 256 == 0 and lay.pooled_offset > lay.vote_offset
+    bad = cd.make_params(B=4, Hq=32, Hkv=8, L=32768, window=64, pool=6, budget=2048, n_cal=64, cap=2176)
+    assert cd.calidrop_compress_workspace_bytes(bad) == 0
+    assert cd.status_string(cd.OK) == "ok"
+    assert "workspace" in cd.status_string(cd.WORKSPACE_TOO_SMALL)
+    assert cd.calidrop_version() >= 100
+    assert ctypes.sizeof(cd.Params) == 13 * 4
+
+
+def test_null_arguments_are_rejected_before_any_cuda_call(lib):
+    """Validation is host-side and precedes every CUDA call, so it works without a device."""
+    p = cd.make_params(B=1, Hq=4, Hkv=2, L=300, window=8, pool=5, budget=40, n_cal=1, cap=40)
+    rc = lib.calidrop_compress(ctypes.byref(p), None, None, None, None, None, None, None, None, None, None,
+                               None, 0, None)
+    assert rc == cd.INVALID_ARG
+    rc = lib.calidrop_decode(ctypes.byref(p), None, None, None, None, None, 1, None, None, None, None, None,
+                             None, None, 0, None)
+    assert rc == cd.INVALID_ARG
