@@ -14,7 +14,8 @@ from dataclasses import dataclass
 import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libcalidrop.so")
+# CALIDROP_LIB selects another build of the same library (e.g. an instrumented one).
+LIB_PATH = os.environ.get("CALIDROP_LIB") or os.path.join(_HERE, "libcalidrop.so")
 _lib = None
 
 OK, INVALID_ARG, UNSUPPORTED, WORKSPACE_TOO_SMALL, CUDA_ERROR = 0, -1, -2, -3, -4

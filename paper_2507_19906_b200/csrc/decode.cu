@@ -12,6 +12,11 @@
 // four warps each running an independent online softmax over interleaved 16-row blocks.
 // Per-split partial results go to the workspace; the CTA that arrives last at a per-unit
 // ticket counter combines them and applies gate and merge.  No CTA ever waits on another.
+//
+// The kernel is latency-sensitive (tens of MB per launch), so dependent global round trips
+// are kept to a minimum: the small loads (query, calibration queries) are issued before the
+// K/V burst so they are not queued behind it, and the finishing CTA fetches everything it
+// needs in two waves (partials + statistics + similarities, then the chosen calibration row).
 #include "common.cuh"
 #include "internal.h"
 
@@ -21,14 +26,33 @@ namespace {
 
 constexpr int kWarps = 4;
 constexpr int kThreads = kWarps * 32;
-constexpr int kBlkRows = 16;                         // rows per pipeline stage of one warp
+constexpr int kBlkRows = 16;                           // rows per pipeline stage of one warp
 constexpr int kStages = 3;
 constexpr int kStageBytes = 2 * kBlkRows * kRowBytes;  // K block then V block
 constexpr int kWarpSmem = kStages * kStageBytes;       // 24 KB
 constexpr int kSmemBytes = kWarps * kWarpSmem;         // 96 KB -> two CTAs per SM
+constexpr int kRhoRegPasses = 2;                       // similarity passes whose loads are issued up front
+constexpr int kPairsPerPass = kThreads / 8;            // 8 lanes per (head, calibration row) pair
 
 __device__ __forceinline__ uint32_t swz(int row, int chunk) {
   return (uint32_t)(row * kRowBytes + ((chunk ^ (row & 7)) << 4));
+}
+
+struct RhoLoad {
+  uint4 q0, q1, c0, c1;
+};
+
+__device__ __forceinline__ void rho_accumulate(const RhoLoad& r, float& dot, float& qq, float& cc) {
+  const uint32_t qw[8] = {r.q0.x, r.q0.y, r.q0.z, r.q0.w, r.q1.x, r.q1.y, r.q1.z, r.q1.w};
+  const uint32_t cw[8] = {r.c0.x, r.c0.y, r.c0.z, r.c0.w, r.c1.x, r.c1.y, r.c1.z, r.c1.w};
+#pragma unroll
+  for (int j = 0; j < 8; ++j) {
+    const float a0 = bf16_lo(qw[j]), a1 = bf16_hi(qw[j]);
+    const float b0 = bf16_lo(cw[j]), b1 = bf16_hi(cw[j]);
+    dot = fmaf(a0, b0, fmaf(a1, b1, dot));
+    qq = fmaf(a0, a0, fmaf(a1, a1, qq));
+    cc = fmaf(b0, b0, fmaf(b1, b1, cc));
+  }
 }
 
 __global__ void __launch_bounds__(kThreads, 2) decode_kernel(const __grid_constant__ DecodeArgs a) {
@@ -46,6 +70,7 @@ __global__ void __launch_bounds__(kThreads, 2) decode_kernel(const __grid_consta
   const size_t lu = (size_t)layer * a.units + unit;
 
   const __nv_bfloat16* q = (const __nv_bfloat16*)P.q;
+  const __nv_bfloat16* Cq = (const __nv_bfloat16*)P.C_q;
   const unsigned char* Kc = (const unsigned char*)P.K + (size_t)unit * a.cap * kRowBytes;
   const unsigned char* Vc = (const unsigned char*)P.V + (size_t)unit * a.cap * kRowBytes;
   const unsigned char* k_new = (const unsigned char*)P.k_new + (size_t)unit * kRowBytes;
@@ -59,7 +84,50 @@ __global__ void __launch_bounds__(kThreads, 2) decode_kernel(const __grid_consta
   unsigned char* wsm = smem + warp * kWarpSmem;
   const uint32_t wsm_u32 = smem_u32(wsm);
 
-  // ---- issue one 16-row block (K and V) of this warp into a stage
+  // ---- (1) small loads first: query fragments (rows 0..G-1 of a 16-row A tile, the rest
+  // zero) and the calibration queries this CTA compares against (c = split, split+nsplit, ...)
+  uint32_t qa[kD / 16][2];
+#pragma unroll
+  for (int kk = 0; kk < kD / 16; ++kk) {
+    qa[kk][0] = 0u; qa[kk][1] = 0u;
+    if (gq < a.G) {
+      const uint32_t* qr = reinterpret_cast<const uint32_t*>(q + (size_t)(hq0 + gq) * kD + kk * 16);
+      qa[kk][0] = __ldg(qr + tq);
+      qa[kk][1] = __ldg(qr + 4 + tq);
+    }
+  }
+  const int n_c = a.n_cal > split ? (a.n_cal - split + a.nsplit - 1) / a.nsplit : 0;
+  const int pairs = n_c * a.G;
+  const int sub = tid & 7;
+  auto rho_load = [&](int pi, RhoLoad& r) {
+    const int g = pi % a.G, c = split + (pi / a.G) * a.nsplit;
+    const uint4* qp = reinterpret_cast<const uint4*>(q + (size_t)(hq0 + g) * kD + sub * 16);
+    const uint4* cp = reinterpret_cast<const uint4*>(Cq + ((size_t)(hq0 + g) * a.n_cal + c) * kD + sub * 16);
+    r.q0 = __ldg(qp); r.q1 = __ldg(qp + 1); r.c0 = __ldg(cp); r.c1 = __ldg(cp + 1);
+  };
+  auto rho_finish = [&](int pi, const RhoLoad& r) {
+    float dot = 0.f, qq = 0.f, cc = 0.f;
+    if (pi < pairs) rho_accumulate(r, dot, qq, cc);
+#pragma unroll
+    for (int o = 1; o < 8; o <<= 1) {
+      dot += __shfl_xor_sync(0xffffffffu, dot, o);
+      qq += __shfl_xor_sync(0xffffffffu, qq, o);
+      cc += __shfl_xor_sync(0xffffffffu, cc, o);
+    }
+    if (sub == 0 && pi < pairs) {
+      const int g = pi % a.G, c = split + (pi / a.G) * a.nsplit;
+      a.rho[(lu * kMaxG + g) * a.n_cal + c] = (qq > 0.f && cc > 0.f) ? dot / (sqrtf(qq) * sqrtf(cc)) : 0.f;
+    }
+  };
+  RhoLoad rl[kRhoRegPasses];
+#pragma unroll
+  for (int ps = 0; ps < kRhoRegPasses; ++ps) {
+    rl[ps] = RhoLoad{};
+    const int pi = ps * kPairsPerPass + (tid >> 3);
+    if (pi < pairs) rho_load(pi, rl[ps]);
+  }
+
+  // ---- (2) the K/V stream: issue one 16-row block (K and V) of this warp into a stage
   auto issue = [&](int i, int stage) {
     const int row_base = r0 + (warp + i * kWarps) * kBlkRows;
     const uint32_t dstK = wsm_u32 + stage * kStageBytes;
@@ -77,14 +145,13 @@ __global__ void __launch_bounds__(kThreads, 2) decode_kernel(const __grid_consta
       cp_async_16(dstV + swz(row, chunk), sv, valid ? 16 : 0);
     }
   };
-
 #pragma unroll
   for (int s = 0; s < kStages - 1; ++s) {
     if (s < my_blocks) issue(s, s);
     cp_async_commit();
   }
 
-  // ---- append: the CTA whose slice holds row kv_len stores the new K/V row into the cache
+  // ---- (3) append: the CTA whose slice holds row kv_len stores the new K/V row into the cache
   if (a.has_new && a.kv_len >= r0 && a.kv_len < r1 && warp == 0) {
     const int chunk = lane & 15;
     const unsigned char* src = (lane < 16 ? k_new : v_new) + chunk * 16;
@@ -93,38 +160,17 @@ __global__ void __launch_bounds__(kThreads, 2) decode_kernel(const __grid_consta
     *reinterpret_cast<uint4*>(dst) = *reinterpret_cast<const uint4*>(src);
   }
 
-  // ---- cosine similarity of q with the calibration queries c = split, split + nsplit, ...
-  {
-    const __nv_bfloat16* Cq = (const __nv_bfloat16*)P.C_q;
-    const int n_c = a.n_cal > split ? (a.n_cal - split + a.nsplit - 1) / a.nsplit : 0;
-    const int pairs = n_c * a.G;
-    for (int pi = warp; pi < pairs; pi += kWarps) {
-      const int g = pi % a.G, c = split + (pi / a.G) * a.nsplit;
-      const uint2 qv = reinterpret_cast<const uint2*>(q + (size_t)(hq0 + g) * kD)[lane];
-      const uint2 cv = reinterpret_cast<const uint2*>(Cq + ((size_t)(hq0 + g) * a.n_cal + c) * kD)[lane];
-      const float q0 = bf16_lo(qv.x), q1 = bf16_hi(qv.x), q2 = bf16_lo(qv.y), q3 = bf16_hi(qv.y);
-      const float c0 = bf16_lo(cv.x), c1 = bf16_hi(cv.x), c2 = bf16_lo(cv.y), c3 = bf16_hi(cv.y);
-      float dot = q0 * c0 + q1 * c1 + q2 * c2 + q3 * c3;
-      float qq = q0 * q0 + q1 * q1 + q2 * q2 + q3 * q3;
-      float cc = c0 * c0 + c1 * c1 + c2 * c2 + c3 * c3;
-      dot = warp_sum(dot); qq = warp_sum(qq); cc = warp_sum(cc);
-      if (lane == 0)
-        a.rho[(lu * kMaxG + g) * a.n_cal + c] = (qq > 0.f && cc > 0.f) ? dot / (sqrtf(qq) * sqrtf(cc)) : 0.f;
-    }
-  }
-
-  // ---- query fragments: rows 0..G-1 of a 16-row A tile, the rest zero
-  uint32_t qa[kD / 16][2];
+  // ---- (4) cosine similarities (their loads are long in flight by now)
 #pragma unroll
-  for (int kk = 0; kk < kD / 16; ++kk) {
-    qa[kk][0] = 0u; qa[kk][1] = 0u;
-    if (gq < a.G) {
-      const uint32_t* qr = reinterpret_cast<const uint32_t*>(q + (size_t)(hq0 + gq) * kD + kk * 16);
-      qa[kk][0] = qr[tq];
-      qa[kk][1] = qr[4 + tq];
-    }
+  for (int ps = 0; ps < kRhoRegPasses; ++ps) rho_finish(ps * kPairsPerPass + (tid >> 3), rl[ps]);
+  for (int base = kRhoRegPasses * kPairsPerPass; base < pairs; base += kPairsPerPass) {
+    const int pi = base + (tid >> 3);
+    RhoLoad r{};
+    if (pi < pairs) rho_load(pi, r);
+    rho_finish(pi, r);
   }
 
+  // ---- (5) main loop
   float o[kD / 8][4];
 #pragma unroll
   for (int n = 0; n < kD / 8; ++n) { o[n][0] = o[n][1] = o[n][2] = o[n][3] = 0.f; }
@@ -189,17 +235,13 @@ __global__ void __launch_bounds__(kThreads, 2) decode_kernel(const __grid_consta
   l += __shfl_xor_sync(0xffffffffu, l, 2);
   __syncthreads();  // all warps are done with their stages: reuse them for the combine
 
-  // ---- CTA combine of the four warps
-  float* wo = reinterpret_cast<float*>(smem);                 // [warp][8][128]
-  float* wml = wo + kWarps * kMaxG * kD;                       // [warp][8][2]
-  if (gq < kMaxG) {
+  // ---- (6) CTA combine of the four warps
+  float* wo = reinterpret_cast<float*>(smem);   // [warp][8][128]
+  float* wml = wo + kWarps * kMaxG * kD;         // [warp][8][2]
 #pragma unroll
-    for (int n = 0; n < kD / 8; ++n) {
-      float2 v = make_float2(o[n][0], o[n][1]);
-      *reinterpret_cast<float2*>(wo + ((warp * kMaxG + gq) * kD + n * 8 + 2 * tq)) = v;
-    }
-    if (tq == 0) { wml[(warp * kMaxG + gq) * 2] = m; wml[(warp * kMaxG + gq) * 2 + 1] = l; }
-  }
+  for (int n = 0; n < kD / 8; ++n)
+    *reinterpret_cast<float2*>(wo + ((warp * kMaxG + gq) * kD + n * 8 + 2 * tq)) = make_float2(o[n][0], o[n][1]);
+  if (tq == 0) { wml[(warp * kMaxG + gq) * 2] = m; wml[(warp * kMaxG + gq) * 2 + 1] = l; }
   __syncthreads();
   const int d = tid;  // one output dimension per thread
   float* part_o = a.part_o + ((lu * a.nsplit + split) * kMaxG) * kD;
@@ -220,14 +262,37 @@ __global__ void __launch_bounds__(kThreads, 2) decode_kernel(const __grid_consta
     if (d == 0) { __stcg(part_ml + g * 2, M); __stcg(part_ml + g * 2 + 1, Lsum); }
   }
 
-  // ---- ticket: the CTA that arrives last for this (layer, unit) finishes the job
-  __threadfence();
+  // ---- (7) ticket: the CTA that arrives last for this (layer, unit) finishes the job.
+  // The barrier orders every thread's stores before thread 0's device-scope fence (fences
+  // are cumulative), which in turn precedes the ticket increment.
   __syncthreads();
-  if (tid == 0) s_ticket = (int)atomicAdd(a.counters + lu, 1u);
+  if (tid == 0) {
+    __threadfence();
+    s_ticket = (int)atomicAdd(a.counters + lu, 1u);
+  }
   __syncthreads();
   if (s_ticket != a.nsplit - 1) return;
   __threadfence();
 
+  // ---- (8) finish: wave one fetches the split statistics, the similarities and the first
+  // chunk of partial outputs together; wave two the chosen calibration row.
+  const float* po = a.part_o + (lu * a.nsplit) * kMaxG * kD;
+  const float* pml = a.part_ml + (lu * a.nsplit) * kMaxG * 2;
+  float* ml_s = wml + kWarps * kMaxG * 2;  // [split][8][2]
+  const int n_items = a.G * (kD / 4);      // (head, 4 consecutive dims) items, one per thread
+  constexpr int kChunk = 8;
+  float4 pv[kChunk];
+  auto load_chunk = [&](int item, int s0) {
+    const int g = item >> 5, d4 = item & 31;
+#pragma unroll
+    for (int s = 0; s < kChunk; ++s) {
+      pv[s] = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (s0 + s < a.nsplit)
+        pv[s] = __ldcg(reinterpret_cast<const float4*>(po + ((s0 + s) * kMaxG + g) * kD) + d4);
+    }
+  };
+  if (tid < n_items) load_chunk(tid, 0);
+  for (int i = tid; i < a.nsplit * kMaxG * 2; i += kThreads) ml_s[i] = __ldcg(pml + i);
   // choice of the calibration row: highest cosine similarity, ties to the largest c
   for (int g = warp; g < a.G; g += kWarps) {
     float best = -INFINITY;
@@ -246,41 +311,49 @@ __global__ void __launch_bounds__(kThreads, 2) decode_kernel(const __grid_consta
   }
   __syncthreads();
 
-  // stage every split's (max, sum) pair in shared memory, then accumulate the partial outputs
-  const float* po = a.part_o + (lu * a.nsplit) * kMaxG * kD;
-  const float* pml = a.part_ml + (lu * a.nsplit) * kMaxG * 2;
-  float* ml_s = reinterpret_cast<float*>(smem) + kWarps * kMaxG * kD + kWarps * kMaxG * 2;  // [split][8][2]
-  for (int i = tid; i < a.nsplit * kMaxG * 2; i += kThreads) ml_s[i] = __ldcg(pml + i);
-  __syncthreads();
-  for (int g = 0; g < a.G; ++g) {
-    float M = -INFINITY;
-    for (int s = 0; s < a.nsplit; ++s) M = fmaxf(M, ml_s[(s * kMaxG + g) * 2]);
-    float Lsum = 0.f, acc = 0.f;
-#pragma unroll 4
-    for (int s = 0; s < a.nsplit; ++s) {
-      const float ms = ml_s[(s * kMaxG + g) * 2];
-      const float sc = ms > -INFINITY ? ex2_approx(ms - M) : 0.f;
-      Lsum += ml_s[(s * kMaxG + g) * 2 + 1] * sc;
-      acc += __ldcg(po + (s * kMaxG + g) * kD + d) * sc;
-    }
-    float outv = acc / Lsum;             // O_a
-    float lse2 = M + log2f(Lsum);        // LSE_a in the log2 domain
+  for (int item = tid; item < n_items; item += kThreads) {
+    const int g = item >> 5, d4 = item & 31;
     const int hq = hq0 + g;
     const int cs = s_cstar[g];
     const float rho = s_rho[g];
-    const float lse_c = P.LSE_c[(size_t)hq * a.n_cal + cs];
-    bool apply = (a.always_apply || rho > a.theta2) && (lse_c > -INFINITY);
+    const size_t crow = (size_t)hq * a.n_cal + cs;
+    const float lse_c = __ldg(P.LSE_c + crow);
+    const float4 oc = __ldg(reinterpret_cast<const float4*>(P.O_c + crow * kD) + d4);
+    float M = -INFINITY;
+    for (int s = 0; s < a.nsplit; ++s) M = fmaxf(M, ml_s[(s * kMaxG + g) * 2]);
+    float Lsum = 0.f;
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int s0 = 0; s0 < a.nsplit; s0 += kChunk) {
+      if (s0 > 0 || item != tid) load_chunk(item, s0);
+#pragma unroll
+      for (int s = 0; s < kChunk; ++s) {
+        if (s0 + s < a.nsplit) {
+          const float ms = ml_s[((s0 + s) * kMaxG + g) * 2];
+          const float sc = ms > -INFINITY ? ex2_approx(ms - M) : 0.f;
+          Lsum = fmaf(ml_s[((s0 + s) * kMaxG + g) * 2 + 1], sc, Lsum);
+          acc.x = fmaf(pv[s].x, sc, acc.x); acc.y = fmaf(pv[s].y, sc, acc.y);
+          acc.z = fmaf(pv[s].z, sc, acc.z); acc.w = fmaf(pv[s].w, sc, acc.w);
+        }
+      }
+    }
+    const float inv = 1.f / Lsum;
+    float4 outv = make_float4(acc.x * inv, acc.y * inv, acc.z * inv, acc.w * inv);  // O_a
+    float lse2 = M + log2f(Lsum);                                                   // LSE_a (log2 domain)
+    const bool apply = (a.always_apply || rho > a.theta2) && (lse_c > -INFINITY);
     if (apply) {
+      // alpha_i = e^{LSE_a - LSE}, alpha_j = e^{LSE_c - LSE}; out = alpha_i O_a + alpha_j O_c (Eq. 1-2)
       const float lc2 = lse_c * kLog2e;
       const float mx = fmaxf(lse2, lc2);
       const float ea = exp2f(lse2 - mx), ec = exp2f(lc2 - mx);
       const float tot = ea + ec;
-      const float oc = P.O_c[((size_t)hq * a.n_cal + cs) * kD + d];
-      outv = (ea * outv + ec * oc) / tot;   // alpha_i O_a + alpha_j O_c   (Eq. 1-2)
+      const float ai = ea / tot, aj = ec / tot;
+      outv = make_float4(ai * outv.x + aj * oc.x, ai * outv.y + aj * oc.y, ai * outv.z + aj * oc.z,
+                         ai * outv.w + aj * oc.w);
       lse2 = mx + log2f(tot);
     }
-    reinterpret_cast<__nv_bfloat16*>(P.out)[(size_t)hq * kD + d] = __float2bfloat16_rn(outv);
-    if (d == 0) {
+    uint2 packed = make_uint2(pack_bf16(outv.x, outv.y), pack_bf16(outv.z, outv.w));
+    reinterpret_cast<uint2*>(reinterpret_cast<__nv_bfloat16*>(P.out) + (size_t)hq * kD)[d4] = packed;
+    if (d4 == 0) {
       if (P.lse_out) P.lse_out[hq] = lse2 * kLn2;
       if (P.flags)
         P.flags[hq] = (uint8_t)((apply ? 1 : 0) | (rho < a.theta1 ? 2 : 0) | (a.n_cal <= 64 ? (cs << 2) : 0));
