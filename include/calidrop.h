@@ -43,8 +43,10 @@ extern "C" {
 #define CALIDROP_UNSUPPORTED (-2)         /* D != 128, Hq/Hkv > 8, device is not sm_100       */
 #define CALIDROP_WORKSPACE_TOO_SMALL (-3)
 #define CALIDROP_CUDA_ERROR (-4)          /* a launch or runtime call failed                  */
+#define CALIDROP_SCRATCH_LIMIT (-5)       /* needs more than CALIDROP_STATIC_SCRATCH_BYTES    */
 
 #define CALIDROP_MAX_LAYERS 32            /* layers per calidrop_decode_batched call          */
+#define CALIDROP_STATIC_SCRATCH_BYTES (4u << 20)  /* built-in scratch of calidrop_decode_static */
 
 typedef struct calidrop_params {
   int32_t B, Hq, Hkv, D;        /* D must be 128; Hq % Hkv == 0; G = Hq/Hkv <= 8              */
@@ -197,6 +199,39 @@ typedef struct calidrop_decode_layer {
 int calidrop_decode_batched(const calidrop_params* p, int32_t n_layers,
                             const calidrop_decode_layer* layers /* HOST */, int32_t kv_len,
                             void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * calidrop_decode for callers that cannot allocate device memory.  (The paper has no
+ * counterpart: this is a packaging variant of the same decode step, not another operation.)
+ *
+ * Some hosts of this library hand it inputs and outputs but have no way to give it a
+ * workspace: a plugin slot of an inference runtime whose memory planner was frozen before the
+ * library was loaded, a callback that runs where cudaMalloc is forbidden (inside a stream
+ * capture, or in a process whose device memory is owned entirely by another allocator), or
+ * code that must not fail for lack of memory.  For them the split-K scratch of the decode
+ * kernel lives in a fixed array of CALIDROP_STATIC_SCRATCH_BYTES (4 MiB) of device memory
+ * that is part of the library image: every GPU that loads the library holds it until the
+ * process exits, and this call, like the others, allocates and frees nothing.
+ *
+ * Arguments and results are exactly those of calidrop_decode without `workspace` and
+ * `workspace_bytes`; the two entry points run the same kernel with the same split factor.
+ *
+ *   - Limit: calidrop_decode_workspace_bytes(p, kv_len + 1) must not exceed
+ *     CALIDROP_STATIC_SCRATCH_BYTES (about B * Hkv <= 900 for n_cal = 64), otherwise the call
+ *     returns CALIDROP_SCRATCH_LIMIT and does nothing.
+ *   - The first call on each device looks the array's device address up and caches it.  Make
+ *     that first call outside any stream capture.
+ *   - All calls on a device share the one array and it keeps whatever the last call left.  The
+ *     part that must start at zero (the arrival counters) is cleared on `stream` ahead of the
+ *     kernel by every call.  Two calls that may overlap on the GPU (different streams without
+ *     an ordering between them) race on the array; serialise them, or give the overlapping
+ *     ones their own workspace through calidrop_decode.
+ */
+int calidrop_decode_static(const calidrop_params* p,
+                           const void* q, const void* k_new, const void* v_new,
+                           void* K_kept, void* V_kept, int32_t kv_len,
+                           const float* O_c, const float* LSE_c, const void* C_q,
+                           void* out, float* lse_out, uint8_t* flags, void* stream);
 
 /*
  * End-to-end variants for callers whose tensors live in HOST memory (pinned memory makes the

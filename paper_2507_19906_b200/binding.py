@@ -18,13 +18,14 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.environ.get("CALIDROP_LIB") or os.path.join(_HERE, "libcalidrop.so")
 _lib = None
 
-OK, INVALID_ARG, UNSUPPORTED, WORKSPACE_TOO_SMALL, CUDA_ERROR = 0, -1, -2, -3, -4
+OK, INVALID_ARG, UNSUPPORTED, WORKSPACE_TOO_SMALL, CUDA_ERROR, SCRATCH_LIMIT = 0, -1, -2, -3, -4, -5
+STATIC_SCRATCH_BYTES = 4 << 20
 MAX_LAYERS = 32
 
 EXPORTS = [
     "calidrop_compress_workspace_bytes", "calidrop_compress", "calidrop_compress_workspace_layout",
     "calidrop_decode_workspace_bytes", "calidrop_decode_workspace_init", "calidrop_decode",
-    "calidrop_decode_batched", "calidrop_compress_host", "calidrop_decode_host",
+    "calidrop_decode_batched", "calidrop_decode_static", "calidrop_compress_host", "calidrop_decode_host",
     "calidrop_status_string", "calidrop_version", "calidrop_launch_count",
 ]
 
@@ -75,6 +76,8 @@ def load():
     lib.calidrop_decode_batched.restype = C.c_int
     lib.calidrop_decode_batched.argtypes = [C.POINTER(Params), C.c_int32, C.POINTER(DecodeLayer), C.c_int32,
                                             vp, C.c_size_t, vp]
+    lib.calidrop_decode_static.restype = C.c_int
+    lib.calidrop_decode_static.argtypes = [C.POINTER(Params)] + [vp] * 5 + [C.c_int32] + [vp] * 7
     lib.calidrop_compress_host.restype = C.c_int
     lib.calidrop_compress_host.argtypes = [C.POINTER(Params)] + [vp] * 18 + [C.c_size_t, vp]
     lib.calidrop_decode_host.restype = C.c_int
@@ -162,6 +165,17 @@ def calidrop_decode(p, q, k_new, v_new, K_kept, V_kept, kv_len, O_c, LSE_c, C_q,
                                 _stream())
     if check:
         _check(rc, "calidrop_decode")
+    return rc
+
+
+def calidrop_decode_static(p, q, k_new, v_new, K_kept, V_kept, kv_len, O_c, LSE_c, C_q, out, lse_out, flags,
+                           check=True) -> int:
+    """calidrop_decode with the library's built-in scratch: no workspace argument, nothing allocated."""
+    rc = load().calidrop_decode_static(C.byref(p), _ptr(q), _ptr(k_new), _ptr(v_new), _ptr(K_kept),
+                                       _ptr(V_kept), int(kv_len), _ptr(O_c), _ptr(LSE_c), _ptr(C_q), _ptr(out),
+                                       _ptr(lse_out), _ptr(flags), _stream())
+    if check:
+        _check(rc, "calidrop_decode_static")
     return rc
 
 

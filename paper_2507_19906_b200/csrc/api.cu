@@ -123,6 +123,30 @@ DecodeWs make_decode_ws(const calidrop_params* p) {
   return w;
 }
 
+// Built-in scratch of calidrop_decode_static.  In host code this name is only a handle for
+// cudaGetSymbolAddress; the kernel must be given the device address that call returns.
+static __device__ __align__(256) unsigned char g_static_decode_scratch[CALIDROP_STATIC_SCRATCH_BYTES];
+
+// Device address of the built-in scratch on the current device (looked up once per device).
+int static_scratch_ptr(void** out) {
+  static void* ptr_of[64];
+  static std::atomic<int> ready[64];
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return cuda_fail(e);
+  if (dev < 0 || dev >= 64) return CALIDROP_UNSUPPORTED;
+  if (!ready[dev].load(std::memory_order_acquire)) {
+    void* ptr = nullptr;
+    e = cudaGetSymbolAddress(&ptr, g_static_decode_scratch);
+    if (e != cudaSuccess) return cuda_fail(e);
+    if (!ptr) return CALIDROP_CUDA_ERROR;
+    ptr_of[dev] = ptr;   // racing first calls store the same value
+    ready[dev].store(1, std::memory_order_release);
+  }
+  *out = ptr_of[dev];
+  return CALIDROP_OK;
+}
+
 }  // namespace
 
 void count_launch(int n) { g_launches.fetch_add((uint64_t)n, std::memory_order_relaxed); }
@@ -254,6 +278,32 @@ int calidrop_decode(const calidrop_params* p, const void* q, const void* k_new, 
   return calidrop_decode_batched(p, 1, &L, kv_len, workspace, workspace_bytes, stream);
 }
 
+int calidrop_decode_static(const calidrop_params* p, const void* q, const void* k_new, const void* v_new,
+                           void* K_kept, void* V_kept, int32_t kv_len, const float* O_c, const float* LSE_c,
+                           const void* C_q, void* out, float* lse_out, uint8_t* flags, void* stream) {
+  int rc = check_common(p);
+  if (rc != CALIDROP_OK) return rc;
+  const DecodeWs w = make_decode_ws(p);
+  if (w.per_layer > (size_t)CALIDROP_STATIC_SCRATCH_BYTES) return CALIDROP_SCRATCH_LIMIT;
+  // Everything calidrop_decode would reject is rejected here too, before the scratch is touched.
+  const void* req[] = {q, K_kept, V_kept, O_c, LSE_c, C_q, out};
+  for (const void* r : req)
+    if (!r || !aligned16(r)) return CALIDROP_INVALID_ARG;
+  if ((k_new != nullptr) != (v_new != nullptr)) return CALIDROP_INVALID_ARG;
+  if (k_new && (!aligned16(k_new) || !aligned16(v_new))) return CALIDROP_INVALID_ARG;
+  const int n_kv = kv_len + (k_new ? 1 : 0);
+  if (kv_len < 0 || n_kv < 1 || n_kv > p->cap) return CALIDROP_INVALID_ARG;
+  if (!device_supported()) return CALIDROP_UNSUPPORTED;
+  void* scratch = nullptr;
+  rc = static_scratch_ptr(&scratch);
+  if (rc != CALIDROP_OK) return rc;
+  // The arrival counters lead the carving; the rest of the scratch is written before it is read.
+  cudaError_t e = cudaMemsetAsync(scratch, 0, w.part_ml, (cudaStream_t)stream);
+  if (e != cudaSuccess) return cuda_fail(e);
+  return calidrop_decode(p, q, k_new, v_new, K_kept, V_kept, kv_len, O_c, LSE_c, C_q, out, lse_out, flags,
+                         scratch, (size_t)CALIDROP_STATIC_SCRATCH_BYTES, stream);
+}
+
 int calidrop_compress_host(const calidrop_params* p, const void* Q_obs_h, const void* K_h, const void* V_h,
                            const float* lse_obs_h, int32_t* kept_idx_h, float* O_c_h, float* LSE_c_h,
                            void* Q_obs, void* K, void* V, float* lse_obs, int32_t* kept_idx, void* K_kept,
@@ -323,6 +373,7 @@ const char* calidrop_status_string(int status) {
     case CALIDROP_UNSUPPORTED: return "unsupported configuration or device";
     case CALIDROP_WORKSPACE_TOO_SMALL: return "workspace too small";
     case CALIDROP_CUDA_ERROR: return g_err_text[0] ? g_err_text : "CUDA error";
+    case CALIDROP_SCRATCH_LIMIT: return "problem needs more scratch than the built-in static buffer holds";
     default: return "unknown status";
   }
 }
