@@ -113,11 +113,17 @@ int calidrop_compress(const calidrop_params* p,
 /*
  * Offsets (bytes from the workspace base) of intermediate arrays of the last
  * calidrop_compress call that used this workspace, for diagnostics and tests:
- *   vote   [B, Hkv, L-W] f32, pooled [B, Hkv, L-W] f32, row_lse [B, Hq, W] f32 (natural log).
+ *   vote   [B, Hkv, L-W] f32, pooled [B, Hkv, L-W] f32, row_lse [B, Hq, W] f32 (natural log;
+ *   not written when lse_obs was supplied), status u32.
+ * status is 0 after a call whose kernels all ran to completion.  The tensor-core kernels wait
+ * on their copy/MMA pipelines with a time limit; a wait that expires (which indicates a bug or
+ * a failing device, not bad input) stores a non-zero code here and the kernel ends early, so
+ * the call's outputs are then undefined.  A caller that wants the check reads the word after
+ * synchronising the stream.
  * Returns CALIDROP_OK, or INVALID_ARG if the parameters are invalid.
  */
 typedef struct calidrop_compress_layout {
-  size_t vote_offset, pooled_offset, row_lse_offset;
+  size_t vote_offset, pooled_offset, row_lse_offset, status_offset;
 } calidrop_compress_layout;
 int calidrop_compress_workspace_layout(const calidrop_params* p, calidrop_compress_layout* out);
 

@@ -37,7 +37,8 @@ class Params(C.Structure):
 
 
 class CompressLayout(C.Structure):
-    _fields_ = [("vote_offset", C.c_size_t), ("pooled_offset", C.c_size_t), ("row_lse_offset", C.c_size_t)]
+    _fields_ = [("vote_offset", C.c_size_t), ("pooled_offset", C.c_size_t), ("row_lse_offset", C.c_size_t),
+                ("status_offset", C.c_size_t)]
 
 
 class DecodeLayer(C.Structure):

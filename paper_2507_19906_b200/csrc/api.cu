@@ -3,6 +3,7 @@
 #include <atomic>
 #include <cmath>
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
 
 #include "../../include/calidrop.h"
@@ -77,6 +78,15 @@ CompressWs make_ws(const CompressGeom& g) {
   w.bitmap = off;  off = align_up(off + (size_t)g.units * g.bitmap_words * 4, 256);
   w.n_tiles = (g.L + 127) / 128;
   w.stat_part = off; off = align_up(off + (size_t)g.B * g.Hq * g.W * w.n_tiles * 8, 256);
+  w.status = off;    off = align_up(off + 4, 256);
+  w.calib_o = w.calib_l = off;
+  if (score_tc_supported(g) && calib_tc_supported(g)) {
+    int gpb, n_cblocks, n_splits;
+    calib_tc_plan(g, &gpb, &n_cblocks, &n_splits);
+    const size_t parts = (size_t)g.units * n_cblocks * n_splits;
+    w.calib_o = off; off = align_up(off + parts * 128 * kD * 4, 256);
+    w.calib_l = off; off = align_up(off + parts * 128 * 4, 256);
+  }
   w.total = off;
   return w;
 }
@@ -92,6 +102,16 @@ int device_supported() {
     major_of[dev] = major;
   }
   return major_of[dev] == 10;
+}
+
+// CALIDROP_COMPRESS_PATH=scalar (read once) routes compress through the CUDA-core kernels, for
+// diagnosis of the tensor-core path.
+bool scalar_path_forced() {
+  static const bool forced = [] {
+    const char* v = getenv("CALIDROP_COMPRESS_PATH");
+    return v && strcmp(v, "scalar") == 0;
+  }();
+  return forced;
 }
 
 // Split-K factor of the decode launch: enough CTAs to fill the machine twice over, never
@@ -169,6 +189,7 @@ int calidrop_compress_workspace_layout(const calidrop_params* p, calidrop_compre
   out->vote_offset = w.vote;
   out->pooled_offset = w.pooled;
   out->row_lse_offset = w.row_lse;
+  out->status_offset = w.status;
   return CALIDROP_OK;
 }
 
@@ -189,22 +210,28 @@ int calidrop_compress(const calidrop_params* p, const void* Q_obs, const void* K
 
   cudaStream_t st = (cudaStream_t)stream;
   char* wsp = (char*)workspace;
-  cudaError_t e = cudaSuccess;
+  cudaError_t e = cudaMemsetAsync(wsp + ws.status, 0, 4, st);
+  if (e != cudaSuccess) return cuda_fail(e);
+  // The contractions run on the tensor cores whenever the tiles cover the shape; the scalar
+  // kernels remain for the rest (more than 512 window rows per kv head, budget >= L).
+  const bool tc_path = score_tc_supported(g) && !scalar_path_forced();
+  const float* row_lse = lse_obs;
   if (!g.keep_all) {
-    const float* row_lse = lse_obs;
     if (!row_lse) {
-      e = launch_row_stats(g, ws, Q_obs, K, wsp, st);
+      e = tc_path ? launch_row_stats_tc(g, ws, Q_obs, K, wsp, st) : launch_row_stats(g, ws, Q_obs, K, wsp, st);
       if (e != cudaSuccess) return cuda_fail(e);
       row_lse = (const float*)(wsp + ws.row_lse);
     }
-    e = launch_votes(g, ws, Q_obs, K, row_lse, wsp, st);
+    e = tc_path ? launch_votes_tc(g, ws, Q_obs, K, row_lse, wsp, st) : launch_votes(g, ws, Q_obs, K, row_lse, wsp, st);
     if (e != cudaSuccess) return cuda_fail(e);
   }
   e = launch_pool_select(g, ws, wsp, kept_idx, st);
   if (e != cudaSuccess) return cuda_fail(e);
   e = launch_gather(g, K, V, kept_idx, K_kept, V_kept, st);
   if (e != cudaSuccess) return cuda_fail(e);
-  e = launch_calib_direct(g, ws, Q_obs, K, V, wsp, O_c, LSE_c, C_q, st);
+  e = (tc_path && calib_tc_supported(g))
+          ? launch_calib_tc(g, ws, Q_obs, K, V, row_lse, wsp, O_c, LSE_c, C_q, st)
+          : launch_calib_direct(g, ws, Q_obs, K, V, wsp, O_c, LSE_c, C_q, st);
   if (e != cudaSuccess) return cuda_fail(e);
   return CALIDROP_OK;
 }

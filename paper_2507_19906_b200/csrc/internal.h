@@ -21,7 +21,7 @@ struct CompressGeom {
 
 // Workspace carving of compress (byte offsets, all 256-byte aligned).
 struct CompressWs {
-  size_t vote, pooled, row_lse, bitmap, stat_part, total;
+  size_t vote, pooled, row_lse, bitmap, stat_part, status, calib_o, calib_l, total;
   int n_tiles;  // 128-key tiles per unit for the partial row statistics
 };
 
@@ -64,6 +64,18 @@ cudaError_t launch_votes(const CompressGeom& g, const CompressWs& ws, const void
 cudaError_t launch_calib_direct(const CompressGeom& g, const CompressWs& ws, const void* Q_obs,
                                 const void* K, const void* V, char* wsp, float* O_c, float* LSE_c,
                                 void* C_q, cudaStream_t st);
+// score_tc.cu / calib_tc.cu: the tcgen05 + TMA path
+int pick_tile_splits(int groups, int n_tiles, int min_tiles);
+bool score_tc_supported(const CompressGeom& g);
+cudaError_t launch_row_stats_tc(const CompressGeom& g, const CompressWs& ws, const void* Q_obs, const void* K,
+                                char* wsp, cudaStream_t st);
+cudaError_t launch_votes_tc(const CompressGeom& g, const CompressWs& ws, const void* Q_obs, const void* K,
+                            const float* row_lse, char* wsp, cudaStream_t st);
+bool calib_tc_supported(const CompressGeom& g);
+void calib_tc_plan(const CompressGeom& g, int* gpb, int* n_cblocks, int* n_splits);
+cudaError_t launch_calib_tc(const CompressGeom& g, const CompressWs& ws, const void* Q_obs, const void* K,
+                            const void* V, const float* row_lse, char* wsp, float* O_c, float* LSE_c, void* C_q,
+                            cudaStream_t st);
 // select.cu
 cudaError_t launch_pool_select(const CompressGeom& g, const CompressWs& ws, char* wsp,
                                int32_t* kept_idx, cudaStream_t st);

@@ -1,0 +1,200 @@
+// Blackwell (sm_100a) building blocks of the tensor-core compress kernels: mbarriers with bounded
+// waits, TMA tile loads, TMEM allocation, tcgen05 MMA issue / commit / TMEM loads, and the shared
+// memory and instruction descriptors of the bf16 UMMA.
+//
+// Conventions used by every kernel built on this header:
+//   * A bf16 tile of R rows x 128 head-dim elements lives in shared memory as two halves of
+//     R x 64 elements; a half is R lines of 128 bytes written by one TMA box with the 128-byte
+//     swizzle (the 16-byte chunk index of a line is XORed with line & 7).  Tile bases are
+//     1024-byte aligned.  Read with the head dimension as the MMA K this is the "K-major" operand
+//     form; read with the rows as K (the V operand of P.V) it is the "MN-major" form.
+//   * Every wait on an mbarrier is bounded: when it expires the thread records an error code in
+//     global memory, raises the CTA's abort flag and every role falls through to the common
+//     teardown, which still frees the tensor memory.  Nothing ever traps or spins forever.
+#pragma once
+
+#include <cuda.h>
+
+#include "common.cuh"
+
+namespace calidrop {
+namespace tc {
+
+constexpr unsigned long long kWaitLimitNs = 2000000000ull;  // 2 s per wait
+
+// ---------------------------------------------------------------- mbarrier
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void fence_mbar_init() {
+  asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+}
+// Orders generic-proxy shared-memory writes before later async-proxy (TMA, MMA) accesses.
+__device__ __forceinline__ void fence_proxy_async_smem() {
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n"
+      ".reg .pred p;\n"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+      "selp.u32 %0, 1, 0, p;\n"
+      "}\n"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ unsigned long long global_timer_ns() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+
+// Shared per-CTA control block of the bounded waits.
+struct Ctl {
+  volatile int abort;       // raised by the first thread whose wait expired
+  unsigned* status;         // global error word (0 = fine)
+};
+
+// Wait for the phase with the given parity to complete.  Returns false when the CTA is aborting
+// (this wait expired, or another thread's did).
+__device__ __forceinline__ bool mbar_wait(Ctl* ctl, uint32_t bar, uint32_t parity, unsigned code) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const unsigned long long t0 = global_timer_ns();
+  unsigned polls = 0;
+  while (!mbar_try_wait(bar, parity)) {
+    if ((++polls & 255u) == 0u) {
+      if (ctl->abort) return false;
+      if (global_timer_ns() - t0 > kWaitLimitNs) {
+        ctl->abort = 1;
+        atomicMax(ctl->status, code);
+        return false;
+      }
+    }
+  }
+  return true;
+}
+
+// ---------------------------------------------------------------- TMA tile loads (no cluster forms)
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1,
+                                            int c2) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+      ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2)
+      : "memory");
+}
+__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1,
+                                            int c2, int c3) {
+  asm volatile(
+      "cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
+      ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
+      : "memory");
+}
+__device__ __forceinline__ void tma_prefetch_desc(const CUtensorMap* map) {
+  asm volatile("prefetch.tensormap [%0];" ::"l"(map) : "memory");
+}
+
+// ---------------------------------------------------------------- tensor memory
+// Whole-warp calls.  The allocated base address (lane 0, first column) is written to smem_dst.
+__device__ __forceinline__ void tmem_alloc(uint32_t smem_dst, uint32_t ncols) {
+  asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_dst), "r"(ncols)
+               : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish() {
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols) {
+  asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before_sync() {
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+}
+__device__ __forceinline__ void tc_fence_after_sync() {
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+}
+
+// 32 consecutive fp32 columns of this thread's TMEM lane (lane = 32 * (warp % 4) + laneid must be
+// encoded in bits 16.. of taddr by the caller).  The load and its completion wait are one
+// statement so that no use of the registers can be scheduled before the wait.
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];\n"
+      "tcgen05.wait::ld.sync.aligned;\n"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+        "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+        "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr)
+      : "memory");
+}
+
+// ---------------------------------------------------------------- UMMA (bf16 x bf16 -> fp32)
+// Shared-memory matrix descriptor, 128-byte swizzle.  lbo/sbo in bytes:
+//   K-major operand : sbo = distance between groups of 8 rows (1024), lbo unused;
+//   MN-major operand: lbo = distance between 64-element blocks along M/N, sbo = distance between
+//                     groups of 8 K-rows (1024).
+__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t saddr, uint32_t lbo, uint32_t sbo) {
+  uint64_t d = 0;
+  d |= (uint64_t)((saddr & 0x3FFFFu) >> 4);
+  d |= (uint64_t)((lbo >> 4) & 0x3FFFu) << 16;
+  d |= (uint64_t)((sbo >> 4) & 0x3FFFu) << 32;
+  d |= 1ull << 46;  // descriptor version of this architecture
+  d |= 2ull << 61;  // 128-byte swizzle
+  return d;
+}
+
+// Instruction descriptor: fp32 accumulator, bf16 A and B, M x N tile, operand majors.
+__host__ __device__ constexpr uint32_t umma_idesc(int M, int N, bool a_mn_major, bool b_mn_major) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((a_mn_major ? 1u : 0u) << 15) | ((b_mn_major ? 1u : 0u) << 16) |
+         ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
+}
+
+// D[tmem] (+)= A[smem] * B[smem]; one thread issues for the CTA.
+__device__ __forceinline__ void umma_ss(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                        uint32_t accumulate) {
+  asm volatile(
+      "{\n"
+      ".reg .pred p;\n"
+      "setp.ne.b32 p, %4, 0;\n"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n"
+      "}\n"
+      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+// The mbarrier receives one arrival when every MMA issued so far by this thread has completed.
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar)
+               : "memory");
+}
+
+constexpr int kHalfCols = 64;          // head-dim elements per shared-memory half tile
+constexpr int kLineBytes = 128;        // one half-tile line
+constexpr int kTileKeys = 128;         // keys per streamed K/V tile
+constexpr int kKvTileBytes = 2 * kTileKeys * kLineBytes;  // 32 KB: both halves of a 128-row tile
+
+// Descriptor of MMA k-step kk (16 head-dim elements) of a K-major tile whose halves are
+// `half_bytes` apart.
+__device__ __forceinline__ uint64_t kmajor_desc(uint32_t tile_base, uint32_t half_bytes, int kk) {
+  return smem_desc_sw128(tile_base + (uint32_t)(kk >> 2) * half_bytes + (uint32_t)(kk & 3) * 32u, 16u, 1024u);
+}
+
+}  // namespace tc
+
+// Host side (tmap.cu): tensor map over a bf16 tensor whose innermost dimension is the 128-element
+// head dimension, read in boxes of 64 elements x box[1] x box[2] (x box[3]) with the 128-byte
+// swizzle and zero fill outside the tensor.  dims/strides/box list the dimensions from the
+// second one on (the head dimension is implied); strides in bytes.  Returns false on failure.
+bool make_tensor_map_bf16(CUtensorMap* out, const void* base, int rank, const uint64_t* dims_from_1,
+                          const uint64_t* strides_from_1, const uint32_t* box_from_1);
+
+}  // namespace calidrop

@@ -43,6 +43,9 @@ def gpu_compress(Q_obs, K, V, *, window, pool, budget, n_cal=1, cap=None, lse_ob
     def ws_f32(off, n):
         return st.ws_compress[off: off + 4 * n].view(torch.float32).cpu().numpy()
 
+    status = int(st.ws_compress[lay.status_offset: lay.status_offset + 4].view(torch.int32).item())
+    assert status == 0, f"a compress kernel gave up waiting on its pipeline (code {status})"
+
     r = SimpleNamespace(
         p=p, st=st,
         kept_idx=st.kept_idx.cpu().numpy(), K_kept=to_bits(st.K_kept), V_kept=to_bits(st.V_kept),
