@@ -73,11 +73,13 @@ CompressWs make_ws(const CompressGeom& g) {
   size_t off = 0;
   const size_t n_cand = (size_t)(g.L > g.W ? g.L - g.W : 0);
   w.vote = off;    off = align_up(off + (size_t)g.units * n_cand * 4, 256);
+  w.vote2 = off;   off = align_up(off + (g.G * g.W > 256 ? (size_t)g.units * n_cand * 4 : 0), 256);
   w.pooled = off;  off = align_up(off + (size_t)g.units * n_cand * 4, 256);
   w.row_lse = off; off = align_up(off + (size_t)g.B * g.Hq * g.W * 4, 256);
   w.bitmap = off;  off = align_up(off + (size_t)g.units * g.bitmap_words * 4, 256);
   w.n_tiles = (g.L + 127) / 128;
-  w.stat_part = off; off = align_up(off + (size_t)g.B * g.Hq * g.W * w.n_tiles * 8, 256);
+  w.stat_slots = w.n_tiles > 128 ? w.n_tiles : 128;
+  w.stat_part = off; off = align_up(off + (size_t)g.B * g.Hq * g.W * w.stat_slots * 8, 256);
   w.status = off;    off = align_up(off + 4, 256);
   w.calib_o = w.calib_l = off;
   if (score_tc_supported(g) && calib_tc_supported(g)) {
@@ -85,7 +87,7 @@ CompressWs make_ws(const CompressGeom& g) {
     calib_tc_plan(g, &gpb, &n_cblocks, &n_splits);
     const size_t parts = (size_t)g.units * n_cblocks * n_splits;
     w.calib_o = off; off = align_up(off + parts * 128 * kD * 4, 256);
-    w.calib_l = off; off = align_up(off + parts * 128 * 4, 256);
+    w.calib_l = off; off = align_up(off + parts * 2 * 128 * 4, 256);
   }
   w.total = off;
   return w;

@@ -22,7 +22,10 @@ namespace {
 
 using namespace tc;
 
-constexpr int kThreads = 192;
+constexpr int kGroups = 2;  // softmax warpgroups; group g owns S buffer g and P buffer g (tiles i % 2 == g)
+constexpr int kProducerWarp = kGroups * 4;
+constexpr int kMmaWarp = kGroups * 4 + 1;
+constexpr int kThreads = kGroups * 128 + 64;
 constexpr int kTmemCols = 512;
 constexpr int kTileBytes = kKvTileBytes;  // 32 KB: Q block, K tile, V tile and P tile alike
 constexpr int kSmemBytes = 7 * kTileBytes + 1024;
@@ -37,7 +40,7 @@ struct CalibArgs {
   const float* row_lse;    // [B, Hq, W] natural log
   const uint32_t* bitmap;  // [units][bitmap_words], bit set = kept
   float* o_part;           // [unit][block][split][128][128]
-  float* l_part;           // [unit][block][split][128]
+  float* l_part;           // [unit][block][split][group][128]
   unsigned* status;
 };
 
@@ -86,7 +89,7 @@ calib_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
     }
     fence_mbar_init();
   }
-  if (warp == 5) {
+  if (warp == kMmaWarp) {
     tmem_alloc(smem_u32(&tmem_slot), kTmemCols);
     tmem_relinquish();
   }
@@ -95,6 +98,7 @@ calib_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
   if (warp < 4) {
     uint4* qz = reinterpret_cast<uint4*>(smem_al);
     for (int i = tid; i < kTileBytes / 16; i += 128) qz[i] = make_uint4(0u, 0u, 0u, 0u);
+    // (only the first warpgroup clears; the barrier below orders it before the TMA)
     fence_proxy_async_smem();
   }
   tc_fence_before_sync();
@@ -109,7 +113,7 @@ calib_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
   const int ng = min(a.gpb, a.G - g0);
   const int rows = ng * a.n_cal;  // valid rows of this block
 
-  if (warp == 4) {
+  if (warp == kProducerWarp) {
     // ------------------------------------------------------------ TMA producer
     if (lane == 0) {
       tma_prefetch_desc(&q_map);
@@ -134,7 +138,7 @@ calib_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
                       (tile0 + i) * kTileKeys, unit);
       }
     }
-  } else if (warp == 5) {
+  } else if (warp == kMmaWarp) {
     // ------------------------------------------------------------ MMA issuer
     if (lane == 0) {
       const uint32_t idesc_s = umma_idesc(128, 128, false, false);
@@ -178,19 +182,19 @@ calib_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
     }
   } else {
     // ------------------------------------------------------------ softmax threads (one row each)
-    const int r = tid;
+    const int grp = warp >> 2, r = tid & 127;
     const bool valid = r < rows;
     float nlse2 = -INFINITY;
     if (valid) {
       const int g = g0 + r / a.n_cal, c = r - (r / a.n_cal) * a.n_cal;
       nlse2 = -a.row_lse[(size_t)(hq0 + g) * a.W + (a.W - a.n_cal + c)] * kLog2e;
     }
-    const uint32_t lane_addr = tmem_base + ((uint32_t)(warp * 32) << 16);
+    const uint32_t lane_addr = tmem_base + ((uint32_t)((warp & 3) * 32) << 16);
     const uint32_t* bm = a.bitmap + (size_t)unit * a.bitmap_words;
-    float l = 0.f;
+    float l0 = 0.f, l1 = 0.f;
     bool ok = true;
-    for (int i = 0; i < nt; ++i) {
-      const int s = i & 1;
+    for (int i = grp; i < nt; i += kGroups) {
+      const int s = i & 1;  // == grp
       const uint32_t ph = (i >> 1) & 1;
       ok = mbar_wait(&ctl, s_full(s), ph, 28u) && mbar_wait(&ctl, p_empty(s), ph ^ 1, 29u);
       ok = __all_sync(0xffffffffu, ok);
@@ -198,16 +202,15 @@ calib_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
       tc_fence_after_sync();
       const int tbase = (tile0 + i) * kTileKeys;
       const uint32_t p_row = p_base + s * kTileBytes + (uint32_t)r * kLineBytes;
-#pragma unroll 1
-      for (int q4 = 0; q4 < 4; ++q4) {
+      const uint32_t taddr = lane_addr + (uint32_t)(s * 128);
+      // probabilities of 32 keys -> bf16 -> the P tile (K-major, 128-byte swizzle)
+      auto soft32 = [&](const uint32_t (&sv)[32], int q4) {
         const int kbase = tbase + 32 * q4;
         uint32_t word = 0xffffffffu;  // bit set = this key does not contribute
         if (kbase < a.n_cand) {
           word = __ldg(bm + (kbase >> 5));
           if (kbase + 32 > a.n_cand) word |= 0xffffffffu << (a.n_cand - kbase);
         }
-        uint32_t sv[32];
-        tmem_ld32(lane_addr + (uint32_t)(s * 128 + 32 * q4), sv);
         uint32_t packed[16];
 #pragma unroll
         for (int e = 0; e < 32; e += 2) {
@@ -215,7 +218,8 @@ calib_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
           float p1 = ex2_approx(fmaf(__uint_as_float(sv[e + 1]), a.scale2, nlse2));
           if ((word >> e) & 1u) p0 = 0.f;
           if ((word >> (e + 1)) & 1u) p1 = 0.f;
-          l += p0 + p1;
+          l0 += p0;
+          l1 += p1;
           packed[e >> 1] = pack_bf16(p0, p1);
         }
         const uint32_t half_off = (uint32_t)(q4 >> 1) * (kTileBytes / 2);
@@ -226,13 +230,26 @@ calib_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
                        "r"(packed[4 * v]), "r"(packed[4 * v + 1]), "r"(packed[4 * v + 2]), "r"(packed[4 * v + 3])
                        : "memory");
         }
-      }
-      fence_proxy_async_smem();
+      };
+      uint32_t ra[32], rb[32];
+      tmem_ld32_issue(taddr, ra);
+      tmem_ld_wait(ra);
+      tmem_ld32_issue(taddr + 32, rb);
+      soft32(ra, 0);
+      tmem_ld_wait(rb);
+      tmem_ld32_issue(taddr + 64, ra);
+      soft32(rb, 1);
+      tmem_ld_wait(ra);
+      tmem_ld32_issue(taddr + 96, rb);
+      soft32(ra, 2);
+      tmem_ld_wait(rb);
       tc_fence_before_sync();
-      mbar_arrive(s_empty(s));
+      mbar_arrive(s_empty(s));  // the logits are in registers: the next S tile may be issued
+      soft32(rb, 3);
+      fence_proxy_async_smem();
       mbar_arrive(p_full(s));
     }
-    // epilogue: the accumulated O rows and the row sums of this key range
+    // epilogue: the accumulated O rows (each group stores half of the columns) and the row sums
     if (ok) {
       ok = nt == 0 || mbar_wait(&ctl, o_full, 0, 30u);
       ok = __all_sync(0xffffffffu, ok);
@@ -242,10 +259,10 @@ calib_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
       const size_t part = ((size_t)unit * a.n_cblocks + cb) * a.n_splits + split;
       float* orow = a.o_part + (part * 128 + r) * kD;
 #pragma unroll 1
-      for (int c0 = 0; c0 < kD; c0 += 32) {
+      for (int c0 = grp * (kD / kGroups); c0 < (grp + 1) * (kD / kGroups); c0 += 32) {
         uint32_t ov[32];
         if (nt > 0) {
-          tmem_ld32(tmem_o + ((uint32_t)(warp * 32) << 16) + c0, ov);
+          tmem_ld32(tmem_o + ((uint32_t)((warp & 3) * 32) << 16) + c0, ov);
         } else {
 #pragma unroll
           for (int e = 0; e < 32; ++e) ov[e] = 0u;
@@ -256,7 +273,7 @@ calib_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
             *reinterpret_cast<uint4*>(orow + c0 + e) = make_uint4(ov[e], ov[e + 1], ov[e + 2], ov[e + 3]);
         }
       }
-      if (valid) a.l_part[part * 128 + r] = l;
+      if (valid) a.l_part[(part * kGroups + grp) * 128 + r] = l0 + l1;
     }
   }
 
@@ -266,7 +283,7 @@ calib_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
   }
   tc_fence_before_sync();
   __syncthreads();
-  if (warp == 5) tmem_dealloc(tmem_base, kTmemCols);
+  if (warp == kMmaWarp) tmem_dealloc(tmem_base, kTmemCols);
 }
 
 // One warp per (batch, query head, calibration row): sum the key-range partials in order, then
@@ -289,7 +306,7 @@ calib_reduce_kernel(const __nv_bfloat16* __restrict__ Q_obs, const float* __rest
   for (int s = 0; s < n_splits; ++s) {
     const float4 v = *reinterpret_cast<const float4*>(o_part + ((part0 + s) * 128 + r) * kD + 4 * lane);
     acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
-    l += l_part[(part0 + s) * 128 + r];
+    for (int grp = 0; grp < kGroups; ++grp) l += l_part[((part0 + s) * kGroups + grp) * 128 + r];
   }
   const int qrow = W - n_cal + c;
   float4 out = make_float4(0.f, 0.f, 0.f, 0.f);

@@ -21,8 +21,9 @@ struct CompressGeom {
 
 // Workspace carving of compress (byte offsets, all 256-byte aligned).
 struct CompressWs {
-  size_t vote, pooled, row_lse, bitmap, stat_part, status, calib_o, calib_l, total;
-  int n_tiles;  // 128-key tiles per unit for the partial row statistics
+  size_t vote, vote2, pooled, row_lse, bitmap, stat_part, status, calib_o, calib_l, total;
+  int n_tiles;     // 128-key tiles per unit (scalar statistics pass: one partial per tile)
+  int stat_slots;  // (max, sum) partial slots per observation row in stat_part
 };
 
 struct DecodeLayerPtrs {

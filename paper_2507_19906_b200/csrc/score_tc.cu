@@ -24,36 +24,66 @@ namespace {
 
 using namespace tc;
 
-constexpr int kThreads = 192;
+constexpr int kGroups = 2;                       // consumer warpgroups (4 warps each)
+constexpr int kConsumers = kGroups * 128;
+constexpr int kProducerWarp = kGroups * 4;
+constexpr int kMmaWarp = kGroups * 4 + 1;
+constexpr int kThreads = kConsumers + 64;
 constexpr int kTmemCols = 512;
 constexpr int kMaxRows = 512;  // G * W handled by the tiles
 
 struct ScoreArgs {
   int Hq, G, W, L, n_cand, GW;
   int n_blocks;    // blocks of observation rows
-  int block_rows;  // rows per block: 128 for the statistics, a multiple of 32 (<= 256) for the votes
+  int block_rows;  // rows per block: 128 for the statistics; a multiple of 32 (<= 256) for the votes
+  int n_buf;       // accumulator ring in TMEM: n_buf buffers of buf_cols columns (n_buf * buf_cols = 512)
+  int buf_cols;
   int n_tiles;     // key tiles to cover
   int n_splits;
   int stages;      // depth of the key-tile ring (2 or 3)
   float scale2;
   const float* row_lse;  // votes: natural-log LSE of every observation row [B, Hq, W]
   float* vote;           // votes: out [units, n_cand]
-  float2* stat_part;     // statistics: out [row][split] (max, sum) in the log2 domain
+  float* vote2;          // votes of the second row block when there are two (summed into vote afterwards)
+  float2* stat_part;     // statistics: out [row][split][group] (max, sum) in the log2 domain
   unsigned* status;
 };
+
+// exp2 of 32 logits against one reference, four independent partial sums
+__device__ __forceinline__ float sum_exp2_32(const uint32_t (&r)[32], float scale2, float neg_ref) {
+  float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
+#pragma unroll
+  for (int e = 0; e < 32; e += 4) {
+    s0 += ex2_approx(fmaf(__uint_as_float(r[e + 0]), scale2, neg_ref));
+    s1 += ex2_approx(fmaf(__uint_as_float(r[e + 1]), scale2, neg_ref));
+    s2 += ex2_approx(fmaf(__uint_as_float(r[e + 2]), scale2, neg_ref));
+    s3 += ex2_approx(fmaf(__uint_as_float(r[e + 3]), scale2, neg_ref));
+  }
+  return (s0 + s1) + (s2 + s3);
+}
+
+__device__ __forceinline__ float max_32(const uint32_t (&r)[32]) {
+  float m0 = -INFINITY, m1 = -INFINITY, m2 = -INFINITY, m3 = -INFINITY;
+#pragma unroll
+  for (int e = 0; e < 32; e += 4) {
+    m0 = fmaxf(m0, __uint_as_float(r[e + 0]));
+    m1 = fmaxf(m1, __uint_as_float(r[e + 1]));
+    m2 = fmaxf(m2, __uint_as_float(r[e + 2]));
+    m3 = fmaxf(m3, __uint_as_float(r[e + 3]));
+  }
+  return fmaxf(fmaxf(m0, m1), fmaxf(m2, m3));
+}
 
 template <bool kVotes>
 __global__ void __launch_bounds__(kThreads, 1)
 score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__ CUtensorMap k_map,
                 const ScoreArgs a) {
-  constexpr int NBUF = kVotes ? 2 : 4;        // accumulator ring in TMEM
-  constexpr int BUFCOLS = kVotes ? 256 : 128;
   extern __shared__ unsigned char smem_raw[];
   __shared__ __align__(8) unsigned long long bars[16];
   __shared__ uint32_t tmem_slot;
   __shared__ Ctl ctl;
-  __shared__ __align__(16) float nlse2_s[kVotes ? kMaxRows : 4];          // -log2-domain LSE per row (-inf: padding)
-  __shared__ float2 ml_s[kVotes ? 1 : 4][kVotes ? 1 : 128];  // running (max, sum) per row block
+  __shared__ __align__(16) float nlse2_s[kVotes ? kMaxRows : 4];  // -log2-domain LSE per row (-inf: padding)
+  __shared__ float2 ml_s[kVotes ? 1 : kGroups][kVotes ? 1 : 4][kVotes ? 1 : 128];  // running (max, sum)
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int split = blockIdx.x, unit = blockIdx.y;
@@ -83,7 +113,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
     for (int b = 0; b < 4; ++b) { mbar_init(t_full(b), 1); mbar_init(t_empty(b), 128); }
     fence_mbar_init();
   }
-  if (warp == 5) {
+  if (warp == kMmaWarp) {
     tmem_alloc(smem_u32(&tmem_slot), kTmemCols);
     tmem_relinquish();
   }
@@ -97,7 +127,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
   tc_fence_after_sync();
   const uint32_t tmem_base = tmem_slot;
 
-  if (warp == 4) {
+  if (warp == kProducerWarp) {
     // ------------------------------------------------------------ TMA producer
     if (lane == 0) {
       tma_prefetch_desc(&q_map);
@@ -109,25 +139,25 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
                       blk * a.block_rows, unit);
       for (int i = 0; i < nt; ++i) {
         const int s = i % a.stages;
-        if (!mbar_wait(&ctl, empty_k(s), ((i / a.stages) & 1) ^ 1, 11u)) break;
+        if (!mbar_wait(&ctl, empty_k(s), ((i / a.stages) & 1) ^ 1, (kVotes ? 31u : 11u) | ((unsigned)i << 8))) break;
         mbar_arrive_expect_tx(full_k(s), kKvTileBytes);
         for (int half = 0; half < 2; ++half)
           tma_load_3d(k_base + s * kKvTileBytes + half * (kKvTileBytes / 2), &k_map, full_k(s), half * kHalfCols,
                       (tile0 + i) * kTileKeys, unit);
       }
     }
-  } else if (warp == 5) {
+  } else if (warp == kMmaWarp) {
     // ------------------------------------------------------------ MMA issuer
     if (lane == 0) {
       const uint32_t idesc = umma_idesc(128, kVotes ? a.block_rows : 128, false, false);
-      bool ok = mbar_wait(&ctl, q_full, 0, 12u);
+      bool ok = mbar_wait(&ctl, q_full, 0, kVotes ? 32u : 12u);
       for (int j = 0; ok && j < n_jobs; ++j) {
         const int i = j / a.n_blocks, blk = j - i * a.n_blocks;
-        const int s = i % a.stages, buf = j % NBUF;
-        if (blk == 0 && !mbar_wait(&ctl, full_k(s), (i / a.stages) & 1, 13u)) break;
-        if (!mbar_wait(&ctl, t_empty(buf), ((j / NBUF) & 1) ^ 1, 14u)) break;
+        const int s = i % a.stages, buf = j % a.n_buf;
+        if (blk == 0 && !mbar_wait(&ctl, full_k(s), (i / a.stages) & 1, (kVotes ? 33u : 13u) | ((unsigned)j << 8))) break;
+        if (!mbar_wait(&ctl, t_empty(buf), ((j / a.n_buf) & 1) ^ 1, (kVotes ? 34u : 14u) | ((unsigned)j << 8))) break;
         tc_fence_after_sync();
-        const uint32_t d = tmem_base + (uint32_t)(buf * BUFCOLS);
+        const uint32_t d = tmem_base + (uint32_t)(buf * a.buf_cols);
         const uint32_t kt = k_base + (uint32_t)s * kKvTileBytes, qt = q_base + (uint32_t)blk * q_blk_bytes;
 #pragma unroll
         for (int kk = 0; kk < kD / 16; ++kk) {
@@ -141,78 +171,99 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
     }
   } else {
     // ------------------------------------------------------------ accumulator consumers
-    const uint32_t lane_addr = tmem_base + ((uint32_t)(warp * 32) << 16);
-    float acc = 0.f;  // votes: running vote of this thread's key
+    // Warpgroup `grp` takes the jobs with job % kGroups == grp; thread ct of a group owns TMEM
+    // lane ct.  The launch shapes keep n_buf a multiple of kGroups, so an accumulator buffer (and
+    // its pair of mbarriers) is only ever consumed by one group and every group sees each phase
+    // of the barriers it waits on.
+    const int grp = warp >> 2, ct = tid & 127;
+    const uint32_t lane_addr = tmem_base + ((uint32_t)((warp & 3) * 32) << 16);
+    float acc0 = 0.f, acc1 = 0.f, acc2 = 0.f, acc3 = 0.f;  // votes: running vote of this thread's key
     if (!kVotes) {
-      for (int blk = 0; blk < 4; ++blk) ml_s[blk][tid] = make_float2(-INFINITY, 0.f);
+      for (int blk = 0; blk < 4; ++blk) ml_s[grp][blk][ct] = make_float2(-INFINITY, 0.f);
     }
     for (int j = 0; j < n_jobs; ++j) {
       const int i = j / a.n_blocks, blk = j - i * a.n_blocks;
-      const int buf = j % NBUF;
-      bool ok = mbar_wait(&ctl, t_full(buf), (j / NBUF) & 1, 15u);
+      if (j % kGroups != grp) continue;
+      const int buf = j % a.n_buf;
+      bool ok = mbar_wait(&ctl, t_full(buf), (j / a.n_buf) & 1, (kVotes ? 35u : 15u) | ((unsigned)j << 8));
       if (!__all_sync(0xffffffffu, ok)) break;
       tc_fence_after_sync();
       const int tbase = (tile0 + i) * kTileKeys;
-      const uint32_t taddr = lane_addr + (uint32_t)(buf * BUFCOLS);
-      uint32_t r[32];
+      const uint32_t taddr = lane_addr + (uint32_t)(buf * a.buf_cols);
+      uint32_t ra[32], rb[32];
       if (kVotes) {
         const float* nl = nlse2_s + blk * a.block_rows;
-        for (int c0 = 0; c0 < a.block_rows; c0 += 32) {
-          tmem_ld32(taddr + c0, r);
+        auto add32 = [&](const uint32_t (&r)[32], int c0) {
 #pragma unroll
           for (int e = 0; e < 32; e += 4) {
             const float4 n4 = *reinterpret_cast<const float4*>(nl + c0 + e);
-            acc += ex2_approx(fmaf(__uint_as_float(r[e + 0]), a.scale2, n4.x));
-            acc += ex2_approx(fmaf(__uint_as_float(r[e + 1]), a.scale2, n4.y));
-            acc += ex2_approx(fmaf(__uint_as_float(r[e + 2]), a.scale2, n4.z));
-            acc += ex2_approx(fmaf(__uint_as_float(r[e + 3]), a.scale2, n4.w));
+            acc0 += ex2_approx(fmaf(__uint_as_float(r[e + 0]), a.scale2, n4.x));
+            acc1 += ex2_approx(fmaf(__uint_as_float(r[e + 1]), a.scale2, n4.y));
+            acc2 += ex2_approx(fmaf(__uint_as_float(r[e + 2]), a.scale2, n4.z));
+            acc3 += ex2_approx(fmaf(__uint_as_float(r[e + 3]), a.scale2, n4.w));
+          }
+        };
+        // block_rows is a multiple of 32: chunks alternate between the two register sets
+        tmem_ld32_issue(taddr, ra);
+        for (int c0 = 0; c0 < a.block_rows; c0 += 64) {
+          tmem_ld_wait(ra);
+          const bool more_b = c0 + 32 < a.block_rows;
+          if (more_b) tmem_ld32_issue(taddr + c0 + 32, rb);
+          add32(ra, c0);
+          if (more_b) {
+            tmem_ld_wait(rb);
+            if (c0 + 64 < a.block_rows) tmem_ld32_issue(taddr + c0 + 64, ra);
+            add32(rb, c0 + 32);
           }
         }
         tc_fence_before_sync();
         mbar_arrive(t_empty(buf));
-        if (blk == a.n_blocks - 1) {
-          const int key = tbase + tid;
-          if (key < a.n_cand) a.vote[(size_t)unit * a.n_cand + key] = acc;
-          acc = 0.f;
+        {
+          const int key = tbase + ct;
+          float* out = blk == 0 ? a.vote : a.vote2;
+          if (key < a.n_cand) out[(size_t)unit * a.n_cand + key] = (acc0 + acc1) + (acc2 + acc3);
+          acc0 = acc1 = acc2 = acc3 = 0.f;
         }
       } else {
-        float2 ml = ml_s[blk][tid];
-        const int row = blk * 128 + tid;
+        float2 ml = ml_s[grp][blk][ct];
+        const int row = blk * 128 + ct;
         // local index of the last key this row may see inside the tile (causal inside the window)
         const int lim = min(a.L - 1, a.n_cand + row % a.W) - tbase;
         const bool full_tile = __all_sync(0xffffffffu, lim >= kTileKeys - 1);
-#pragma unroll 1
-        for (int c0 = 0; c0 < kTileKeys; c0 += 32) {
-          tmem_ld32(taddr + c0, r);
-          float cmax = -INFINITY;
-          if (full_tile) {
+        auto fold32 = [&](uint32_t (&r)[32], int c0) {
+          if (!full_tile) {
 #pragma unroll
-            for (int e = 0; e < 32; ++e) cmax = fmaxf(cmax, __uint_as_float(r[e]));
-          } else {
-#pragma unroll
-            for (int e = 0; e < 32; ++e) {
+            for (int e = 0; e < 32; ++e)
               if (c0 + e > lim) r[e] = 0xff800000u;  // -inf
-              cmax = fmaxf(cmax, __uint_as_float(r[e]));
-            }
           }
-          const float m_new = fmaxf(ml.x, cmax * a.scale2);
+          const float m_new = fmaxf(ml.x, max_32(r) * a.scale2);
           if (m_new > -INFINITY) {
-            float sum = 0.f;
-#pragma unroll
-            for (int e = 0; e < 32; ++e) sum += ex2_approx(fmaf(__uint_as_float(r[e]), a.scale2, -m_new));
-            ml.y = ml.y * ex2_approx(ml.x - m_new) + sum;
+            ml.y = ml.y * ex2_approx(ml.x - m_new) + sum_exp2_32(r, a.scale2, -m_new);
             ml.x = m_new;
           }
-        }
+        };
+        tmem_ld32_issue(taddr, ra);
+        tmem_ld_wait(ra);
+        tmem_ld32_issue(taddr + 32, rb);
+        fold32(ra, 0);
+        tmem_ld_wait(rb);
+        tmem_ld32_issue(taddr + 64, ra);
+        fold32(rb, 32);
+        tmem_ld_wait(ra);
+        tmem_ld32_issue(taddr + 96, rb);
+        fold32(ra, 64);
+        tmem_ld_wait(rb);
         tc_fence_before_sync();
-        mbar_arrive(t_empty(buf));
-        ml_s[blk][tid] = ml;
+        mbar_arrive(t_empty(buf));  // the accumulator is in registers: hand the buffer back early
+        fold32(rb, 96);
+        ml_s[grp][blk][ct] = ml;
       }
     }
     if (!kVotes && !ctl.abort) {
       for (int blk = 0; blk < a.n_blocks; ++blk) {
-        const int row = blk * 128 + tid;
-        if (row < a.GW) a.stat_part[((size_t)hq0 * a.W + row) * a.n_splits + split] = ml_s[blk][tid];
+        const int row = blk * 128 + ct;
+        if (row < a.GW)
+          a.stat_part[(((size_t)hq0 * a.W + row) * a.n_splits + split) * kGroups + grp] = ml_s[grp][blk][ct];
       }
     }
   }
@@ -223,7 +274,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
   }
   tc_fence_before_sync();
   __syncthreads();
-  if (warp == 5) tmem_dealloc(tmem_base, kTmemCols);
+  if (warp == kMmaWarp) tmem_dealloc(tmem_base, kTmemCols);
 }
 
 // Combine the per-split statistics of every observation row into its natural-log LSE.
@@ -238,6 +289,11 @@ __global__ void row_lse_from_splits_kernel(const float2* __restrict__ stat_part,
   for (int i = 0; i < n_splits; ++i)
     if (p[i].x > -INFINITY) l += p[i].y * exp2f(p[i].x - m);
   row_lse[r] = (m + log2f(l)) * kLn2;
+}
+
+__global__ void add_votes_kernel(float* __restrict__ vote, const float* __restrict__ vote2, size_t n) {
+  const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < n) vote[i] += vote2[i];
 }
 
 template <bool kVotes>
@@ -285,8 +341,10 @@ cudaError_t launch_row_stats_tc(const CompressGeom& g, const CompressWs& ws, con
   a.n_blocks = (GW + 127) / 128;
   a.block_rows = 128;
   a.n_tiles = (g.L + kTileKeys - 1) / kTileKeys;
+  a.n_buf = 4;
+  a.buf_cols = 128;
   a.n_splits = pick_tile_splits(g.units, a.n_tiles, 4);
-  if (a.n_splits > ws.n_tiles) a.n_splits = ws.n_tiles;
+  if (a.n_splits * kGroups > ws.stat_slots) a.n_splits = ws.stat_slots / kGroups;
   a.stages = a.n_blocks <= 3 ? 3 : 2;
   a.scale2 = g.scale2;
   a.stat_part = (float2*)(wsp + ws.stat_part);
@@ -304,7 +362,7 @@ cudaError_t launch_row_stats_tc(const CompressGeom& g, const CompressWs& ws, con
   score_tc_kernel<false><<<dim3(a.n_splits, g.units), kThreads, smem, st>>>(qm, km, a);
   const int rows = g.B * g.Hq * g.W;
   row_lse_from_splits_kernel<<<(rows + 127) / 128, 128, 0, st>>>(a.stat_part, (float*)(wsp + ws.row_lse), rows,
-                                                                 a.n_splits);
+                                                                 a.n_splits * kGroups);
   count_launch(2);
   return cudaGetLastError();
 }
@@ -315,14 +373,19 @@ cudaError_t launch_votes_tc(const CompressGeom& g, const CompressWs& ws, const v
   const int GW = g.G * g.W;
   ScoreArgs a{};
   a.Hq = g.Hq; a.G = g.G; a.W = g.W; a.L = g.L; a.n_cand = g.n_cand; a.GW = GW;
-  a.n_blocks = (GW + 255) / 256;
+  // One accumulator of up to 256 row columns per (key tile, row block); with two row blocks each
+  // warpgroup sums one block and the two partial votes are added afterwards.
+  a.n_blocks = GW <= 256 ? 1 : 2;
   a.block_rows = ((GW + a.n_blocks - 1) / a.n_blocks + 31) / 32 * 32;
+  a.n_buf = 2;
+  a.buf_cols = 256;
   a.n_tiles = (g.n_cand + kTileKeys - 1) / kTileKeys;
   a.n_splits = pick_tile_splits(g.units, a.n_tiles, 4);
-  a.stages = 3;
+  a.stages = a.n_blocks * a.block_rows <= 384 ? 3 : 2;
   a.scale2 = g.scale2;
   a.row_lse = row_lse;
   a.vote = (float*)(wsp + ws.vote);
+  a.vote2 = (float*)(wsp + ws.vote2);
   a.status = (unsigned*)(wsp + ws.status);
   CUtensorMap qm, km;
   const uint64_t qd[2] = {(uint64_t)GW, (uint64_t)g.units}, qs[2] = {256, (uint64_t)GW * 256};
@@ -336,6 +399,11 @@ cudaError_t launch_votes_tc(const CompressGeom& g, const CompressWs& ws, const v
   if (e != cudaSuccess) return e;
   score_tc_kernel<true><<<dim3(a.n_splits, g.units), kThreads, smem, st>>>(qm, km, a);
   count_launch(1);
+  if (a.n_blocks == 2) {
+    const size_t n = (size_t)g.units * g.n_cand;
+    add_votes_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(a.vote, a.vote2, n);
+    count_launch(1);
+  }
   return cudaGetLastError();
 }
 

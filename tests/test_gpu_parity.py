@@ -34,6 +34,9 @@ SMALL = [
     (2, 6, 3, 1301, 32, 5, 64, 32),      # spans several 128-key tiles with a ragged tail
     (1, 4, 4, 130, 64, 7, 65, 64),       # L - W < one tile, k_sel = 1
     (1, 2, 1, 96, 8, 7, 95, 3),          # a single evicted candidate
+    (1, 7, 1, 700, 64, 7, 160, 64),      # 448 window rows per kv head: two row blocks in the vote pass
+    (1, 16, 2, 900, 64, 5, 200, 16),     # G = 8, W = 64: 512 window rows, four 128-row statistic blocks
+    (1, 4, 1, 3000, 128, 7, 400, 128),   # W = 128: one query head per calibration row block
 ]
 
 
