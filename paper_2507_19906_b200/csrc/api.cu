@@ -78,7 +78,7 @@ CompressWs make_ws(const CompressGeom& g) {
   w.row_lse = off; off = align_up(off + (size_t)g.B * g.Hq * g.W * 4, 256);
   w.bitmap = off;  off = align_up(off + (size_t)g.units * g.bitmap_words * 4, 256);
   w.n_tiles = (g.L + 127) / 128;
-  w.stat_slots = w.n_tiles > 128 ? w.n_tiles : 128;
+  w.stat_slots = w.n_tiles > 320 ? w.n_tiles : 320;
   w.stat_part = off; off = align_up(off + (size_t)g.B * g.Hq * g.W * w.stat_slots * 8, 256);
   w.status = off;    off = align_up(off + 4, 256);
   w.calib_o = w.calib_l = off;

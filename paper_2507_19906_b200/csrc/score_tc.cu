@@ -1,20 +1,25 @@
 // Window scoring on the tensor cores (tcgen05 MMA, accumulator in TMEM, operands fed by TMA).
 //
-// Two kernels over one skeleton.  A CTA owns one (batch, kv-head) unit and a contiguous range of
-// 128-key tiles; the unit's G*W observation rows stay resident in shared memory, the key tiles
-// stream through a TMA ring.  Warp roles: warps 0-3 read the accumulator out of TMEM (one TMEM
-// lane per thread), warp 4 is the TMA producer, warp 5 allocates TMEM and issues the MMAs.
+// Two kernels over one skeleton.  The work is the linear space of (virtual unit, key tile) pairs;
+// it is cut into equal contiguous ranges, one per CTA, and at most one CTA per SM is launched, so
+// a CTA streams a long run of key tiles through its TMA ring and pays its start-up once.  A
+// virtual unit is a (batch, kv-head) unit, or for the statistics one half of its window rows when
+// there are more than 256; its query rows stay resident in shared memory and are reloaded when
+// the CTA's range crosses into the next virtual unit.
+// Warp roles: two consumer warpgroups read the accumulators out of TMEM (one TMEM lane per
+// thread, group g owns accumulator buffer g), one warp is the TMA producer, one warp allocates TMEM
+// and issues the MMAs.  Every MMA has N = 256 where the shape allows it: with both operands in
+// shared memory, narrower tiles are limited by operand fetch, not by the tensor pipe.
 //
-//   statistics (kVotes = false):  S = Q K^T, query rows on the TMEM lanes.  Thread r keeps the
-//       running (max, sum) of exp2(scale2 * s) over the keys row r may see (causal inside the
-//       window).  Per-split partials are combined into the natural-log row LSE by
-//       row_lse_reduce_kernel.  Skipped altogether when the caller supplies the row LSE.
-//   votes (kVotes = true):  S^T = K Q^T, KEYS on the TMEM lanes, so the vote of a key,
-//       sum over rows of exp2(scale2 * s - lse2[row]), is a per-thread sum over the accumulator's
-//       columns: no cross-thread reduction and fp32 probabilities throughout.  Candidate keys
-//       (t < L - W) are seen by every window row, so this pass needs no mask.
-//
-// Both passes are co-limited by the tensor pipe and the exponential unit (one exp2 per logit).
+//   statistics (kVotes = false):  S = Q K^T, 128 query rows on the TMEM lanes, 256 keys per tile.
+//       Thread r keeps the running (max, sum) of exp2(scale2 * s) over the keys row r may see
+//       (causal inside the window).  Per-CTA partials are combined into the natural-log row LSE by
+//       row_lse_from_parts_kernel.  Skipped altogether when the caller supplies the row LSE.
+//   votes (kVotes = true):  S^T = K Q^T, 128 KEYS on the TMEM lanes and up to 256 query rows as
+//       columns, so the vote of a key, sum over rows of exp2(scale2 * s - lse2[row]), is a
+//       per-thread sum over the accumulator's columns: no cross-thread reduction and fp32
+//       probabilities throughout.  Candidate keys (t < L - W) are seen by every window row, so this
+//       pass needs no mask.
 #include "internal.h"
 #include "tc_common.cuh"
 
@@ -24,28 +29,31 @@ namespace {
 
 using namespace tc;
 
-constexpr int kGroups = 2;                       // consumer warpgroups (4 warps each)
-constexpr int kConsumers = kGroups * 128;
+constexpr int kGroups = 2;  // consumer warpgroups (4 warps each); group g consumes accumulator g
 constexpr int kProducerWarp = kGroups * 4;
 constexpr int kMmaWarp = kGroups * 4 + 1;
-constexpr int kThreads = kConsumers + 64;
-constexpr int kTmemCols = 512;
-constexpr int kMaxRows = 512;  // G * W handled by the tiles
+constexpr int kThreads = kGroups * 128 + 64;
+constexpr int kTmemCols = 512;  // two accumulators of 256 columns
+constexpr int kBufCols = 256;
+constexpr int kMaxRows = 512;   // G * W handled by the tiles
+constexpr int kSms = 148;
 
 struct ScoreArgs {
   int Hq, G, W, L, n_cand, GW;
-  int n_blocks;    // blocks of observation rows
-  int block_rows;  // rows per block: 128 for the statistics; a multiple of 32 (<= 256) for the votes
-  int n_buf;       // accumulator ring in TMEM: n_buf buffers of buf_cols columns (n_buf * buf_cols = 512)
-  int buf_cols;
-  int n_tiles;     // key tiles to cover
-  int n_splits;
-  int stages;      // depth of the key-tile ring (2 or 3)
+  int vu_per_unit;    // virtual units per (batch, kv-head) unit
+  int vu_rows;        // window rows a virtual unit starts at: vu % vu_per_unit * vu_rows
+  int n_blocks;       // row blocks (= accumulators) per key tile
+  int block_rows;     // rows per block: 128 for the statistics, a multiple of 32 (<= 256) for the votes
+  int n_tiles;        // key tiles per virtual unit
+  int total_tiles;    // virtual units * n_tiles
+  int tiles_per_cta;
+  int stages;         // depth of the key-tile ring
+  int max_slots;      // statistics: partial slots per row (CTAs that can share a virtual unit)
   float scale2;
   const float* row_lse;  // votes: natural-log LSE of every observation row [B, Hq, W]
   float* vote;           // votes: out [units, n_cand]
-  float* vote2;          // votes of the second row block when there are two (summed into vote afterwards)
-  float2* stat_part;     // statistics: out [row][split][group] (max, sum) in the log2 domain
+  float* vote2;          // votes of the second row block when there are two (added to vote afterwards)
+  float2* stat_part;     // statistics: out [row][slot][group] (max, sum) in the log2 domain
   unsigned* status;
 };
 
@@ -74,23 +82,26 @@ __device__ __forceinline__ float max_32(const uint32_t (&r)[32]) {
   return fmaxf(fmaxf(m0, m1), fmaxf(m2, m3));
 }
 
+
 template <bool kVotes>
 __global__ void __launch_bounds__(kThreads, 1)
 score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__ CUtensorMap k_map,
                 const ScoreArgs a) {
+  constexpr int TILE_KEYS = kVotes ? 128 : 256;
+  constexpr uint32_t STAGE_BYTES = TILE_KEYS * 256;
   extern __shared__ unsigned char smem_raw[];
   __shared__ __align__(8) unsigned long long bars[16];
   __shared__ uint32_t tmem_slot;
   __shared__ Ctl ctl;
-  __shared__ __align__(16) float nlse2_s[kVotes ? kMaxRows : 4];  // -log2-domain LSE per row (-inf: padding)
-  __shared__ float2 ml_s[kVotes ? 1 : kGroups][kVotes ? 1 : 4][kVotes ? 1 : 128];  // running (max, sum)
+  __shared__ __align__(16) float nlse2_s[kVotes ? kGroups * 4 : 1][kVotes ? kMaxRows : 4];  // -lse2 per row, one copy per warp
+  __shared__ float2 ml_s[kVotes ? 1 : kGroups][kVotes ? 1 : 2][kVotes ? 1 : 128];       // running (max, sum)
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int split = blockIdx.x, unit = blockIdx.y;
-  const int tile0 = (int)((long long)a.n_tiles * split / a.n_splits);
-  const int tile1 = (int)((long long)a.n_tiles * (split + 1) / a.n_splits);
-  const int nt = tile1 - tile0;
-  const int n_jobs = nt * a.n_blocks;  // one job = one (key tile, row block) accumulator
+  const int cta = blockIdx.x;
+  const int g_begin = cta * a.tiles_per_cta;
+  const int g_end = min(a.total_tiles, g_begin + a.tiles_per_cta);
+  const int nt = g_end - g_begin;
+  const int Hkv = a.Hq / a.G;
 
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   const uint32_t q_half_bytes = (uint32_t)a.block_rows * kLineBytes;
@@ -99,28 +110,24 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
   const uint32_t k_base = q_base + (uint32_t)a.n_blocks * q_blk_bytes;
 
   const uint32_t bar0 = smem_u32(bars);
-  const uint32_t q_full = bar0;
-  auto full_k = [&](int s) { return bar0 + 8u * (1 + s); };
-  auto empty_k = [&](int s) { return bar0 + 8u * (4 + s); };
-  auto t_full = [&](int b) { return bar0 + 8u * (7 + b); };
-  auto t_empty = [&](int b) { return bar0 + 8u * (11 + b); };
+  const uint32_t q_full = bar0, q_empty = bar0 + 8u;
+  auto full_k = [&](int s) { return bar0 + 8u * (2 + s); };
+  auto empty_k = [&](int s) { return bar0 + 8u * (6 + s); };
+  auto t_full = [&](int b) { return bar0 + 8u * (10 + b); };
+  auto t_empty = [&](int b) { return bar0 + 8u * (12 + b); };
 
   if (tid == 0) {
     ctl.abort = 0;
     ctl.status = a.status;
     mbar_init(q_full, 1);
-    for (int s = 0; s < 3; ++s) { mbar_init(full_k(s), 1); mbar_init(empty_k(s), 1); }
-    for (int b = 0; b < 4; ++b) { mbar_init(t_full(b), 1); mbar_init(t_empty(b), 128); }
+    mbar_init(q_empty, 1);
+    for (int s = 0; s < 4; ++s) { mbar_init(full_k(s), 1); mbar_init(empty_k(s), 1); }
+    for (int b = 0; b < 2; ++b) { mbar_init(t_full(b), 1); mbar_init(t_empty(b), 128); }
     fence_mbar_init();
   }
   if (warp == kMmaWarp) {
     tmem_alloc(smem_u32(&tmem_slot), kTmemCols);
     tmem_relinquish();
-  }
-  const int hq0 = (unit / (a.Hq / a.G)) * a.Hq + (unit % (a.Hq / a.G)) * a.G;  // first query head of the unit
-  if (kVotes) {
-    for (int r = tid; r < kMaxRows; r += kThreads)
-      nlse2_s[r] = r < a.GW ? -a.row_lse[(size_t)hq0 * a.W + r] * kLog2e : -INFINITY;
   }
   tc_fence_before_sync();
   __syncthreads();
@@ -132,140 +139,190 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
     if (lane == 0) {
       tma_prefetch_desc(&q_map);
       tma_prefetch_desc(&k_map);
-      mbar_arrive_expect_tx(q_full, (uint32_t)a.n_blocks * q_blk_bytes);
-      for (int blk = 0; blk < a.n_blocks; ++blk)
-        for (int half = 0; half < 2; ++half)
-          tma_load_3d(q_base + blk * q_blk_bytes + half * q_half_bytes, &q_map, q_full, half * kHalfCols,
-                      blk * a.block_rows, unit);
+      int cur_vu = -1, seg = 0;
       for (int i = 0; i < nt; ++i) {
+        const int g = g_begin + i;
+        const int vu = g / a.n_tiles, tile = g - vu * a.n_tiles;
+        const int unit = vu / a.vu_per_unit;
+        if (vu != cur_vu) {
+          // the query rows of the next virtual unit replace the current ones once its MMAs are done
+          if (seg > 0 && !mbar_wait(&ctl, q_empty, (seg - 1) & 1, (kVotes ? 36u : 16u) | ((unsigned)i << 8))) break;
+          const int row0 = (vu - unit * a.vu_per_unit) * a.vu_rows;
+          mbar_arrive_expect_tx(q_full, (uint32_t)a.n_blocks * q_blk_bytes);
+          for (int blk = 0; blk < a.n_blocks; ++blk)
+            for (int half = 0; half < 2; ++half)
+              tma_load_3d(q_base + blk * q_blk_bytes + half * q_half_bytes, &q_map, q_full, half * kHalfCols,
+                          row0 + blk * a.block_rows, unit);
+          cur_vu = vu;
+          ++seg;
+        }
         const int s = i % a.stages;
         if (!mbar_wait(&ctl, empty_k(s), ((i / a.stages) & 1) ^ 1, (kVotes ? 31u : 11u) | ((unsigned)i << 8))) break;
-        mbar_arrive_expect_tx(full_k(s), kKvTileBytes);
+        mbar_arrive_expect_tx(full_k(s), STAGE_BYTES);
         for (int half = 0; half < 2; ++half)
-          tma_load_3d(k_base + s * kKvTileBytes + half * (kKvTileBytes / 2), &k_map, full_k(s), half * kHalfCols,
-                      (tile0 + i) * kTileKeys, unit);
+          tma_load_3d(k_base + s * STAGE_BYTES + half * (STAGE_BYTES / 2), &k_map, full_k(s), half * kHalfCols,
+                      tile * TILE_KEYS, unit);
       }
     }
   } else if (warp == kMmaWarp) {
     // ------------------------------------------------------------ MMA issuer
     if (lane == 0) {
-      const uint32_t idesc = umma_idesc(128, kVotes ? a.block_rows : 128, false, false);
-      bool ok = mbar_wait(&ctl, q_full, 0, kVotes ? 32u : 12u);
-      for (int j = 0; ok && j < n_jobs; ++j) {
-        const int i = j / a.n_blocks, blk = j - i * a.n_blocks;
-        const int s = i % a.stages, buf = j % a.n_buf;
-        if (blk == 0 && !mbar_wait(&ctl, full_k(s), (i / a.stages) & 1, (kVotes ? 33u : 13u) | ((unsigned)j << 8))) break;
-        if (!mbar_wait(&ctl, t_empty(buf), ((j / a.n_buf) & 1) ^ 1, (kVotes ? 34u : 14u) | ((unsigned)j << 8))) break;
-        tc_fence_after_sync();
-        const uint32_t d = tmem_base + (uint32_t)(buf * a.buf_cols);
-        const uint32_t kt = k_base + (uint32_t)s * kKvTileBytes, qt = q_base + (uint32_t)blk * q_blk_bytes;
-#pragma unroll
-        for (int kk = 0; kk < kD / 16; ++kk) {
-          const uint64_t kd = kmajor_desc(kt, kKvTileBytes / 2, kk);
-          const uint64_t qd = kmajor_desc(qt, q_half_bytes, kk);
-          umma_ss(d, kVotes ? kd : qd, kVotes ? qd : kd, idesc, kk > 0 ? 1u : 0u);
+      const uint32_t idesc = umma_idesc(128, kVotes ? a.block_rows : 256, false, false);
+      int cur_vu = -1, seg = 0, j = 0;
+      for (int i = 0; i < nt; ++i) {
+        const int g = g_begin + i;
+        const int vu = g / a.n_tiles;
+        if (vu != cur_vu) {
+          if (!mbar_wait(&ctl, q_full, seg & 1, (kVotes ? 32u : 12u) | ((unsigned)i << 8))) break;
+          cur_vu = vu;
+          ++seg;
         }
-        umma_commit(t_full(buf));
-        if (blk == a.n_blocks - 1) umma_commit(empty_k(s));
+        const int s = i % a.stages;
+        if (!mbar_wait(&ctl, full_k(s), (i / a.stages) & 1, (kVotes ? 33u : 13u) | ((unsigned)i << 8))) break;
+        bool ok = true;
+        for (int blk = 0; blk < a.n_blocks; ++blk, ++j) {
+          const int buf = j & 1;
+          if (!mbar_wait(&ctl, t_empty(buf), ((j >> 1) & 1) ^ 1, (kVotes ? 34u : 14u) | ((unsigned)j << 8))) {
+            ok = false;
+            break;
+          }
+          tc_fence_after_sync();
+          const uint32_t d = tmem_base + (uint32_t)(buf * kBufCols);
+          const uint32_t kt = k_base + (uint32_t)s * STAGE_BYTES, qt = q_base + (uint32_t)blk * q_blk_bytes;
+#pragma unroll
+          for (int kk = 0; kk < kD / 16; ++kk) {
+            const uint64_t kd = kmajor_desc(kt, STAGE_BYTES / 2, kk);
+            const uint64_t qd = kmajor_desc(qt, q_half_bytes, kk);
+            umma_ss(d, kVotes ? kd : qd, kVotes ? qd : kd, idesc, kk > 0 ? 1u : 0u);
+          }
+          umma_commit(t_full(buf));
+        }
+        if (!ok) break;
+        umma_commit(empty_k(s));
+        const bool last_of_vu = (i == nt - 1) || ((g + 1) / a.n_tiles != vu);
+        if (last_of_vu) umma_commit(q_empty);
       }
     }
   } else {
     // ------------------------------------------------------------ accumulator consumers
-    // Warpgroup `grp` takes the jobs with job % kGroups == grp; thread ct of a group owns TMEM
-    // lane ct.  The launch shapes keep n_buf a multiple of kGroups, so an accumulator buffer (and
-    // its pair of mbarriers) is only ever consumed by one group and every group sees each phase
-    // of the barriers it waits on.
+    // Thread ct of warpgroup grp owns TMEM lane ct and consumes the jobs (key tile, row block) whose
+    // running index is congruent to grp mod 2, i.e. the accumulator buffer grp.
     const int grp = warp >> 2, ct = tid & 127;
-    const uint32_t lane_addr = tmem_base + ((uint32_t)((warp & 3) * 32) << 16);
+    const uint32_t lane_addr = tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)(grp * kBufCols);
     float acc0 = 0.f, acc1 = 0.f, acc2 = 0.f, acc3 = 0.f;  // votes: running vote of this thread's key
-    if (!kVotes) {
-      for (int blk = 0; blk < 4; ++blk) ml_s[grp][blk][ct] = make_float2(-INFINITY, 0.f);
-    }
-    for (int j = 0; j < n_jobs; ++j) {
-      const int i = j / a.n_blocks, blk = j - i * a.n_blocks;
-      if (j % kGroups != grp) continue;
-      const int buf = j % a.n_buf;
-      bool ok = mbar_wait(&ctl, t_full(buf), (j / a.n_buf) & 1, (kVotes ? 35u : 15u) | ((unsigned)j << 8));
-      if (!__all_sync(0xffffffffu, ok)) break;
-      tc_fence_after_sync();
-      const int tbase = (tile0 + i) * kTileKeys;
-      const uint32_t taddr = lane_addr + (uint32_t)(buf * a.buf_cols);
-      uint32_t ra[32], rb[32];
-      if (kVotes) {
-        const float* nl = nlse2_s + blk * a.block_rows;
-        auto add32 = [&](const uint32_t (&r)[32], int c0) {
-#pragma unroll
-          for (int e = 0; e < 32; e += 4) {
-            const float4 n4 = *reinterpret_cast<const float4*>(nl + c0 + e);
-            acc0 += ex2_approx(fmaf(__uint_as_float(r[e + 0]), a.scale2, n4.x));
-            acc1 += ex2_approx(fmaf(__uint_as_float(r[e + 1]), a.scale2, n4.y));
-            acc2 += ex2_approx(fmaf(__uint_as_float(r[e + 2]), a.scale2, n4.z));
-            acc3 += ex2_approx(fmaf(__uint_as_float(r[e + 3]), a.scale2, n4.w));
-          }
-        };
-        // block_rows is a multiple of 32: chunks alternate between the two register sets
-        tmem_ld32_issue(taddr, ra);
-        for (int c0 = 0; c0 < a.block_rows; c0 += 64) {
-          tmem_ld_wait(ra);
-          const bool more_b = c0 + 32 < a.block_rows;
-          if (more_b) tmem_ld32_issue(taddr + c0 + 32, rb);
-          add32(ra, c0);
-          if (more_b) {
-            tmem_ld_wait(rb);
-            if (c0 + 64 < a.block_rows) tmem_ld32_issue(taddr + c0 + 64, ra);
-            add32(rb, c0 + 32);
-          }
+    int cur_vu = -1, j = 0;
+    bool ok = true;
+
+    // statistics: store this group's partial (max, sum) of every row of the virtual unit `vu`
+    auto flush_stats = [&](int vu) {
+      const int unit = vu / a.vu_per_unit;
+      const int hq0 = (unit / Hkv) * a.Hq + (unit % Hkv) * a.G;
+      const int row0 = (vu - unit * a.vu_per_unit) * a.vu_rows;
+      const int slot = cta - (vu * a.n_tiles) / a.tiles_per_cta;
+      for (int blk = 0; blk < a.n_blocks; ++blk) {
+        const int row = row0 + blk * 128 + ct;
+        if (row < a.GW)
+          a.stat_part[(((size_t)hq0 * a.W + row) * a.max_slots + slot) * kGroups + grp] = ml_s[grp][blk][ct];
+      }
+    };
+
+    for (int i = 0; i < nt && ok; ++i) {
+      const int g = g_begin + i;
+      const int vu = g / a.n_tiles, tile = g - vu * a.n_tiles;
+      const int unit = vu / a.vu_per_unit;
+      const int row0 = (vu - unit * a.vu_per_unit) * a.vu_rows;
+      if (vu != cur_vu) {
+        if (kVotes) {
+          // this warp's copy of -lse2 of the unit's window rows (-inf for the padding rows); warps
+          // keep their own copy so that no barrier wider than a warp is needed here
+          const int hq0 = (unit / Hkv) * a.Hq + (unit % Hkv) * a.G;
+          __syncwarp();
+          for (int r = lane; r < kMaxRows; r += 32)
+            nlse2_s[warp][r] = r < a.GW ? -a.row_lse[(size_t)hq0 * a.W + r] * kLog2e : -INFINITY;
+          __syncwarp();
+        } else {
+          if (cur_vu >= 0) flush_stats(cur_vu);
+          for (int blk = 0; blk < 2; ++blk) ml_s[grp][blk][ct] = make_float2(-INFINITY, 0.f);
         }
-        tc_fence_before_sync();
-        mbar_arrive(t_empty(buf));
-        {
+        cur_vu = vu;
+      }
+      const int tbase = tile * TILE_KEYS;
+      for (int blk = 0; blk < a.n_blocks; ++blk, ++j) {
+        if ((j & 1) != grp) continue;
+        ok = mbar_wait(&ctl, t_full(grp), (j >> 1) & 1, (kVotes ? 35u : 15u) | ((unsigned)j << 8));
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) break;
+        tc_fence_after_sync();
+        uint32_t ra[32], rb[32];
+        if (kVotes) {
+          const float* nl = nlse2_s[warp] + blk * a.block_rows;
+          auto add32 = [&](const uint32_t (&r)[32], int c0) {
+#pragma unroll
+            for (int e = 0; e < 32; e += 4) {
+              const float4 n4 = *reinterpret_cast<const float4*>(nl + c0 + e);
+              acc0 += ex2_approx(fmaf(__uint_as_float(r[e + 0]), a.scale2, n4.x));
+              acc1 += ex2_approx(fmaf(__uint_as_float(r[e + 1]), a.scale2, n4.y));
+              acc2 += ex2_approx(fmaf(__uint_as_float(r[e + 2]), a.scale2, n4.z));
+              acc3 += ex2_approx(fmaf(__uint_as_float(r[e + 3]), a.scale2, n4.w));
+            }
+          };
+          // block_rows is a multiple of 32: chunks alternate between the two register sets
+          tmem_ld32_issue(lane_addr, ra);
+          for (int c0 = 0; c0 < a.block_rows; c0 += 64) {
+            tmem_ld_wait(ra);
+            const bool more_b = c0 + 32 < a.block_rows;
+            if (more_b) tmem_ld32_issue(lane_addr + c0 + 32, rb);
+            add32(ra, c0);
+            if (more_b) {
+              tmem_ld_wait(rb);
+              if (c0 + 64 < a.block_rows) tmem_ld32_issue(lane_addr + c0 + 64, ra);
+              add32(rb, c0 + 32);
+            }
+          }
+          tc_fence_before_sync();
+          mbar_arrive(t_empty(grp));
           const int key = tbase + ct;
           float* out = blk == 0 ? a.vote : a.vote2;
           if (key < a.n_cand) out[(size_t)unit * a.n_cand + key] = (acc0 + acc1) + (acc2 + acc3);
           acc0 = acc1 = acc2 = acc3 = 0.f;
-        }
-      } else {
-        float2 ml = ml_s[grp][blk][ct];
-        const int row = blk * 128 + ct;
-        // local index of the last key this row may see inside the tile (causal inside the window)
-        const int lim = min(a.L - 1, a.n_cand + row % a.W) - tbase;
-        const bool full_tile = __all_sync(0xffffffffu, lim >= kTileKeys - 1);
-        auto fold32 = [&](uint32_t (&r)[32], int c0) {
-          if (!full_tile) {
+        } else {
+          float2 ml = ml_s[grp][blk][ct];
+          const int row = row0 + blk * 128 + ct;
+          // local index of the last key this row may see inside the tile (causal inside the window)
+          const int lim = min(a.L - 1, a.n_cand + row % a.W) - tbase;
+          const bool full_tile = __all_sync(0xffffffffu, lim >= TILE_KEYS - 1);
+          auto fold32 = [&](uint32_t (&r)[32], int c0) {
+            if (!full_tile) {
 #pragma unroll
-            for (int e = 0; e < 32; ++e)
-              if (c0 + e > lim) r[e] = 0xff800000u;  // -inf
+              for (int e = 0; e < 32; ++e)
+                if (c0 + e > lim) r[e] = 0xff800000u;  // -inf
+            }
+            const float m_new = fmaxf(ml.x, max_32(r) * a.scale2);
+            if (m_new > -INFINITY) {
+              ml.y = ml.y * ex2_approx(ml.x - m_new) + sum_exp2_32(r, a.scale2, -m_new);
+              ml.x = m_new;
+            }
+          };
+          tmem_ld32_issue(lane_addr, ra);
+#pragma unroll 1
+          for (int c0 = 0; c0 < TILE_KEYS; c0 += 64) {
+            tmem_ld_wait(ra);
+            tmem_ld32_issue(lane_addr + c0 + 32, rb);
+            fold32(ra, c0);
+            tmem_ld_wait(rb);
+            if (c0 + 64 < TILE_KEYS) {
+              tmem_ld32_issue(lane_addr + c0 + 64, ra);
+            } else {
+              tc_fence_before_sync();
+              mbar_arrive(t_empty(grp));  // the accumulator is in registers: hand the buffer back early
+            }
+            fold32(rb, c0 + 32);
           }
-          const float m_new = fmaxf(ml.x, max_32(r) * a.scale2);
-          if (m_new > -INFINITY) {
-            ml.y = ml.y * ex2_approx(ml.x - m_new) + sum_exp2_32(r, a.scale2, -m_new);
-            ml.x = m_new;
-          }
-        };
-        tmem_ld32_issue(taddr, ra);
-        tmem_ld_wait(ra);
-        tmem_ld32_issue(taddr + 32, rb);
-        fold32(ra, 0);
-        tmem_ld_wait(rb);
-        tmem_ld32_issue(taddr + 64, ra);
-        fold32(rb, 32);
-        tmem_ld_wait(ra);
-        tmem_ld32_issue(taddr + 96, rb);
-        fold32(ra, 64);
-        tmem_ld_wait(rb);
-        tc_fence_before_sync();
-        mbar_arrive(t_empty(buf));  // the accumulator is in registers: hand the buffer back early
-        fold32(rb, 96);
-        ml_s[grp][blk][ct] = ml;
+          ml_s[grp][blk][ct] = ml;
+        }
       }
     }
-    if (!kVotes && !ctl.abort) {
-      for (int blk = 0; blk < a.n_blocks; ++blk) {
-        const int row = blk * 128 + ct;
-        if (row < a.GW)
-          a.stat_part[(((size_t)hq0 * a.W + row) * a.n_splits + split) * kGroups + grp] = ml_s[grp][blk][ct];
-      }
-    }
+    if (!kVotes && ok && cur_vu >= 0 && !ctl.abort) flush_stats(cur_vu);
   }
 
   // ---------------------------------------------------------------- teardown (every path)
@@ -277,16 +334,22 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
   if (warp == kMmaWarp) tmem_dealloc(tmem_base, kTmemCols);
 }
 
-// Combine the per-split statistics of every observation row into its natural-log LSE.
-__global__ void row_lse_from_splits_kernel(const float2* __restrict__ stat_part, float* __restrict__ row_lse,
-                                           int rows, int n_splits) {
+// Combine the partial statistics of every observation row into its natural-log LSE.  The
+// partials of a row are those of the CTAs whose tile range overlaps the row's virtual unit.
+__global__ void row_lse_from_parts_kernel(const float2* __restrict__ stat_part, float* __restrict__ row_lse,
+                                          int rows, int GW, int vu_per_unit, int n_tiles, int tiles_per_cta,
+                                          int max_slots) {
   const int r = blockIdx.x * blockDim.x + threadIdx.x;
   if (r >= rows) return;
-  const float2* p = stat_part + (size_t)r * n_splits;
+  const int unit = r / GW, row = r - unit * GW;
+  const int vu = unit * vu_per_unit + row / 256;
+  const int first = (vu * n_tiles) / tiles_per_cta, last = ((vu + 1) * n_tiles - 1) / tiles_per_cta;
+  const int n = (last - first + 1) * kGroups;
+  const float2* p = stat_part + (size_t)r * max_slots * kGroups;
   float m = -INFINITY;
-  for (int i = 0; i < n_splits; ++i) m = fmaxf(m, p[i].x);
+  for (int i = 0; i < n; ++i) m = fmaxf(m, p[i].x);
   float l = 0.f;
-  for (int i = 0; i < n_splits; ++i)
+  for (int i = 0; i < n; ++i)
     if (p[i].x > -INFINITY) l += p[i].y * exp2f(p[i].x - m);
   row_lse[r] = (m + log2f(l)) * kLn2;
 }
@@ -308,12 +371,18 @@ cudaError_t set_smem_limit(int bytes) {
   return e;
 }
 
+// Equal contiguous tile ranges over at most one CTA per SM.
+void partition_tiles(ScoreArgs& a, int virtual_units) {
+  a.total_tiles = virtual_units * a.n_tiles;
+  const int ctas = a.total_tiles < kSms ? a.total_tiles : kSms;
+  a.tiles_per_cta = (a.total_tiles + ctas - 1) / ctas;
+}
+
 }  // namespace
 
 // Number of key-range splits per work group so that `groups * splits` CTAs fill whole waves of
 // the 148 SMs (one CTA per SM) while every CTA keeps at least `min_tiles` tiles.
 int pick_tile_splits(int groups, int n_tiles, int min_tiles) {
-  const int kSms = 148;
   int max_s = n_tiles / (min_tiles > 0 ? min_tiles : 1);
   if (max_s < 1) max_s = 1;
   if (max_s > 64) max_s = 64;
@@ -338,14 +407,15 @@ cudaError_t launch_row_stats_tc(const CompressGeom& g, const CompressWs& ws, con
   const int GW = g.G * g.W;
   ScoreArgs a{};
   a.Hq = g.Hq; a.G = g.G; a.W = g.W; a.L = g.L; a.n_cand = g.n_cand; a.GW = GW;
-  a.n_blocks = (GW + 127) / 128;
+  a.vu_per_unit = (GW + 255) / 256;
+  a.vu_rows = 256;
+  a.n_blocks = GW <= 128 ? 1 : 2;
   a.block_rows = 128;
-  a.n_tiles = (g.L + kTileKeys - 1) / kTileKeys;
-  a.n_buf = 4;
-  a.buf_cols = 128;
-  a.n_splits = pick_tile_splits(g.units, a.n_tiles, 4);
-  if (a.n_splits * kGroups > ws.stat_slots) a.n_splits = ws.stat_slots / kGroups;
-  a.stages = a.n_blocks <= 3 ? 3 : 2;
+  a.n_tiles = (g.L + 255) / 256;
+  partition_tiles(a, g.units * a.vu_per_unit);
+  a.max_slots = (a.n_tiles + a.tiles_per_cta - 1) / a.tiles_per_cta + 1;
+  if (a.max_slots * kGroups > ws.stat_slots) return cudaErrorInvalidValue;
+  a.stages = 2;  // 64 KB tiles of 256 keys
   a.scale2 = g.scale2;
   a.stat_part = (float2*)(wsp + ws.stat_part);
   a.status = (unsigned*)(wsp + ws.status);
@@ -353,16 +423,18 @@ cudaError_t launch_row_stats_tc(const CompressGeom& g, const CompressWs& ws, con
   const uint64_t qd[2] = {(uint64_t)GW, (uint64_t)g.units}, qs[2] = {256, (uint64_t)GW * 256};
   const uint32_t qb[2] = {128, 1};
   const uint64_t kd[2] = {(uint64_t)g.L, (uint64_t)g.units}, ks[2] = {256, (uint64_t)g.L * 256};
-  const uint32_t kb[2] = {(uint32_t)kTileKeys, 1};
+  const uint32_t kb[2] = {256, 1};
   if (!make_tensor_map_bf16(&qm, Q_obs, 3, qd, qs, qb) || !make_tensor_map_bf16(&km, K, 3, kd, ks, kb))
     return cudaErrorInvalidValue;
-  const int smem = a.n_blocks * 128 * 256 + a.stages * kKvTileBytes + 1024;
+  const int smem = a.n_blocks * 128 * 256 + a.stages * 256 * 256 + 1024;
   cudaError_t e = set_smem_limit<false>(smem);
   if (e != cudaSuccess) return e;
-  score_tc_kernel<false><<<dim3(a.n_splits, g.units), kThreads, smem, st>>>(qm, km, a);
+  const int grid = (a.total_tiles + a.tiles_per_cta - 1) / a.tiles_per_cta;
+  score_tc_kernel<false><<<grid, kThreads, smem, st>>>(qm, km, a);
   const int rows = g.B * g.Hq * g.W;
-  row_lse_from_splits_kernel<<<(rows + 127) / 128, 128, 0, st>>>(a.stat_part, (float*)(wsp + ws.row_lse), rows,
-                                                                 a.n_splits * kGroups);
+  row_lse_from_parts_kernel<<<(rows + 127) / 128, 128, 0, st>>>(a.stat_part, (float*)(wsp + ws.row_lse), rows, GW,
+                                                                a.vu_per_unit, a.n_tiles, a.tiles_per_cta,
+                                                                a.max_slots);
   count_launch(2);
   return cudaGetLastError();
 }
@@ -373,15 +445,16 @@ cudaError_t launch_votes_tc(const CompressGeom& g, const CompressWs& ws, const v
   const int GW = g.G * g.W;
   ScoreArgs a{};
   a.Hq = g.Hq; a.G = g.G; a.W = g.W; a.L = g.L; a.n_cand = g.n_cand; a.GW = GW;
+  a.vu_per_unit = 1;
+  a.vu_rows = 0;
   // One accumulator of up to 256 row columns per (key tile, row block); with two row blocks each
   // warpgroup sums one block and the two partial votes are added afterwards.
   a.n_blocks = GW <= 256 ? 1 : 2;
   a.block_rows = ((GW + a.n_blocks - 1) / a.n_blocks + 31) / 32 * 32;
-  a.n_buf = 2;
-  a.buf_cols = 256;
   a.n_tiles = (g.n_cand + kTileKeys - 1) / kTileKeys;
-  a.n_splits = pick_tile_splits(g.units, a.n_tiles, 4);
-  a.stages = a.n_blocks * a.block_rows <= 384 ? 3 : 2;
+  partition_tiles(a, g.units);
+  const int q_bytes = a.n_blocks * a.block_rows * 256;
+  a.stages = q_bytes <= 65536 ? 4 : (q_bytes <= 98304 ? 3 : 2);
   a.scale2 = g.scale2;
   a.row_lse = row_lse;
   a.vote = (float*)(wsp + ws.vote);
@@ -394,10 +467,11 @@ cudaError_t launch_votes_tc(const CompressGeom& g, const CompressWs& ws, const v
   const uint32_t kb[2] = {(uint32_t)kTileKeys, 1};
   if (!make_tensor_map_bf16(&qm, Q_obs, 3, qd, qs, qb) || !make_tensor_map_bf16(&km, K, 3, kd, ks, kb))
     return cudaErrorInvalidValue;
-  const int smem = a.n_blocks * a.block_rows * 256 + a.stages * kKvTileBytes + 1024;
+  const int smem = q_bytes + a.stages * kKvTileBytes + 1024;
   cudaError_t e = set_smem_limit<true>(smem);
   if (e != cudaSuccess) return e;
-  score_tc_kernel<true><<<dim3(a.n_splits, g.units), kThreads, smem, st>>>(qm, km, a);
+  const int grid = (a.total_tiles + a.tiles_per_cta - 1) / a.tiles_per_cta;
+  score_tc_kernel<true><<<grid, kThreads, smem, st>>>(qm, km, a);
   count_launch(1);
   if (a.n_blocks == 2) {
     const size_t n = (size_t)g.units * g.n_cand;

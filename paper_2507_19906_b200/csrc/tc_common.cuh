@@ -20,7 +20,9 @@
 namespace calidrop {
 namespace tc {
 
-constexpr unsigned long long kWaitLimitNs = 2000000000ull;  // 2 s per wait
+// Limit of one wait in SM clock cycles (about 2 s at the boost clock); the cycle counter is read
+// in a few cycles, so checking it costs nothing on waits entered thousands of times per CTA.
+constexpr long long kWaitLimitCycles = 4000000000ll;
 
 // ---------------------------------------------------------------- mbarrier
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
@@ -52,12 +54,6 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
       : "memory");
   return ok != 0;
 }
-__device__ __forceinline__ unsigned long long global_timer_ns() {
-  unsigned long long t;
-  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-  return t;
-}
-
 // Shared per-CTA control block of the bounded waits.
 struct Ctl {
   volatile int abort;       // raised by the first thread whose wait expired
@@ -68,12 +64,14 @@ struct Ctl {
 // (this wait expired, or another thread's did).
 __device__ __forceinline__ bool mbar_wait(Ctl* ctl, uint32_t bar, uint32_t parity, unsigned code) {
   if (mbar_try_wait(bar, parity)) return true;
-  const unsigned long long t0 = global_timer_ns();
+  long long t0 = 0;
   unsigned polls = 0;
   while (!mbar_try_wait(bar, parity)) {
-    if ((++polls & 255u) == 0u) {
+    if ((++polls & 1023u) == 0u) {
       if (ctl->abort) return false;
-      if (global_timer_ns() - t0 > kWaitLimitNs) {
+      const long long now = clock64();
+      if (t0 == 0) t0 = now;
+      if (now - t0 > kWaitLimitCycles) {
         ctl->abort = 1;
         atomicCAS(ctl->status, 0u, code);  // the first wait that expired names the culprit
         return false;
