@@ -227,7 +227,8 @@ int calidrop_compress(const calidrop_params* p, const void* Q_obs, const void* K
     e = tc_path ? launch_votes_tc(g, ws, Q_obs, K, row_lse, wsp, st) : launch_votes(g, ws, Q_obs, K, row_lse, wsp, st);
     if (e != cudaSuccess) return cuda_fail(e);
   }
-  e = launch_pool_select(g, ws, wsp, kept_idx, st);
+  e = (select_cluster_supported(g) && !scalar_path_forced()) ? launch_pool_select_cluster(g, ws, wsp, kept_idx, st)
+                                                             : launch_pool_select(g, ws, wsp, kept_idx, st);
   if (e != cudaSuccess) return cuda_fail(e);
   e = launch_gather(g, K, V, kept_idx, K_kept, V_kept, st);
   if (e != cudaSuccess) return cuda_fail(e);

@@ -1,0 +1,216 @@
+// Pooling + per-(batch, kv-head) top-k on a thread-block cluster.
+//
+// The single-CTA selection of select.cu uses one SM per unit; with a few dozen units most of the
+// GPU idles.  Here a cluster of eight CTAs shares a unit: CTA r owns the contiguous key range
+// [r * chunk, (r + 1) * chunk), every thread keeps its ROWS keys (pooled votes as fp32 bit
+// patterns) in registers, and the CTAs exchange only their 256-bin histograms and their counts
+// through distributed shared memory.  The algorithm is the same exact radix select: four 8-bit
+// passes find the bit pattern T of the k-th largest pooled vote and how many candidates equal to
+// T still fit; an ordered compaction then emits, ascending, every candidate above T and the first
+// need_eq candidates equal to T (ties go to the lowest index), plus the kept bitmap.
+// Key (row i, thread tid) of CTA r is candidate r * chunk + i * 1024 + tid, so a warp covers 32
+// consecutive candidates: loads coalesce and one ballot is one bitmap word.
+#include <cooperative_groups.h>
+
+#include "common.cuh"
+#include "internal.h"
+
+namespace calidrop {
+
+namespace {
+
+namespace cg = cooperative_groups;
+
+constexpr int kClu = 8;
+constexpr int kT = 1024;
+constexpr int kW = kT / 32;
+
+template <int ROWS>
+__global__ void __cluster_dims__(kClu, 1, 1) __launch_bounds__(kT)
+pool_select_cluster_kernel(const float* __restrict__ vote, float* __restrict__ pooled,
+                           uint32_t* __restrict__ bitmap, int32_t* __restrict__ kept_idx, int n_cand, int L,
+                           int pool, int k_sel, int n_kept, int bitmap_words) {
+  __shared__ unsigned hist[kW][256];
+  __shared__ unsigned mine[2][256];   // this CTA's histogram of the current pass (double-buffered)
+  __shared__ unsigned total[256];
+  __shared__ unsigned sel_bin, sel_k;
+  __shared__ unsigned cnt[2];         // this CTA's counts of keys > T and == T
+  __shared__ unsigned wsum[ROWS * kW][2];
+
+  cg::cluster_group cluster = cg::this_cluster();
+  const int rank = (int)cluster.block_rank();
+  const int unit = blockIdx.y;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int chunk = ROWS * kT;
+  const float* v = vote + (size_t)unit * n_cand;
+  float* pl = pooled + (size_t)unit * n_cand;
+  uint32_t* bm = bitmap + (size_t)unit * bitmap_words;
+  int32_t* kept = kept_idx + (size_t)unit * n_kept;
+
+  // 1. zero-padded average pool with a constant divisor; keys stay in registers
+  unsigned key[ROWS];
+  const int half = pool >> 1;
+  const float fpool = (float)pool;
+#pragma unroll
+  for (int i = 0; i < ROWS; ++i) {
+    const int t = rank * chunk + i * kT + tid;
+    key[i] = 0u;
+    if (t < n_cand) {
+      float acc = 0.f;
+      for (int d = -half; d <= half; ++d) {
+        const int u = t + d;
+        if (u >= 0 && u < n_cand) acc += v[u];
+      }
+      const float p = acc / fpool;
+      pl[t] = p;
+      key[i] = __float_as_uint(p);
+    }
+  }
+
+  // 2. radix select, most significant byte first; the histograms of the eight CTAs are summed
+  // through distributed shared memory
+  unsigned prefix = 0, k = (unsigned)k_sel;
+  for (int pass = 0; pass < 4; ++pass) {
+    const int shift = 24 - 8 * pass;
+    for (int i = tid; i < kW * 256; i += kT) (&hist[0][0])[i] = 0;
+    __syncthreads();
+#pragma unroll
+    for (int i = 0; i < ROWS; ++i) {
+      const int t = rank * chunk + i * kT + tid;
+      const bool in = t < n_cand && ((pass == 0) || ((key[i] >> (shift + 8)) == prefix));
+      if (in) atomicAdd(&hist[warp][(key[i] >> shift) & 255u], 1u);
+    }
+    __syncthreads();
+    if (tid < 256) {
+      unsigned s = 0;
+#pragma unroll 8
+      for (int w = 0; w < kW; ++w) s += hist[w][tid];
+      mine[pass & 1][tid] = s;
+    }
+    cluster.sync();
+    if (tid < 256) {
+      unsigned s = 0;
+      for (int r = 0; r < kClu; ++r) s += cluster.map_shared_rank(&mine[pass & 1][0], r)[tid];
+      total[tid] = s;
+    }
+    __syncthreads();
+    if (warp == 0) {
+      // lane 0 owns the 8 highest bins; walk bins downwards until k candidates are covered
+      const int base = 255 - 8 * lane;
+      unsigned c[8], s = 0;
+#pragma unroll
+      for (int j = 0; j < 8; ++j) { c[j] = total[base - j]; s += c[j]; }
+      unsigned incl = s;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        unsigned n = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += n;
+      }
+      const unsigned ball = __ballot_sync(0xffffffffu, incl >= k);
+      const int target = __ffs(ball) - 1;  // always found: the candidates number at least k
+      if (lane == target) {
+        unsigned run = incl - s;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+          if (run + c[j] >= k) { sel_bin = (unsigned)(base - j); sel_k = k - run; break; }
+          run += c[j];
+        }
+      }
+    }
+    __syncthreads();
+    prefix = (prefix << 8) | sel_bin;
+    k = sel_k;
+  }
+  const unsigned T = prefix;   // bit pattern of the k-th largest pooled vote
+  const unsigned need_eq = k;  // how many candidates equal to T are taken (lowest positions)
+
+  // 3. ordered compaction.  Per (row, warp): how many keys are above T / equal to T.
+  unsigned gt_mask[ROWS], eq_mask[ROWS];
+#pragma unroll
+  for (int i = 0; i < ROWS; ++i) {
+    const int t = rank * chunk + i * kT + tid;
+    const bool valid = t < n_cand;
+    gt_mask[i] = __ballot_sync(0xffffffffu, valid && key[i] > T);
+    eq_mask[i] = __ballot_sync(0xffffffffu, valid && key[i] == T);
+    if (lane == 0) {
+      wsum[i * kW + warp][0] = __popc(gt_mask[i]);
+      wsum[i * kW + warp][1] = __popc(eq_mask[i]);
+    }
+  }
+  __syncthreads();
+  // exclusive scan of the ROWS * 32 warp counts in index order (row-major), by the first warp
+  if (warp == 0) {
+    unsigned run_gt = 0, run_eq = 0;
+    for (int base = 0; base < ROWS * kW; base += 32) {
+      const unsigned g0 = wsum[base + lane][0], e0 = wsum[base + lane][1];
+      unsigned ig = g0, ie = e0;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const unsigned a = __shfl_up_sync(0xffffffffu, ig, o);
+        const unsigned b = __shfl_up_sync(0xffffffffu, ie, o);
+        if (lane >= o) { ig += a; ie += b; }
+      }
+      wsum[base + lane][0] = run_gt + ig - g0;
+      wsum[base + lane][1] = run_eq + ie - e0;
+      run_gt += __shfl_sync(0xffffffffu, ig, 31);
+      run_eq += __shfl_sync(0xffffffffu, ie, 31);
+    }
+    if (lane == 0) { cnt[0] = run_gt; cnt[1] = run_eq; }
+  }
+  cluster.sync();
+  unsigned before_gt = 0, before_eq = 0;  // keys of the lower-ranked CTAs
+  for (int r = 0; r < rank; ++r) {
+    const unsigned* c = cluster.map_shared_rank(&cnt[0], r);
+    before_gt += c[0];
+    before_eq += c[1];
+  }
+  const unsigned lt = (1u << lane) - 1u;
+#pragma unroll
+  for (int i = 0; i < ROWS; ++i) {
+    const int t = rank * chunk + i * kT + tid;
+    const unsigned gt_before = before_gt + wsum[i * kW + warp][0] + __popc(gt_mask[i] & lt);
+    const unsigned eq_before = before_eq + wsum[i * kW + warp][1] + __popc(eq_mask[i] & lt);
+    bool take = false;
+    if (t < n_cand) {
+      if (key[i] > T) take = true;
+      else if (key[i] == T) take = eq_before < need_eq;
+      if (take) kept[gt_before + min(eq_before, need_eq)] = t;
+    } else if (t < L) {
+      take = true;  // observation-window rows are always kept
+    }
+    const unsigned word = __ballot_sync(0xffffffffu, take);
+    const int t0 = rank * chunk + i * kT + warp * 32;
+    if (lane == 0 && t0 < L) bm[t0 >> 5] = word;
+  }
+  // the window rows close the kept list
+  if (rank == 0)
+    for (int j = tid; j < L - n_cand; j += kT) kept[k_sel + j] = n_cand + j;
+  cluster.sync();  // no CTA leaves while another may still read its shared memory
+}
+
+template <int ROWS>
+void launch_rows(const CompressGeom& g, const CompressWs& ws, char* wsp, int32_t* kept_idx, cudaStream_t st) {
+  pool_select_cluster_kernel<ROWS><<<dim3(kClu, g.units), kT, 0, st>>>(
+      (const float*)(wsp + ws.vote), (float*)(wsp + ws.pooled), (uint32_t*)(wsp + ws.bitmap), kept_idx, g.n_cand,
+      g.L, g.pool, g.k_sel, g.n_kept, g.bitmap_words);
+}
+
+}  // namespace
+
+// The cluster kernel keeps at most 32 keys per thread: 8 CTAs x 1024 threads x 32.
+bool select_cluster_supported(const CompressGeom& g) { return !g.keep_all && g.L <= kClu * kT * 32; }
+
+cudaError_t launch_pool_select_cluster(const CompressGeom& g, const CompressWs& ws, char* wsp, int32_t* kept_idx,
+                                       cudaStream_t st) {
+  const int rows = (g.L + kClu * kT - 1) / (kClu * kT);
+  if (rows <= 1) launch_rows<1>(g, ws, wsp, kept_idx, st);
+  else if (rows <= 2) launch_rows<2>(g, ws, wsp, kept_idx, st);
+  else if (rows <= 4) launch_rows<4>(g, ws, wsp, kept_idx, st);
+  else if (rows <= 8) launch_rows<8>(g, ws, wsp, kept_idx, st);
+  else if (rows <= 16) launch_rows<16>(g, ws, wsp, kept_idx, st);
+  else launch_rows<32>(g, ws, wsp, kept_idx, st);
+  count_launch(1);
+  return cudaGetLastError();
+}
+
+}  // namespace calidrop
