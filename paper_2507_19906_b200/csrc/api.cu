@@ -83,9 +83,9 @@ CompressWs make_ws(const CompressGeom& g) {
   w.status = off;    off = align_up(off + 4, 256);
   w.calib_o = w.calib_l = off;
   if (score_tc_supported(g) && calib_tc_supported(g)) {
-    int gpb, n_cblocks, n_splits;
-    calib_tc_plan(g, &gpb, &n_cblocks, &n_splits);
-    const size_t parts = (size_t)g.units * n_cblocks * n_splits;
+    int gpb, n_cblocks, tpc, max_slots;
+    size_t parts;
+    calib_tc_plan(g, &gpb, &n_cblocks, &tpc, &max_slots, &parts);
     w.calib_o = off; off = align_up(off + parts * 128 * kD * 4, 256);
     w.calib_l = off; off = align_up(off + parts * 2 * 128 * 4, 256);
   }

@@ -73,7 +73,8 @@ cudaError_t launch_row_stats_tc(const CompressGeom& g, const CompressWs& ws, con
 cudaError_t launch_votes_tc(const CompressGeom& g, const CompressWs& ws, const void* Q_obs, const void* K,
                             const float* row_lse, char* wsp, cudaStream_t st);
 bool calib_tc_supported(const CompressGeom& g);
-void calib_tc_plan(const CompressGeom& g, int* gpb, int* n_cblocks, int* n_splits);
+void calib_tc_plan(const CompressGeom& g, int* gpb, int* n_cblocks, int* tiles_per_cta, int* max_slots,
+                   size_t* parts);
 cudaError_t launch_calib_tc(const CompressGeom& g, const CompressWs& ws, const void* Q_obs, const void* K,
                             const void* V, const float* row_lse, char* wsp, float* O_c, float* LSE_c, void* C_q,
                             cudaStream_t st);
