@@ -178,7 +178,19 @@ def run_gpu(args):
             cd.calidrop_compress(p, Qd, Kd, Vd, None, st.kept_idx, st.K_kept, st.V_kept, st.O_c, st.LSE_c,
                                  st.C_q, st.ws_compress)
 
+    if args.batched_decode:
+        # one launch per decode step covering all layer states (calidrop_decode_batched)
+        ws_b = torch.zeros((cd.calidrop_decode_workspace_bytes(p, cap) * S,), dtype=torch.uint8, device="cuda")
+        layer_arrays = [cd.make_decode_layers([
+            dict(q=dq[t], k_new=dkn[t], v_new=dvn[t], K_kept=st.K_kept, V_kept=st.V_kept, O_c=st.O_c,
+                 LSE_c=st.LSE_c, C_q=st.C_q, out=outs[s], lse_out=lses[s], flags=flgs[s])
+            for s, st in enumerate(states)]) for t in range(T)]
+
     def decode_phase():
+        if args.batched_decode:
+            for t in range(T):
+                cd.calidrop_decode_batched(p, layer_arrays[t], cfg.budget + t, ws_b)
+            return
         for t in range(T):
             for s, st in enumerate(states):
                 cd.calidrop_decode(p, dq[t], dkn[t], dvn[t], st.K_kept, st.V_kept, cfg.budget + t, st.O_c,
@@ -236,7 +248,7 @@ def run_gpu(args):
     t_comp, t_dec, t_tot = (float(x) for x in times.cpu())
 
     dec_bytes_step = sum(decode_bytes(cfg, n_cal, cfg.budget + t + 1) for t in range(T)) * S
-    dec_launches = T * S * args.steps
+    dec_launches = T * (1 if args.batched_decode else S) * args.steps
     dec_gbs = dec_bytes_step * args.steps / (t_dec * 1e-3) / 1e9
     comp_ms_layer = t_comp / (args.steps * S)
     comp_tflops = compress_flops(cfg, n_cal) / (comp_ms_layer * 1e-3) / 1e12
@@ -298,7 +310,7 @@ def run_gpu(args):
         cpu = time_oracle(sample_inputs, n_cal, T, q_bits, kn_bits, vn_bits, args.cpu_units)
 
     avg_launch_s = t_dec * 1e-3 / dec_launches
-    bytes_per_launch = dec_bytes_step / (T * S)
+    bytes_per_launch = dec_bytes_step / (T * (1 if args.batched_decode else S))
     result = {
         "metric": METRIC, "value": dec_gbs * world, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": t_tot / args.steps, "higher_is_better": True,
@@ -311,6 +323,8 @@ def run_gpu(args):
                          f"visited round-robin, prompts of {2 * cfg.B * cfg.Hkv * cfg.L * cfg.D * 2 / 1e6:.0f} MB",
                    "lse_obs": "not supplied (row statistics recomputed inside the step)",
                    "launch": "eager C-ABI calls" if args.no_graph else "CUDA-graph replay of the captured C-ABI calls",
+                   "decode_entry": "calidrop_decode_batched over the layer states" if args.batched_decode
+                   else "calidrop_decode per layer state",
                    "parallelism": "replicas only" if world > 1 else "single GPU"},
         "decode": {"us_per_launch": avg_launch_s * 1e6, "gbs": dec_gbs, "launches": dec_launches,
                    "bytes_per_launch": bytes_per_launch,
@@ -438,6 +452,8 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=1)
     ap.add_argument("--cpu-units", type=int, default=4)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--batched-decode", action="store_true",
+                    help="one calidrop_decode_batched launch per decode step over all layer states")
     ap.add_argument("--no-graph", action="store_true", help="launch every call eagerly instead of replaying CUDA graphs")
     args = ap.parse_args()
     if args.impl == "reference":

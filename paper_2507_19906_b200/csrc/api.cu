@@ -276,10 +276,11 @@ int calidrop_decode_batched(const calidrop_params* p, int32_t n_layers, const ca
   a.B = p->B; a.Hq = p->Hq; a.Hkv = p->Hkv; a.G = p->Hq / p->Hkv; a.n_cal = p->n_cal; a.cap = p->cap;
   a.kv_len = kv_len; a.n_kv = n_kv; a.has_new = has_new ? 1 : 0;
   a.units = p->B * p->Hkv; a.n_layers = n_layers;
-  a.nsplit = decode_nsplit(a.units * n_layers, n_kv);
-  if (a.nsplit > w.max_split) a.nsplit = w.max_split;
+  // the splits of a unit form one thread-block cluster: 1, 2, 4 or 8 CTAs
+  int want = decode_nsplit(a.units * n_layers, n_kv);
+  a.nsplit = 1;
+  while (a.nsplit * 2 <= want && a.nsplit < 8) a.nsplit *= 2;
   a.rows_per_split = (n_kv + a.nsplit - 1) / a.nsplit;
-  a.nsplit = (n_kv + a.rows_per_split - 1) / a.rows_per_split;
   a.scale2 = scale2_of(p);
   a.theta1 = p->theta1; a.theta2 = p->theta2; a.always_apply = p->theta2 <= -1.0f;
   // The workspace is laid out array by array with the layer index outermost inside each

@@ -7,22 +7,31 @@
 // HBM traffic (about 2G flop per byte), so the contraction uses the warp-level mma.sync path
 // with G <= 8 rows of a 16-row tile; tcgen05 tiles (64 rows minimum) would add nothing here.
 //
-// Grid: (split, batch*kv-head, layer).  Each CTA streams its slice of rows through
-// shared memory with 16-byte cp.async copies (XOR-swizzled so ldmatrix is conflict-free),
-// four warps each running an independent online softmax over interleaved 16-row blocks.
-// Per-split partial results go to the workspace; the CTA that arrives last at a per-unit
-// ticket counter combines them and applies gate and merge.  No CTA ever waits on another.
+// Grid: (split, batch*kv-head, layer); the splits of one (unit, layer) form a thread-block
+// cluster of 1, 2, 4 or 8 CTAs.  Each CTA streams its slice of rows through shared memory with
+// 16-byte cp.async copies (XOR-swizzled so ldmatrix is conflict-free), four warps each running
+// an independent online softmax over interleaved 16-row blocks.  The splits are combined inside
+// the cluster through distributed shared memory: every CTA finishes a slice of the 128 output
+// dimensions for all heads of the group, so there is no global-memory round trip, no ticket and
+// no CTA that works alone at the end.
 //
-// The kernel is latency-sensitive (tens of MB per launch), so dependent global round trips
-// are kept to a minimum: the small loads (query, calibration queries) are issued before the
-// K/V burst so they are not queued behind it, and the finishing CTA fetches everything it
-// needs in two waves (partials + statistics + similarities, then the chosen calibration row).
+// A launch moves only tens of MB, so its latency chain matters as much as its bandwidth:
+//   * the launch carries the programmatic-serialisation attribute and the kernel prefetches its
+//     K/V slice into L2 before the dependency wait, so the HBM reads of one decode call overlap
+//     the tail of whatever runs ahead of it in the stream;
+//   * the K/V copies are issued first, the similarity work (which needs only q and C_q) runs while
+//     they are in flight, and the cluster exchanges each CTA's best (similarity, row) pair early,
+//     so the chosen O_c row is already being fetched while the partial outputs are combined.
+#include <cooperative_groups.h>
+
 #include "common.cuh"
 #include "internal.h"
 
 namespace calidrop {
 
 namespace {
+
+namespace cg = cooperative_groups;
 
 constexpr int kWarps = 4;
 constexpr int kThreads = kWarps * 32;
@@ -31,8 +40,6 @@ constexpr int kStages = 3;
 constexpr int kStageBytes = 2 * kBlkRows * kRowBytes;  // K block then V block
 constexpr int kWarpSmem = kStages * kStageBytes;       // 24 KB
 constexpr int kSmemBytes = kWarps * kWarpSmem;         // 96 KB -> two CTAs per SM
-constexpr int kRhoRegPasses = 2;                       // similarity passes whose loads are issued up front
-constexpr int kPairsPerPass = kThreads / 8;            // 8 lanes per (head, calibration row) pair
 
 __device__ __forceinline__ uint32_t swz(int row, int chunk) {
   return (uint32_t)(row * kRowBytes + ((chunk ^ (row & 7)) << 4));
@@ -55,19 +62,37 @@ __device__ __forceinline__ void rho_accumulate(const RhoLoad& r, float& dot, flo
   }
 }
 
+// Order-preserving map of a float onto unsigned integers; with the row index in the low word,
+// one 64-bit max picks the highest similarity and, among equals, the largest row index.
+__device__ __forceinline__ unsigned long long rank_key(float rho, int c) {
+  unsigned u = __float_as_uint(rho);
+  u = (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+  return ((unsigned long long)u << 32) | (unsigned)c;
+}
+__device__ __forceinline__ float rank_key_value(unsigned long long k) {
+  unsigned u = (unsigned)(k >> 32);
+  u = (u & 0x80000000u) ? (u & 0x7fffffffu) : ~u;
+  return __uint_as_float(u);
+}
+
+__device__ __forceinline__ void cluster_arrive() {
+  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void cluster_wait() {
+  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+
 __global__ void __launch_bounds__(kThreads, 2) decode_kernel(const __grid_constant__ DecodeArgs a) {
   extern __shared__ __align__(128) unsigned char smem[];
-  __shared__ int s_ticket;
-  __shared__ int s_cstar[kMaxG];
-  __shared__ float s_rho[kMaxG];
+  __shared__ unsigned long long s_best[kMaxG];  // best (similarity, row) of this CTA's calibration rows
 
-  const int split = blockIdx.x, unit = blockIdx.y, layer = blockIdx.z;
+  cg::cluster_group cluster = cg::this_cluster();
+  const int split = blockIdx.x, unit = blockIdx.y, layer = blockIdx.z;  // cluster rank == split
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int gq = lane >> 2, tq = lane & 3;  // MMA fragment coordinates
   const DecodeLayerPtrs& P = a.layer[layer];
   const int b = unit / a.Hkv, h = unit % a.Hkv;
   const int hq0 = b * a.Hq + h * a.G;  // first query head of this kv group
-  const size_t lu = (size_t)layer * a.units + unit;
 
   const __nv_bfloat16* q = (const __nv_bfloat16*)P.q;
   const __nv_bfloat16* Cq = (const __nv_bfloat16*)P.C_q;
@@ -84,50 +109,26 @@ __global__ void __launch_bounds__(kThreads, 2) decode_kernel(const __grid_consta
   unsigned char* wsm = smem + warp * kWarpSmem;
   const uint32_t wsm_u32 = smem_u32(wsm);
 
-  // ---- (1) small loads first: query fragments (rows 0..G-1 of a 16-row A tile, the rest
-  // zero) and the calibration queries this CTA compares against (c = split, split+nsplit, ...)
-  uint32_t qa[kD / 16][2];
-#pragma unroll
-  for (int kk = 0; kk < kD / 16; ++kk) {
-    qa[kk][0] = 0u; qa[kk][1] = 0u;
-    if (gq < a.G) {
-      const uint32_t* qr = reinterpret_cast<const uint32_t*>(q + (size_t)(hq0 + gq) * kD + kk * 16);
-      qa[kk][0] = __ldg(qr + tq);
-      qa[kk][1] = __ldg(qr + 4 + tq);
+  // ---- (0) overlap with the kernel ahead of this one in the stream.  Until the dependency wait
+  // nothing the predecessor may have written is read and nothing is written; the only early work
+  // is an L2 prefetch of this CTA's slice of the retained cache, which cannot observe stale data
+  // (L2 is the point of coherence) and turns the later cp.async stream into L2 hits.
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  if (tid == 0) {
+    const int n_old = min(r1, a.kv_len) - r0;  // rows already in the cache (the appended row is not)
+    if (n_old > 0) {
+      const unsigned bytes = (unsigned)n_old * kRowBytes;
+      asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(Kc + (size_t)r0 * kRowBytes), "r"(bytes)
+                   : "memory");
+      asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(Vc + (size_t)r0 * kRowBytes), "r"(bytes)
+                   : "memory");
     }
   }
-  const int n_c = a.n_cal > split ? (a.n_cal - split + a.nsplit - 1) / a.nsplit : 0;
-  const int pairs = n_c * a.G;
-  const int sub = tid & 7;
-  auto rho_load = [&](int pi, RhoLoad& r) {
-    const int g = pi % a.G, c = split + (pi / a.G) * a.nsplit;
-    const uint4* qp = reinterpret_cast<const uint4*>(q + (size_t)(hq0 + g) * kD + sub * 16);
-    const uint4* cp = reinterpret_cast<const uint4*>(Cq + ((size_t)(hq0 + g) * a.n_cal + c) * kD + sub * 16);
-    r.q0 = __ldg(qp); r.q1 = __ldg(qp + 1); r.c0 = __ldg(cp); r.c1 = __ldg(cp + 1);
-  };
-  auto rho_finish = [&](int pi, const RhoLoad& r) {
-    float dot = 0.f, qq = 0.f, cc = 0.f;
-    if (pi < pairs) rho_accumulate(r, dot, qq, cc);
-#pragma unroll
-    for (int o = 1; o < 8; o <<= 1) {
-      dot += __shfl_xor_sync(0xffffffffu, dot, o);
-      qq += __shfl_xor_sync(0xffffffffu, qq, o);
-      cc += __shfl_xor_sync(0xffffffffu, cc, o);
-    }
-    if (sub == 0 && pi < pairs) {
-      const int g = pi % a.G, c = split + (pi / a.G) * a.nsplit;
-      a.rho[(lu * kMaxG + g) * a.n_cal + c] = (qq > 0.f && cc > 0.f) ? dot / (sqrtf(qq) * sqrtf(cc)) : 0.f;
-    }
-  };
-  RhoLoad rl[kRhoRegPasses];
-#pragma unroll
-  for (int ps = 0; ps < kRhoRegPasses; ++ps) {
-    rl[ps] = RhoLoad{};
-    const int pi = ps * kPairsPerPass + (tid >> 3);
-    if (pi < pairs) rho_load(pi, rl[ps]);
-  }
+  if (tid < kMaxG) s_best[tid] = 0ull;
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  __syncthreads();
 
-  // ---- (2) the K/V stream: issue one 16-row block (K and V) of this warp into a stage
+  // ---- (1) the K/V stream first: issue one 16-row block (K and V) of this warp into a stage
   auto issue = [&](int i, int stage) {
     const int row_base = r0 + (warp + i * kWarps) * kBlkRows;
     const uint32_t dstK = wsm_u32 + stage * kStageBytes;
@@ -151,6 +152,18 @@ __global__ void __launch_bounds__(kThreads, 2) decode_kernel(const __grid_consta
     cp_async_commit();
   }
 
+  // ---- (2) query fragments (rows 0..G-1 of a 16-row A tile, the rest zero)
+  uint32_t qa[kD / 16][2];
+#pragma unroll
+  for (int kk = 0; kk < kD / 16; ++kk) {
+    qa[kk][0] = 0u; qa[kk][1] = 0u;
+    if (gq < a.G) {
+      const uint32_t* qr = reinterpret_cast<const uint32_t*>(q + (size_t)(hq0 + gq) * kD + kk * 16);
+      qa[kk][0] = __ldg(qr + tq);
+      qa[kk][1] = __ldg(qr + 4 + tq);
+    }
+  }
+
   // ---- (3) append: the CTA whose slice holds row kv_len stores the new K/V row into the cache
   if (a.has_new && a.kv_len >= r0 && a.kv_len < r1 && warp == 0) {
     const int chunk = lane & 15;
@@ -160,15 +173,46 @@ __global__ void __launch_bounds__(kThreads, 2) decode_kernel(const __grid_consta
     *reinterpret_cast<uint4*>(dst) = *reinterpret_cast<const uint4*>(src);
   }
 
-  // ---- (4) cosine similarities (their loads are long in flight by now)
+  // ---- (4) cosine similarities of this CTA's calibration rows (c = split, split + nsplit, ...),
+  // eight lanes per (head, row) pair; the best pair per head goes to s_best
+  {
+    const int n_c = a.n_cal > split ? (a.n_cal - split + a.nsplit - 1) / a.nsplit : 0;
+    const int pairs = n_c * a.G;
+    const int sub = tid & 7;
+    constexpr int kPairsPerPass = kThreads / 8;
+    for (int base = 0; base < pairs; base += 2 * kPairsPerPass) {
+      RhoLoad rl[2];
 #pragma unroll
-  for (int ps = 0; ps < kRhoRegPasses; ++ps) rho_finish(ps * kPairsPerPass + (tid >> 3), rl[ps]);
-  for (int base = kRhoRegPasses * kPairsPerPass; base < pairs; base += kPairsPerPass) {
-    const int pi = base + (tid >> 3);
-    RhoLoad r{};
-    if (pi < pairs) rho_load(pi, r);
-    rho_finish(pi, r);
+      for (int u = 0; u < 2; ++u) {
+        const int pi = base + u * kPairsPerPass + (tid >> 3);
+        rl[u] = RhoLoad{};
+        if (pi < pairs) {
+          const int g = pi % a.G, c = split + (pi / a.G) * a.nsplit;
+          const uint4* qp = reinterpret_cast<const uint4*>(q + (size_t)(hq0 + g) * kD + sub * 16);
+          const uint4* cp = reinterpret_cast<const uint4*>(Cq + ((size_t)(hq0 + g) * a.n_cal + c) * kD + sub * 16);
+          rl[u].q0 = __ldg(qp); rl[u].q1 = __ldg(qp + 1); rl[u].c0 = __ldg(cp); rl[u].c1 = __ldg(cp + 1);
+        }
+      }
+#pragma unroll
+      for (int u = 0; u < 2; ++u) {
+        const int pi = base + u * kPairsPerPass + (tid >> 3);
+        float dot = 0.f, qq = 0.f, cc = 0.f;
+        if (pi < pairs) rho_accumulate(rl[u], dot, qq, cc);
+#pragma unroll
+        for (int o = 1; o < 8; o <<= 1) {
+          dot += __shfl_xor_sync(0xffffffffu, dot, o);
+          qq += __shfl_xor_sync(0xffffffffu, qq, o);
+          cc += __shfl_xor_sync(0xffffffffu, cc, o);
+        }
+        if (sub == 0 && pi < pairs) {
+          const int g = pi % a.G, c = split + (pi / a.G) * a.nsplit;
+          const float rho = (qq > 0.f && cc > 0.f) ? dot / (sqrtf(qq) * sqrtf(cc)) : 0.f;
+          atomicMax(&s_best[g], rank_key(rho, c));
+        }
+      }
+    }
   }
+  cluster_arrive();  // (A) this CTA's s_best is final
 
   // ---- (5) main loop
   float o[kD / 8][4];
@@ -235,110 +279,73 @@ __global__ void __launch_bounds__(kThreads, 2) decode_kernel(const __grid_consta
   l += __shfl_xor_sync(0xffffffffu, l, 2);
   __syncthreads();  // all warps are done with their stages: reuse them for the combine
 
-  // ---- (6) CTA combine of the four warps
-  float* wo = reinterpret_cast<float*>(smem);   // [warp][8][128]
-  float* wml = wo + kWarps * kMaxG * kD;         // [warp][8][2]
+  // ---- (6) CTA combine of the four warps into this split's partial: xo[g][d], xml[g] = (m, l)
+  float* wo = reinterpret_cast<float*>(smem);             // [warp][8][128]
+  float* wml = wo + kWarps * kMaxG * kD;                   // [warp][8][2]
+  float* xo = wml + kWarps * kMaxG * 2;                    // [8][128]
+  float* xml = xo + kMaxG * kD;                            // [8][2]
 #pragma unroll
   for (int n = 0; n < kD / 8; ++n)
     *reinterpret_cast<float2*>(wo + ((warp * kMaxG + gq) * kD + n * 8 + 2 * tq)) = make_float2(o[n][0], o[n][1]);
   if (tq == 0) { wml[(warp * kMaxG + gq) * 2] = m; wml[(warp * kMaxG + gq) * 2 + 1] = l; }
   __syncthreads();
-  const int d = tid;  // one output dimension per thread
-  float* part_o = a.part_o + ((lu * a.nsplit + split) * kMaxG) * kD;
-  float* part_ml = a.part_ml + ((lu * a.nsplit + split) * kMaxG) * 2;
-  for (int g = 0; g < a.G; ++g) {
-    float M = -INFINITY;
+  {
+    const int d = tid;  // one output dimension per thread
+    for (int g = 0; g < a.G; ++g) {
+      float M = -INFINITY;
 #pragma unroll
-    for (int w = 0; w < kWarps; ++w) M = fmaxf(M, wml[(w * kMaxG + g) * 2]);
-    float Lsum = 0.f, acc = 0.f;
+      for (int w = 0; w < kWarps; ++w) M = fmaxf(M, wml[(w * kMaxG + g) * 2]);
+      float Lsum = 0.f, acc = 0.f;
 #pragma unroll
-    for (int w = 0; w < kWarps; ++w) {
-      const float mw = wml[(w * kMaxG + g) * 2];
-      const float sc = mw > -INFINITY ? ex2_approx(mw - M) : 0.f;
-      Lsum += wml[(w * kMaxG + g) * 2 + 1] * sc;
-      acc += wo[(w * kMaxG + g) * kD + d] * sc;
-    }
-    __stcg(part_o + g * kD + d, acc);
-    if (d == 0) { __stcg(part_ml + g * 2, M); __stcg(part_ml + g * 2 + 1, Lsum); }
-  }
-
-  // ---- (7) ticket: the CTA that arrives last for this (layer, unit) finishes the job.
-  // The barrier orders every thread's stores before thread 0's device-scope fence (fences
-  // are cumulative), which in turn precedes the ticket increment.
-  __syncthreads();
-  if (tid == 0) {
-    __threadfence();
-    s_ticket = (int)atomicAdd(a.counters + lu, 1u);
-  }
-  __syncthreads();
-  if (s_ticket != a.nsplit - 1) return;
-  __threadfence();
-
-  // ---- (8) finish: wave one fetches the split statistics, the similarities and the first
-  // chunk of partial outputs together; wave two the chosen calibration row.
-  const float* po = a.part_o + (lu * a.nsplit) * kMaxG * kD;
-  const float* pml = a.part_ml + (lu * a.nsplit) * kMaxG * 2;
-  float* ml_s = wml + kWarps * kMaxG * 2;  // [split][8][2]
-  const int n_items = a.G * (kD / 4);      // (head, 4 consecutive dims) items, one per thread
-  constexpr int kChunk = 8;
-  float4 pv[kChunk];
-  auto load_chunk = [&](int item, int s0) {
-    const int g = item >> 5, d4 = item & 31;
-#pragma unroll
-    for (int s = 0; s < kChunk; ++s) {
-      pv[s] = make_float4(0.f, 0.f, 0.f, 0.f);
-      if (s0 + s < a.nsplit)
-        pv[s] = __ldcg(reinterpret_cast<const float4*>(po + ((s0 + s) * kMaxG + g) * kD) + d4);
-    }
-  };
-  if (tid < n_items) load_chunk(tid, 0);
-  for (int i = tid; i < a.nsplit * kMaxG * 2; i += kThreads) ml_s[i] = __ldcg(pml + i);
-  // choice of the calibration row: highest cosine similarity, ties to the largest c
-  for (int g = warp; g < a.G; g += kWarps) {
-    float best = -INFINITY;
-    int bc = 0;
-    for (int c = lane; c < a.n_cal; c += 32) {
-      const float r = __ldcg(a.rho + (lu * kMaxG + g) * a.n_cal + c);
-      if (r >= best) { best = r; bc = c; }
-    }
-#pragma unroll
-    for (int off = 16; off > 0; off >>= 1) {
-      const float ob = __shfl_xor_sync(0xffffffffu, best, off);
-      const int oc = __shfl_xor_sync(0xffffffffu, bc, off);
-      if (ob > best || (ob == best && oc > bc)) { best = ob; bc = oc; }
-    }
-    if (lane == 0) { s_cstar[g] = bc; s_rho[g] = best; }
-  }
-  __syncthreads();
-
-  for (int item = tid; item < n_items; item += kThreads) {
-    const int g = item >> 5, d4 = item & 31;
-    const int hq = hq0 + g;
-    const int cs = s_cstar[g];
-    const float rho = s_rho[g];
-    const size_t crow = (size_t)hq * a.n_cal + cs;
-    const float lse_c = __ldg(P.LSE_c + crow);
-    const float4 oc = __ldg(reinterpret_cast<const float4*>(P.O_c + crow * kD) + d4);
-    float M = -INFINITY;
-    for (int s = 0; s < a.nsplit; ++s) M = fmaxf(M, ml_s[(s * kMaxG + g) * 2]);
-    float Lsum = 0.f;
-    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-    for (int s0 = 0; s0 < a.nsplit; s0 += kChunk) {
-      if (s0 > 0 || item != tid) load_chunk(item, s0);
-#pragma unroll
-      for (int s = 0; s < kChunk; ++s) {
-        if (s0 + s < a.nsplit) {
-          const float ms = ml_s[((s0 + s) * kMaxG + g) * 2];
-          const float sc = ms > -INFINITY ? ex2_approx(ms - M) : 0.f;
-          Lsum = fmaf(ml_s[((s0 + s) * kMaxG + g) * 2 + 1], sc, Lsum);
-          acc.x = fmaf(pv[s].x, sc, acc.x); acc.y = fmaf(pv[s].y, sc, acc.y);
-          acc.z = fmaf(pv[s].z, sc, acc.z); acc.w = fmaf(pv[s].w, sc, acc.w);
-        }
+      for (int w = 0; w < kWarps; ++w) {
+        const float mw = wml[(w * kMaxG + g) * 2];
+        const float sc = mw > -INFINITY ? ex2_approx(mw - M) : 0.f;
+        Lsum += wml[(w * kMaxG + g) * 2 + 1] * sc;
+        acc += wo[(w * kMaxG + g) * kD + d] * sc;
       }
+      xo[g * kD + d] = acc;
+      if (d == 0) { xml[g * 2] = M; xml[g * 2 + 1] = Lsum; }
     }
-    const float inv = 1.f / Lsum;
-    float4 outv = make_float4(acc.x * inv, acc.y * inv, acc.z * inv, acc.w * inv);  // O_a
-    float lse2 = M + log2f(Lsum);                                                   // LSE_a (log2 domain)
+  }
+  cluster_wait();    // (A) every CTA's s_best can be read
+  cluster_arrive();  // (B) this CTA's partial (xo, xml) is final
+
+  // ---- (7) finish.  This CTA owns 128 / nsplit output dimensions of every head of the group.
+  const int dpc = kD / a.nsplit;
+  const int n_items = a.G * dpc;
+  // Two items per thread at most would need nsplit >= G / ... ; in general loop over the items.
+  for (int item0 = 0; item0 < n_items; item0 += kThreads) {
+    const int item = item0 + tid;
+    const bool act = item < n_items;
+    const int g = act ? item / dpc : 0, d = split * dpc + (act ? item % dpc : 0);
+    const int hq = hq0 + g;
+    // the calibration row: best similarity over all CTAs, ties to the largest row index
+    unsigned long long best = 0ull;
+    for (int s = 0; s < a.nsplit; ++s) {
+      const unsigned long long k = *cluster.map_shared_rank(&s_best[g], s);
+      best = k > best ? k : best;
+    }
+    const int cs = (int)(unsigned)(best & 0xffffffffull);
+    const float rho = rank_key_value(best);
+    const size_t crow = (size_t)hq * a.n_cal + cs;
+    float lse_c = 0.f, oc = 0.f;
+    if (act) {  // in flight while the partials are exchanged
+      lse_c = __ldg(P.LSE_c + crow);
+      oc = __ldg(P.O_c + crow * kD + d);
+    }
+    if (item0 == 0) cluster_wait();  // (B) every CTA's partial can be read
+    float M = -INFINITY;
+    for (int s = 0; s < a.nsplit; ++s) M = fmaxf(M, cluster.map_shared_rank(xml, s)[g * 2]);
+    float Lsum = 0.f, acc = 0.f;
+    for (int s = 0; s < a.nsplit; ++s) {
+      const float* rml = cluster.map_shared_rank(xml, s);
+      const float ms = rml[g * 2];
+      const float sc = ms > -INFINITY ? ex2_approx(ms - M) : 0.f;
+      Lsum = fmaf(rml[g * 2 + 1], sc, Lsum);
+      acc = fmaf(cluster.map_shared_rank(xo, s)[g * kD + d], sc, acc);
+    }
+    float outv = acc / Lsum;             // O_a
+    float lse2 = M + log2f(Lsum);        // LSE_a (log2 domain)
     const bool apply = (a.always_apply || rho > a.theta2) && (lse_c > -INFINITY);
     if (apply) {
       // alpha_i = e^{LSE_a - LSE}, alpha_j = e^{LSE_c - LSE}; out = alpha_i O_a + alpha_j O_c (Eq. 1-2)
@@ -346,20 +353,20 @@ __global__ void __launch_bounds__(kThreads, 2) decode_kernel(const __grid_consta
       const float mx = fmaxf(lse2, lc2);
       const float ea = exp2f(lse2 - mx), ec = exp2f(lc2 - mx);
       const float tot = ea + ec;
-      const float ai = ea / tot, aj = ec / tot;
-      outv = make_float4(ai * outv.x + aj * oc.x, ai * outv.y + aj * oc.y, ai * outv.z + aj * oc.z,
-                         ai * outv.w + aj * oc.w);
+      outv = (ea / tot) * outv + (ec / tot) * oc;
       lse2 = mx + log2f(tot);
     }
-    uint2 packed = make_uint2(pack_bf16(outv.x, outv.y), pack_bf16(outv.z, outv.w));
-    reinterpret_cast<uint2*>(reinterpret_cast<__nv_bfloat16*>(P.out) + (size_t)hq * kD)[d4] = packed;
-    if (d4 == 0) {
-      if (P.lse_out) P.lse_out[hq] = lse2 * kLn2;
-      if (P.flags)
-        P.flags[hq] = (uint8_t)((apply ? 1 : 0) | (rho < a.theta1 ? 2 : 0) | (a.n_cal <= 64 ? (cs << 2) : 0));
+    if (act) {
+      reinterpret_cast<__nv_bfloat16*>(P.out)[(size_t)hq * kD + d] = __float2bfloat16_rn(outv);
+      if (d == 0) {
+        if (P.lse_out) P.lse_out[hq] = lse2 * kLn2;
+        if (P.flags)
+          P.flags[hq] = (uint8_t)((apply ? 1 : 0) | (rho < a.theta1 ? 2 : 0) | (a.n_cal <= 64 ? (cs << 2) : 0));
+      }
     }
   }
-  if (tid == 0) a.counters[lu] = 0u;  // ready for the next call
+  cluster_arrive();  // (C) no CTA leaves while another may still read its shared memory
+  cluster_wait();
 }
 
 }  // namespace
@@ -374,8 +381,22 @@ cudaError_t launch_decode(const DecodeArgs& a, cudaStream_t st) {
     if (e != cudaSuccess) return e;
     if (dev >= 0 && dev < 64) attr_set[dev] = true;
   }
-  dim3 grid(a.nsplit, a.units, a.n_layers);
-  decode_kernel<<<grid, kThreads, kSmemBytes, st>>>(a);
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = dim3(a.nsplit, a.units, a.n_layers);
+  cfg.blockDim = dim3(kThreads);
+  cfg.dynamicSmemBytes = kSmemBytes;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[2];
+  attr[0].id = cudaLaunchAttributeClusterDimension;  // the splits of a unit are one cluster
+  attr[0].val.clusterDim.x = a.nsplit;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[1].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 2;
+  e = cudaLaunchKernelEx(&cfg, decode_kernel, a);
+  if (e != cudaSuccess) return e;
   count_launch(1);
   return cudaGetLastError();
 }
