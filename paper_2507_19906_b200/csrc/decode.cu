@@ -124,11 +124,60 @@ __global__ void __launch_bounds__(kThreads, 2) decode_kernel(const __grid_consta
                    : "memory");
     }
   }
+  // calibration rows of this CTA: the contiguous range [c_begin, c_begin + n_c)
+  const int c_per = (a.n_cal + a.nsplit - 1) / a.nsplit;
+  const int c_begin = min(a.n_cal, split * c_per);
+  const int n_c = min(a.n_cal, c_begin + c_per) - c_begin;
+  if (tid >= 32 && tid < 32 + a.G && n_c > 0) {  // same for the small operands of the similarity
+    const int g = tid - 32;
+    asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(Cq + ((size_t)(hq0 + g) * a.n_cal + c_begin) * kD),
+                 "r"((unsigned)n_c * kRowBytes)
+                 : "memory");
+    if (g == 0)
+      asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(q + (size_t)hq0 * kD),
+                   "r"((unsigned)a.G * kRowBytes)
+                   : "memory");
+  }
   if (tid < kMaxG) s_best[tid] = 0ull;
   asm volatile("griddepcontrol.wait;" ::: "memory");
   __syncthreads();
 
-  // ---- (1) the K/V stream first: issue one 16-row block (K and V) of this warp into a stage
+  // ---- (1) loads of the similarity operands go out ahead of the K/V burst so that they are not
+  // queued behind it: four lanes per (head, calibration row) pair, 32 pairs per pass, the first
+  // two passes in flight at once
+  constexpr int kPairsPerPass = kThreads / 4;
+  const int pairs = n_c * a.G;
+  const int sub = tid & 3;
+  auto rho_load = [&](int pi, RhoLoad (&r)[2]) {
+    r[0] = RhoLoad{}; r[1] = RhoLoad{};
+    if (pi < pairs) {
+      const int g = pi % a.G, c = c_begin + pi / a.G;
+      const uint4* qp = reinterpret_cast<const uint4*>(q + (size_t)(hq0 + g) * kD + sub * 32);
+      const uint4* cp = reinterpret_cast<const uint4*>(Cq + ((size_t)(hq0 + g) * a.n_cal + c) * kD + sub * 32);
+      r[0].q0 = __ldg(qp); r[0].q1 = __ldg(qp + 1); r[0].c0 = __ldg(cp); r[0].c1 = __ldg(cp + 1);
+      r[1].q0 = __ldg(qp + 2); r[1].q1 = __ldg(qp + 3); r[1].c0 = __ldg(cp + 2); r[1].c1 = __ldg(cp + 3);
+    }
+  };
+  auto rho_finish = [&](int pi, const RhoLoad (&r)[2]) {
+    float dot = 0.f, qq = 0.f, cc = 0.f;
+    if (pi < pairs) { rho_accumulate(r[0], dot, qq, cc); rho_accumulate(r[1], dot, qq, cc); }
+#pragma unroll
+    for (int o = 1; o < 4; o <<= 1) {
+      dot += __shfl_xor_sync(0xffffffffu, dot, o);
+      qq += __shfl_xor_sync(0xffffffffu, qq, o);
+      cc += __shfl_xor_sync(0xffffffffu, cc, o);
+    }
+    if (sub == 0 && pi < pairs) {
+      const int g = pi % a.G, c = c_begin + pi / a.G;
+      const float rho = (qq > 0.f && cc > 0.f) ? dot / (sqrtf(qq) * sqrtf(cc)) : 0.f;
+      atomicMax(&s_best[g], rank_key(rho, c));
+    }
+  };
+  RhoLoad rl0[2], rl1[2];
+  rho_load(tid >> 2, rl0);
+  rho_load(kPairsPerPass + (tid >> 2), rl1);
+
+  // ---- (2) the K/V stream: issue one 16-row block (K and V) of this warp into a stage
   auto issue = [&](int i, int stage) {
     const int row_base = r0 + (warp + i * kWarps) * kBlkRows;
     const uint32_t dstK = wsm_u32 + stage * kStageBytes;
@@ -152,7 +201,7 @@ __global__ void __launch_bounds__(kThreads, 2) decode_kernel(const __grid_consta
     cp_async_commit();
   }
 
-  // ---- (2) query fragments (rows 0..G-1 of a 16-row A tile, the rest zero)
+  // ---- (3) query fragments (rows 0..G-1 of a 16-row A tile, the rest zero)
   uint32_t qa[kD / 16][2];
 #pragma unroll
   for (int kk = 0; kk < kD / 16; ++kk) {
@@ -164,7 +213,7 @@ __global__ void __launch_bounds__(kThreads, 2) decode_kernel(const __grid_consta
     }
   }
 
-  // ---- (3) append: the CTA whose slice holds row kv_len stores the new K/V row into the cache
+  // ---- (3b) append: the CTA whose slice holds row kv_len stores the new K/V row into the cache
   if (a.has_new && a.kv_len >= r0 && a.kv_len < r1 && warp == 0) {
     const int chunk = lane & 15;
     const unsigned char* src = (lane < 16 ? k_new : v_new) + chunk * 16;
@@ -173,44 +222,13 @@ __global__ void __launch_bounds__(kThreads, 2) decode_kernel(const __grid_consta
     *reinterpret_cast<uint4*>(dst) = *reinterpret_cast<const uint4*>(src);
   }
 
-  // ---- (4) cosine similarities of this CTA's calibration rows (c = split, split + nsplit, ...),
-  // eight lanes per (head, row) pair; the best pair per head goes to s_best
-  {
-    const int n_c = a.n_cal > split ? (a.n_cal - split + a.nsplit - 1) / a.nsplit : 0;
-    const int pairs = n_c * a.G;
-    const int sub = tid & 7;
-    constexpr int kPairsPerPass = kThreads / 8;
-    for (int base = 0; base < pairs; base += 2 * kPairsPerPass) {
-      RhoLoad rl[2];
-#pragma unroll
-      for (int u = 0; u < 2; ++u) {
-        const int pi = base + u * kPairsPerPass + (tid >> 3);
-        rl[u] = RhoLoad{};
-        if (pi < pairs) {
-          const int g = pi % a.G, c = split + (pi / a.G) * a.nsplit;
-          const uint4* qp = reinterpret_cast<const uint4*>(q + (size_t)(hq0 + g) * kD + sub * 16);
-          const uint4* cp = reinterpret_cast<const uint4*>(Cq + ((size_t)(hq0 + g) * a.n_cal + c) * kD + sub * 16);
-          rl[u].q0 = __ldg(qp); rl[u].q1 = __ldg(qp + 1); rl[u].c0 = __ldg(cp); rl[u].c1 = __ldg(cp + 1);
-        }
-      }
-#pragma unroll
-      for (int u = 0; u < 2; ++u) {
-        const int pi = base + u * kPairsPerPass + (tid >> 3);
-        float dot = 0.f, qq = 0.f, cc = 0.f;
-        if (pi < pairs) rho_accumulate(rl[u], dot, qq, cc);
-#pragma unroll
-        for (int o = 1; o < 8; o <<= 1) {
-          dot += __shfl_xor_sync(0xffffffffu, dot, o);
-          qq += __shfl_xor_sync(0xffffffffu, qq, o);
-          cc += __shfl_xor_sync(0xffffffffu, cc, o);
-        }
-        if (sub == 0 && pi < pairs) {
-          const int g = pi % a.G, c = split + (pi / a.G) * a.nsplit;
-          const float rho = (qq > 0.f && cc > 0.f) ? dot / (sqrtf(qq) * sqrtf(cc)) : 0.f;
-          atomicMax(&s_best[g], rank_key(rho, c));
-        }
-      }
-    }
+  // ---- (4) cosine similarities of this CTA's calibration rows; the best pair per head goes to
+  // s_best (the K/V copies are in flight meanwhile)
+  rho_finish(tid >> 2, rl0);
+  rho_finish(kPairsPerPass + (tid >> 2), rl1);
+  for (int base = 2 * kPairsPerPass; base < pairs; base += kPairsPerPass) {
+    rho_load(base + (tid >> 2), rl0);
+    rho_finish(base + (tid >> 2), rl0);
   }
   cluster_arrive();  // (A) this CTA's s_best is final
 
@@ -291,7 +309,9 @@ __global__ void __launch_bounds__(kThreads, 2) decode_kernel(const __grid_consta
   __syncthreads();
   {
     const int d = tid;  // one output dimension per thread
-    for (int g = 0; g < a.G; ++g) {
+#pragma unroll
+    for (int g = 0; g < kMaxG; ++g) {
+      if (g >= a.G) break;
       float M = -INFINITY;
 #pragma unroll
       for (int w = 0; w < kWarps; ++w) M = fmaxf(M, wml[(w * kMaxG + g) * 2]);
@@ -321,9 +341,12 @@ __global__ void __launch_bounds__(kThreads, 2) decode_kernel(const __grid_consta
     const int hq = hq0 + g;
     // the calibration row: best similarity over all CTAs, ties to the largest row index
     unsigned long long best = 0ull;
-    for (int s = 0; s < a.nsplit; ++s) {
-      const unsigned long long k = *cluster.map_shared_rank(&s_best[g], s);
-      best = k > best ? k : best;
+#pragma unroll
+    for (int s = 0; s < 8; ++s) {
+      if (s < a.nsplit) {
+        const unsigned long long k = *cluster.map_shared_rank(&s_best[g], s);
+        best = k > best ? k : best;
+      }
     }
     const int cs = (int)(unsigned)(best & 0xffffffffull);
     const float rho = rank_key_value(best);
@@ -334,15 +357,25 @@ __global__ void __launch_bounds__(kThreads, 2) decode_kernel(const __grid_consta
       oc = __ldg(P.O_c + crow * kD + d);
     }
     if (item0 == 0) cluster_wait();  // (B) every CTA's partial can be read
+    float ms[8], ls[8], os[8];
+#pragma unroll
+    for (int s = 0; s < 8; ++s) {  // all remote reads in flight together
+      ms[s] = -INFINITY; ls[s] = 0.f; os[s] = 0.f;
+      if (s < a.nsplit) {
+        const float2 ml2 = *reinterpret_cast<const float2*>(cluster.map_shared_rank(xml, s) + g * 2);
+        ms[s] = ml2.x; ls[s] = ml2.y;
+        os[s] = cluster.map_shared_rank(xo, s)[g * kD + d];
+      }
+    }
     float M = -INFINITY;
-    for (int s = 0; s < a.nsplit; ++s) M = fmaxf(M, cluster.map_shared_rank(xml, s)[g * 2]);
+#pragma unroll
+    for (int s = 0; s < 8; ++s) M = fmaxf(M, ms[s]);
     float Lsum = 0.f, acc = 0.f;
-    for (int s = 0; s < a.nsplit; ++s) {
-      const float* rml = cluster.map_shared_rank(xml, s);
-      const float ms = rml[g * 2];
-      const float sc = ms > -INFINITY ? ex2_approx(ms - M) : 0.f;
-      Lsum = fmaf(rml[g * 2 + 1], sc, Lsum);
-      acc = fmaf(cluster.map_shared_rank(xo, s)[g * kD + d], sc, acc);
+#pragma unroll
+    for (int s = 0; s < 8; ++s) {
+      const float sc = ms[s] > -INFINITY ? ex2_approx(ms[s] - M) : 0.f;
+      Lsum = fmaf(ls[s], sc, Lsum);
+      acc = fmaf(os[s], sc, acc);
     }
     float outv = acc / Lsum;             // O_a
     float lse2 = M + log2f(Lsum);        // LSE_a (log2 domain)
