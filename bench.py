@@ -35,9 +35,9 @@ import numpy as np  # noqa: E402
 METRIC = "decode attn HBM GB/s (% of peak); compress+calibrate ms/layer (% TC peak)"
 UNIT = "GB/s"
 FALLBACK_HBM_GBS, FALLBACK_BF16_TFLOPS = 6650.0, 1590.0
-# dram__bytes_read.sum + dram__bytes_write.sum per decode launch from the committed ncu capture
-# (see profiles/); None until a capture of the current kernel exists.
-DECODE_DRAM_TRAFFIC_PER_LAUNCH = None
+# dram__bytes_read.sum + dram__bytes_write.sum per decode launch at config 3 from the committed ncu
+# capture (profiles/decode_kernel_config3.md); reported only for that workload.
+DECODE_DRAM_TRAFFIC_PER_LAUNCH = 35854080
 
 
 def load_peaks():
@@ -335,7 +335,8 @@ def run_gpu(args):
                      "min_bytes_gbs": comp_gbs, "frac_of_measured_hbm": comp_gbs / peaks["hbm_gbs"]},
         "roofline": {"bound": "hbm", "kernel": "decode_kernel", "achieved": dec_gbs, "peak": peaks["hbm_gbs"],
                      "unit": "GB/s", "frac": dec_gbs / peaks["hbm_gbs"], "peak_source": peaks["source"],
-                     "traffic": DECODE_DRAM_TRAFFIC_PER_LAUNCH},
+                     "traffic": DECODE_DRAM_TRAFFIC_PER_LAUNCH
+                     if (args.config == 3 and n_cal == 64 and not args.batched_decode) else None},
         "roofline_compress": {"bound": "tensor", "achieved": comp_tflops, "peak": peaks["bf16_tflops_sustained"],
                               "unit": "TFLOP/s", "frac": comp_tflops / peaks["bf16_tflops_sustained"],
                               "peak_source": peaks["source"] + " (sustained bf16 GEMM)"},
