@@ -4,20 +4,22 @@
 // Work is the linear space of (virtual unit, 128-key tile) pairs, a virtual unit being one block
 // of up to 128 calibration rows (whole query heads, n_cal rows each) of a (batch, kv-head) unit;
 // it is cut into equal contiguous ranges, one per CTA, at most one CTA per SM.  Per tile:
-//     MMA 1   S = Q_c K^T       query rows on the TMEM lanes; Q_c itself sits in tensor memory
-//                               (written once per virtual unit), the K tile comes from TMA
+//     MMA 1   S = Q_c K^T       query rows on the TMEM lanes; Q_c block resident in shared memory
+//                               (reloaded per virtual unit), the K tile comes from TMA
 //     threads p = exp2(scale2 * s - lse2[row]), zero for kept keys (bitmap) and for keys outside
-//             the candidates; row sums l kept in fp32; p rounded to bf16 and stored back into the
-//             first 64 columns of the same accumulator buffer, as the A operand of
+//             the candidates; row sums l kept in fp32; p rounded to bf16 and stored into tensor
+//             memory as the A operand of
 //     MMA 2   O += P V          V tile from TMA, read as the MN-major B operand
-// With A in tensor memory both MMAs fetch only their B operand from shared memory, which keeps
-// the N = 128 tiles at the tensor pipe's rate.  lse2[row] is the row's LSE over ALL the keys it
-// sees (from the statistics pass or the caller), so every p <= 1 and no running maximum or
-// rescaling is needed: the partial (O, l) of the key ranges simply add up.
-// calib_reduce_kernel sums them in a fixed order and writes O_c = O / l, LSE_c = lse + log l, C_q.
-// Warp roles: two softmax warpgroups (group g owns accumulator buffer g, i.e. the tiles with
+// MMAs that accumulate into the same tensor-memory tile execute one after the other (about 150
+// cycles each for a 128x128x16 step, twice its math time), so the issuer interleaves the eight
+// k-steps of S(i+2) with the eight of P.V(i): two independent accumulation chains keep the pipe
+// busy.  lse2[row] is the row's LSE over ALL the keys it sees (from the statistics pass or the
+// caller), so every p <= 1 and no running maximum or rescaling is needed: the partial (O, l) of
+// the key ranges simply add up.  calib_reduce_kernel sums them in a fixed order and writes
+// O_c = O / l, LSE_c = lse + log l, C_q.
+// Warp roles: two softmax warpgroups (group g owns S buffer g and P buffer g, i.e. the tiles with
 // local index i % 2 == g), one TMA producer warp, one warp that allocates TMEM and issues MMAs.
-// Tensor memory: S/P buffers at columns 0 and 128, O at 256, Q_c at 384 (64 columns).
+// Tensor memory: S buffers at columns 0 and 128, O at 256, P buffers (64 columns each) at 384, 448.
 #include "internal.h"
 #include "tc_common.cuh"
 
@@ -32,10 +34,10 @@ constexpr int kProducerWarp = kGroups * 4;
 constexpr int kMmaWarp = kGroups * 4 + 1;
 constexpr int kThreads = kGroups * 128 + 64;
 constexpr int kTmemCols = 512;
-constexpr uint32_t kColO = 256, kColQ = 384;
+constexpr uint32_t kColO = 256, kColP = 384;
 constexpr int kStages = 3;                 // K ring and V ring alike
 constexpr int kTileBytes = kKvTileBytes;   // 32 KB
-constexpr int kSmemBytes = 2 * kStages * kTileBytes + 1024;
+constexpr int kSmemBytes = (1 + 2 * kStages) * kTileBytes + 1024;  // Q_c block, K ring, V ring
 constexpr int kSms = 148;
 
 struct CalibArgs {
@@ -46,7 +48,6 @@ struct CalibArgs {
   int total_tiles, tiles_per_cta, max_slots;
   int bitmap_words;
   float scale2;
-  const __nv_bfloat16* Q_obs;
   const float* row_lse;    // [B, Hq, W] natural log
   const uint32_t* bitmap;  // [units][bitmap_words], bit set = kept
   float* o_part;           // [virtual unit][slot][128][128]
@@ -55,8 +56,8 @@ struct CalibArgs {
 };
 
 __global__ void __launch_bounds__(kThreads, 1)
-calib_tc_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__ CUtensorMap v_map,
-                const CalibArgs a) {
+calib_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__ CUtensorMap k_map,
+                const __grid_constant__ CUtensorMap v_map, const CalibArgs a) {
   extern __shared__ unsigned char smem_raw[];
   __shared__ __align__(8) unsigned long long bars[20];
   __shared__ uint32_t tmem_slot;
@@ -70,11 +71,13 @@ calib_tc_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant
   const int Hkv = a.Hq / a.G;
 
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-  const uint32_t k_base = smem_base;
+  const uint32_t q_base = smem_base;
+  const uint32_t k_base = q_base + kTileBytes;
   const uint32_t v_base = k_base + kStages * kTileBytes;
+  unsigned char* const smem_al = smem_raw + (smem_base - smem_u32(smem_raw));
 
   const uint32_t bar0 = smem_u32(bars);
-  const uint32_t o_full = bar0, seg_ready = bar0 + 8u;
+  const uint32_t o_full = bar0, o_empty = bar0 + 8u, q_full = bar0 + 144u, q_empty = bar0 + 152u;
   auto full_k = [&](int s) { return bar0 + 8u * (2 + s); };
   auto empty_k = [&](int s) { return bar0 + 8u * (5 + s); };
   auto full_v = [&](int s) { return bar0 + 8u * (8 + s); };
@@ -86,7 +89,9 @@ calib_tc_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant
     ctl.abort = 0;
     ctl.status = a.status;
     mbar_init(o_full, 1);
-    mbar_init(seg_ready, kGroups * 128);
+    mbar_init(o_empty, kGroups * 128);
+    mbar_init(q_full, 1);
+    mbar_init(q_empty, 1);
     for (int s = 0; s < kStages; ++s) {
       mbar_init(full_k(s), 1); mbar_init(empty_k(s), 1);
       mbar_init(full_v(s), 1); mbar_init(empty_v(s), 1);
@@ -98,6 +103,10 @@ calib_tc_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant
     tmem_alloc(smem_u32(&tmem_slot), kTmemCols);
     tmem_relinquish();
   }
+  // The query block's box may cover fewer than 128 rows: clear the block once so that the rows no
+  // TMA box writes hold zeros.
+  for (int i = tid; i < kTileBytes / 16; i += kThreads) reinterpret_cast<uint4*>(smem_al)[i] = make_uint4(0u, 0u, 0u, 0u);
+  fence_proxy_async_smem();
   tc_fence_before_sync();
   __syncthreads();
   tc_fence_after_sync();
@@ -110,12 +119,23 @@ calib_tc_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant
   if (warp == kProducerWarp) {
     // ------------------------------------------------------------ TMA producer
     if (lane == 0) {
+      tma_prefetch_desc(&q_map);
       tma_prefetch_desc(&k_map);
       tma_prefetch_desc(&v_map);
+      int seg = 0;
       for (int i = 0; i < nt; ++i) {
         const int g = g_begin + i;
         const int vu = g / a.n_tiles, tile = g - vu * a.n_tiles;
         const int unit = vu / a.n_cblocks;
+        if (seg_first(i)) {
+          // the Q_c block of the next virtual unit replaces the current one once its MMAs are done
+          if (seg > 0 && !mbar_wait(&ctl, q_empty, (seg - 1) & 1, 20u | ((unsigned)i << 8))) break;
+          const int g0 = (vu - unit * a.n_cblocks) * a.gpb;
+          mbar_arrive_expect_tx(q_full, 2u * (uint32_t)(a.gpb * a.n_cal) * kLineBytes);
+          for (int half = 0; half < 2; ++half)
+            tma_load_4d(q_base + half * (kTileBytes / 2), &q_map, q_full, half * kHalfCols, 0, g0, unit);
+          ++seg;
+        }
         const int s = i % kStages;
         const uint32_t ph = ((i / kStages) & 1) ^ 1;
         if (!mbar_wait(&ctl, empty_k(s), ph, 21u | ((unsigned)i << 8))) break;
@@ -132,61 +152,79 @@ calib_tc_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant
     }
   } else if (warp == kMmaWarp) {
     // ------------------------------------------------------------ MMA issuer
-    // Issue order: S(0), then for every tile i: S(i+1) (unless tile i+1 starts a new virtual unit,
-    // whose Q_c is only written after O of the current one has been read out), P.V(i).  The tensor
-    // pipe executes in issue order, so S(i+2) cannot overwrite buffer i % 2 before P.V(i) has read P.
+    // At the start of a virtual unit S(i) and S(i+1) are issued (k-steps interleaved); from then on
+    // P.V(i) is issued together with S(i+2), again interleaved, as soon as P(i) is complete (which
+    // also means S(i) has been read out of its buffer).  S never runs ahead across a change of
+    // virtual unit: its Q_c block is only loaded once the current unit's MMAs are done.
     if (lane == 0) {
-      const uint32_t idesc = umma_idesc(128, 128, false, false);     // S: B = K tile, K-major
-      const uint32_t idesc_o = umma_idesc(128, 128, false, true);    // O: B = V tile, MN-major
-      const uint32_t tmem_q = tmem_base + kColQ, tmem_o = tmem_base + kColO;
-      int next_s = 0, seg = 0;
+      const uint32_t idesc = umma_idesc(128, 128, false, false);     // S: A = Q_c, B = K tile, K-major
+      const uint32_t idesc_o = umma_idesc(128, 128, false, true);    // O: A = P (TMEM), B = V tile, MN-major
+      const uint32_t tmem_o = tmem_base + kColO;
+      int seg = 0;
       bool ok = true;
-      auto issue_s = [&](int i) -> bool {
-        const int s = i % kStages, buf = i & 1;
-        if (!mbar_wait(&ctl, full_k(s), (i / kStages) & 1, 24u | ((unsigned)i << 8))) return false;
-        tc_fence_after_sync();
-#pragma unroll
-        for (int kk = 0; kk < kD / 16; ++kk)
-          umma_ts(tmem_base + (uint32_t)(buf * 128), tmem_q + (uint32_t)(kk * 8),
-                  kmajor_desc(k_base + s * kTileBytes, kTileBytes / 2, kk), idesc, kk > 0 ? 1u : 0u);
-        umma_commit(s_full(buf));
-        umma_commit(empty_k(s));
-        return true;
+      // k-step kk of S(i) and of P.V(i)
+      auto s_step = [&](int i, int kk) {
+        const int s = i % kStages;
+        umma_ss(tmem_base + (uint32_t)((i & 1) * 128), kmajor_desc(q_base, kTileBytes / 2, kk),
+                kmajor_desc(k_base + s * kTileBytes, kTileBytes / 2, kk), idesc, kk > 0 ? 1u : 0u);
       };
+      auto pv_step = [&](int i, int kk, bool first) {
+        // A: P, 16 keys = 8 columns per step.  B: V tile with the keys as K, i.e. MN-major: blocks
+        // of 64 head-dim elements are half a tile apart, groups of 8 keys 1024 bytes apart.
+        const int s = i % kStages;
+        const uint64_t vd = smem_desc_sw128(v_base + s * kTileBytes + (uint32_t)kk * 16u * kLineBytes,
+                                            kTileBytes / 2, 1024u);
+        umma_ts(tmem_o, tmem_base + kColP + (uint32_t)((i & 1) * 64 + kk * 8), vd, idesc_o,
+                (!first || kk > 0) ? 1u : 0u);
+      };
+      auto wait_k = [&](int i) { return mbar_wait(&ctl, full_k(i % kStages), (i / kStages) & 1, 24u | ((unsigned)i << 8)); };
+      auto s_done = [&](int i) { umma_commit(s_full(i & 1)); umma_commit(empty_k(i % kStages)); };
       for (int i = 0; ok && i < nt; ++i) {
-        while (ok && next_s < nt && next_s <= i + 1) {
-          if (seg_first(next_s)) {
-            if (next_s > i) break;  // not across the boundary: P.V(i) and the read-out of O come first
-            ok = mbar_wait(&ctl, seg_ready, seg & 1, 23u | ((unsigned)i << 8));
-            ++seg;
-            if (!ok) break;
-          }
-          ok = issue_s(next_s);
-          ++next_s;
-        }
-        if (!ok) break;
-        const int s = i % kStages, buf = i & 1;
-        if (!mbar_wait(&ctl, p_full(buf), (i >> 1) & 1, 26u | ((unsigned)i << 8))) break;
-        if (!mbar_wait(&ctl, full_v(s), (i / kStages) & 1, 27u | ((unsigned)i << 8))) break;
-        tc_fence_after_sync();
         const bool first = seg_first(i);
+        if (first) {
+          // new virtual unit: its Q_c block must have landed, and O of the previous unit must have
+          // been read out before the first P.V overwrites it
+          ok = mbar_wait(&ctl, q_full, seg & 1, 23u | ((unsigned)i << 8));
+          if (ok && seg > 0) ok = mbar_wait(&ctl, o_empty, (seg - 1) & 1, 25u | ((unsigned)i << 8));
+          ++seg;
+          if (!ok) break;
+          const bool two = !seg_last(i);
+          ok = wait_k(i) && (!two || wait_k(i + 1));
+          if (!ok) break;
+          tc_fence_after_sync();
+#pragma unroll
+          for (int kk = 0; kk < kD / 16; ++kk) {
+            s_step(i, kk);
+            if (two) s_step(i + 1, kk);
+          }
+          s_done(i);
+          if (two) s_done(i + 1);
+        }
+        // P.V(i), together with S(i+2) when that tile belongs to the same virtual unit
+        const bool with_s = !seg_last(i) && !seg_last(i + 1);
+        if (!mbar_wait(&ctl, p_full(i & 1), (i >> 1) & 1, 26u | ((unsigned)i << 8))) break;
+        if (!mbar_wait(&ctl, full_v(i % kStages), (i / kStages) & 1, 27u | ((unsigned)i << 8))) break;
+        if (with_s && !wait_k(i + 2)) break;
+        tc_fence_after_sync();
 #pragma unroll
         for (int kk = 0; kk < kTileKeys / 16; ++kk) {
-          // A: P, 16 keys = 8 columns per step.  B: V tile with the keys as K, i.e. MN-major: blocks
-          // of 64 head-dim elements are half a tile apart, groups of 8 keys 1024 bytes apart.
-          const uint64_t vd = smem_desc_sw128(v_base + s * kTileBytes + (uint32_t)kk * 16u * kLineBytes,
-                                              kTileBytes / 2, 1024u);
-          umma_ts(tmem_o, tmem_base + (uint32_t)(buf * 128 + kk * 8), vd, idesc_o, (!first || kk > 0) ? 1u : 0u);
+          pv_step(i, kk, first);
+          if (with_s) s_step(i + 2, kk);
         }
-        umma_commit(empty_v(s));
-        if (seg_last(i)) umma_commit(o_full);
+        if (with_s) s_done(i + 2);
+        umma_commit(empty_v(i % kStages));
+        if (seg_last(i)) {
+          umma_commit(o_full);
+          umma_commit(q_empty);
+        }
       }
     }
   } else {
     // ------------------------------------------------------------ softmax threads (one row each)
     const int grp = warp >> 2, r = tid & 127;
     const uint32_t lane_bits = (uint32_t)((warp & 3) * 32) << 16;
-    const uint32_t taddr = tmem_base + lane_bits + (uint32_t)(grp * 128);  // this group's S/P buffer
+    const uint32_t taddr = tmem_base + lane_bits + (uint32_t)(grp * 128);  // this group's S buffer
+    const uint32_t paddr = tmem_base + lane_bits + kColP + (uint32_t)(grp * 64);  // and its P buffer
     float l0 = 0.f, l1 = 0.f, nlse2 = -INFINITY;
     int cur_vu = -1, seg = 0;
     bool ok = true, valid = false;
@@ -212,34 +250,22 @@ calib_tc_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant
         }
       }
       if (valid) a.l_part[(part * kGroups + grp) * 128 + r] = l0 + l1;
+      tc_fence_before_sync();
+      mbar_arrive(o_empty);
       return true;
     };
-    // Write this thread's half (64 head-dim elements) of its query row into the Q_c columns.
+    // This thread's row of the virtual unit: is there one, and its -lse2.
     auto load_q = [&](int vu) {
       const int unit = vu / a.n_cblocks, cb = vu - unit * a.n_cblocks;
       const int hq0 = (unit / Hkv) * a.Hq + (unit % Hkv) * a.G;
       const int g0 = cb * a.gpb;
       const int rows = min(a.gpb, a.G - g0) * a.n_cal;
       valid = r < rows;
-      uint32_t qv[32];
-#pragma unroll
-      for (int e = 0; e < 32; ++e) qv[e] = 0u;
       nlse2 = -INFINITY;
       if (valid) {
         const int g = g0 + r / a.n_cal, c = r - (r / a.n_cal) * a.n_cal;
-        const size_t qrow = (size_t)(hq0 + g) * a.W + (a.W - a.n_cal + c);
-        nlse2 = -a.row_lse[qrow] * kLog2e;
-        const uint4* src = reinterpret_cast<const uint4*>(a.Q_obs + qrow * kD + grp * 64);
-#pragma unroll
-        for (int e = 0; e < 8; ++e) {
-          const uint4 v = __ldg(src + e);
-          qv[4 * e] = v.x; qv[4 * e + 1] = v.y; qv[4 * e + 2] = v.z; qv[4 * e + 3] = v.w;
-        }
+        nlse2 = -a.row_lse[(size_t)(hq0 + g) * a.W + (a.W - a.n_cal + c)] * kLog2e;
       }
-      tmem_st32(tmem_base + lane_bits + kColQ + (uint32_t)(grp * 32), qv);
-      tmem_st_wait();
-      tc_fence_before_sync();
-      mbar_arrive(seg_ready);
     };
 
     const uint32_t* bm_all = a.bitmap;
@@ -276,7 +302,7 @@ calib_tc_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       tc_fence_after_sync();
-      // probabilities of 32 keys -> bf16 pairs -> columns [16 q, 16 q + 16) of the same buffer
+      // probabilities of 32 keys -> bf16 pairs -> columns [16 q, 16 q + 16) of the P buffer
       auto soft32 = [&](const uint32_t (&sv)[32], int q, uint32_t w) {
         uint32_t packed[16];
 #pragma unroll
@@ -289,7 +315,7 @@ calib_tc_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant
           l1 += p1;
           packed[e >> 1] = pack_bf16(p0, p1);
         }
-        tmem_st16(taddr + (uint32_t)(16 * q), packed);
+        tmem_st16(paddr + (uint32_t)(16 * q), packed);
       };
       uint32_t ra[32], rb[32];
       tmem_ld32_issue(taddr, ra);
@@ -391,13 +417,18 @@ cudaError_t launch_calib_tc(const CompressGeom& g, const CompressWs& ws, const v
   a.total_tiles = g.units * a.n_cblocks * a.n_tiles;
   a.bitmap_words = g.bitmap_words;
   a.scale2 = g.scale2;
-  a.Q_obs = (const __nv_bfloat16*)Q_obs;
   a.row_lse = row_lse;
   a.bitmap = (const uint32_t*)(wsp + ws.bitmap);
   a.o_part = (float*)(wsp + ws.calib_o);
   a.l_part = (float*)(wsp + ws.calib_l);
   a.status = (unsigned*)(wsp + ws.status);
-  CUtensorMap km, vm;
+  CUtensorMap qm, km, vm;
+  // calibration rows: [head dim][c < n_cal][g < G][unit], starting at observation row W - n_cal
+  const uint64_t qd[3] = {(uint64_t)g.n_cal, (uint64_t)g.G, (uint64_t)g.units};
+  const uint64_t qs[3] = {256, (uint64_t)g.W * 256, (uint64_t)g.G * g.W * 256};
+  const uint32_t qb[3] = {(uint32_t)g.n_cal, (uint32_t)a.gpb, 1};
+  const char* q0 = (const char*)Q_obs + (size_t)(g.W - g.n_cal) * 256;
+  if (!make_tensor_map_bf16(&qm, q0, 4, qd, qs, qb)) return cudaErrorInvalidValue;
   const uint64_t kd[2] = {(uint64_t)g.L, (uint64_t)g.units}, ks[2] = {256, (uint64_t)g.L * 256};
   const uint32_t kb[2] = {(uint32_t)kTileKeys, 1};
   if (!make_tensor_map_bf16(&km, K, 3, kd, ks, kb) || !make_tensor_map_bf16(&vm, V, 3, kd, ks, kb))
@@ -412,7 +443,7 @@ cudaError_t launch_calib_tc(const CompressGeom& g, const CompressWs& ws, const v
     if (dev >= 0 && dev < 64) attr_set[dev] = true;
   }
   const int grid = (a.total_tiles + a.tiles_per_cta - 1) / a.tiles_per_cta;
-  calib_tc_kernel<<<grid, kThreads, kSmemBytes, st>>>(km, vm, a);
+  calib_tc_kernel<<<grid, kThreads, kSmemBytes, st>>>(qm, km, vm, a);
   const int total = g.B * g.Hq * g.n_cal;
   calib_reduce_kernel<<<(total + 3) / 4, 128, 0, st>>>((const __nv_bfloat16*)Q_obs, row_lse, a.o_part, a.l_part, O_c,
                                                       LSE_c, (__nv_bfloat16*)C_q, g.B, g.Hq, g.G, g.W, g.n_cal,
