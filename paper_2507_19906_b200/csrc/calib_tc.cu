@@ -113,8 +113,10 @@ calib_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
   const uint32_t tmem_base = tmem_slot;
 
   // first tile of a run of tiles of one virtual unit inside this CTA's range
-  auto seg_first = [&](int i) { return i == 0 || (g_begin + i) % a.n_tiles == 0; };
-  auto seg_last = [&](int i) { return i == nt - 1 || (g_begin + i + 1) % a.n_tiles == 0; };
+  // (the position inside the tile space is tracked incrementally: no division per tile)
+  const int vu_begin = g_begin / a.n_tiles, tile_begin = g_begin - vu_begin * a.n_tiles;
+  auto seg_first = [&](int i, int tile) { return i == 0 || tile == 0; };
+  auto seg_last = [&](int i, int tile) { return i == nt - 1 || tile == a.n_tiles - 1; };
 
   if (warp == kProducerWarp) {
     // ------------------------------------------------------------ TMA producer
@@ -122,12 +124,10 @@ calib_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
       tma_prefetch_desc(&q_map);
       tma_prefetch_desc(&k_map);
       tma_prefetch_desc(&v_map);
-      int seg = 0;
-      for (int i = 0; i < nt; ++i) {
-        const int g = g_begin + i;
-        const int vu = g / a.n_tiles, tile = g - vu * a.n_tiles;
-        const int unit = vu / a.n_cblocks;
-        if (seg_first(i)) {
+      int seg = 0, vu = vu_begin, tile = tile_begin, unit = vu_begin / a.n_cblocks;
+      for (int i = 0; i < nt; ++i, ++tile) {
+        if (tile == a.n_tiles) { tile = 0; ++vu; unit = vu / a.n_cblocks; }
+        if (seg_first(i, tile)) {
           // the Q_c block of the next virtual unit replaces the current one once its MMAs are done
           if (seg > 0 && !mbar_wait(&ctl, q_empty, (seg - 1) & 1, 20u | ((unsigned)i << 8))) break;
           const int g0 = (vu - unit * a.n_cblocks) * a.gpb;
@@ -179,8 +179,10 @@ calib_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
       };
       auto wait_k = [&](int i) { return mbar_wait(&ctl, full_k(i % kStages), (i / kStages) & 1, 24u | ((unsigned)i << 8)); };
       auto s_done = [&](int i) { umma_commit(s_full(i & 1)); umma_commit(empty_k(i % kStages)); };
-      for (int i = 0; ok && i < nt; ++i) {
-        const bool first = seg_first(i);
+      int tile = tile_begin;
+      for (int i = 0; ok && i < nt; ++i, ++tile) {
+        if (tile == a.n_tiles) tile = 0;
+        const bool first = seg_first(i, tile), last = seg_last(i, tile);
         if (first) {
           // new virtual unit: its Q_c block must have landed, and O of the previous unit must have
           // been read out before the first P.V overwrites it
@@ -188,7 +190,7 @@ calib_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
           if (ok && seg > 0) ok = mbar_wait(&ctl, o_empty, (seg - 1) & 1, 25u | ((unsigned)i << 8));
           ++seg;
           if (!ok) break;
-          const bool two = !seg_last(i);
+          const bool two = !last;
           ok = wait_k(i) && (!two || wait_k(i + 1));
           if (!ok) break;
           tc_fence_after_sync();
@@ -201,7 +203,7 @@ calib_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
           if (two) s_done(i + 1);
         }
         // P.V(i), together with S(i+2) when that tile belongs to the same virtual unit
-        const bool with_s = !seg_last(i) && !seg_last(i + 1);
+        const bool with_s = !last && !seg_last(i + 1, tile + 1);
         if (!mbar_wait(&ctl, p_full(i & 1), (i >> 1) & 1, 26u | ((unsigned)i << 8))) break;
         if (!mbar_wait(&ctl, full_v(i % kStages), (i / kStages) & 1, 27u | ((unsigned)i << 8))) break;
         if (with_s && !wait_k(i + 2)) break;
@@ -213,7 +215,7 @@ calib_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
         }
         if (with_s) s_done(i + 2);
         umma_commit(empty_v(i % kStages));
-        if (seg_last(i)) {
+        if (last) {
           umma_commit(o_full);
           umma_commit(q_empty);
         }
@@ -269,9 +271,9 @@ calib_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
     };
 
     const uint32_t* bm_all = a.bitmap;
-    for (int i = 0; i < nt; ++i) {
-      const int g = g_begin + i;
-      const int vu = g / a.n_tiles, tile = g - vu * a.n_tiles;
+    int vu = vu_begin, tile = tile_begin, unit = vu_begin / a.n_cblocks;
+    for (int i = 0; i < nt; ++i, ++tile) {
+      if (tile == a.n_tiles) { tile = 0; ++vu; unit = vu / a.n_cblocks; }
       if (vu != cur_vu) {
         if (cur_vu >= 0) {
           ok = store_partial(cur_vu);
@@ -285,7 +287,6 @@ calib_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
       if ((i & 1) != grp) continue;
       // kept-key bits of the tile's 128 keys (bit set = the key does not contribute), fetched
       // before the wait so that the loads are off the critical path
-      const int unit = vu / a.n_cblocks;
       const uint32_t* bm = bm_all + (size_t)unit * a.bitmap_words;
       const int tbase = tile * kTileKeys;
       uint32_t word[4];

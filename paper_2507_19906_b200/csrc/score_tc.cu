@@ -102,6 +102,8 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
   const int g_end = min(a.total_tiles, g_begin + a.tiles_per_cta);
   const int nt = g_end - g_begin;
   const int Hkv = a.Hq / a.G;
+  // (the position inside the tile space is tracked incrementally: no division per tile)
+  const int vu_begin = g_begin / a.n_tiles, tile_begin = g_begin - vu_begin * a.n_tiles;
 
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   const uint32_t q_half_bytes = (uint32_t)a.block_rows * kLineBytes;
@@ -139,11 +141,9 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
     if (lane == 0) {
       tma_prefetch_desc(&q_map);
       tma_prefetch_desc(&k_map);
-      int cur_vu = -1, seg = 0;
-      for (int i = 0; i < nt; ++i) {
-        const int g = g_begin + i;
-        const int vu = g / a.n_tiles, tile = g - vu * a.n_tiles;
-        const int unit = vu / a.vu_per_unit;
+      int cur_vu = -1, seg = 0, vu = vu_begin, tile = tile_begin, unit = vu_begin / a.vu_per_unit;
+      for (int i = 0; i < nt; ++i, ++tile) {
+        if (tile == a.n_tiles) { tile = 0; ++vu; unit = vu / a.vu_per_unit; }
         if (vu != cur_vu) {
           // the query rows of the next virtual unit replace the current ones once its MMAs are done
           if (seg > 0 && !mbar_wait(&ctl, q_empty, (seg - 1) & 1, (kVotes ? 36u : 16u) | ((unsigned)i << 8))) break;
@@ -168,10 +168,9 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
     // ------------------------------------------------------------ MMA issuer
     if (lane == 0) {
       const uint32_t idesc = umma_idesc(128, kVotes ? a.block_rows : 256, false, false);
-      int cur_vu = -1, seg = 0, j = 0;
-      for (int i = 0; i < nt; ++i) {
-        const int g = g_begin + i;
-        const int vu = g / a.n_tiles;
+      int cur_vu = -1, seg = 0, j = 0, vu = vu_begin, tile = tile_begin;
+      for (int i = 0; i < nt; ++i, ++tile) {
+        if (tile == a.n_tiles) { tile = 0; ++vu; }
         if (vu != cur_vu) {
           if (!mbar_wait(&ctl, q_full, seg & 1, (kVotes ? 32u : 12u) | ((unsigned)i << 8))) break;
           cur_vu = vu;
@@ -199,7 +198,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
         }
         if (!ok) break;
         umma_commit(empty_k(s));
-        const bool last_of_vu = (i == nt - 1) || ((g + 1) / a.n_tiles != vu);
+        const bool last_of_vu = (i == nt - 1) || (tile == a.n_tiles - 1);
         if (last_of_vu) umma_commit(q_empty);
       }
     }
@@ -226,11 +225,13 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
       }
     };
 
-    for (int i = 0; i < nt && ok; ++i) {
-      const int g = g_begin + i;
-      const int vu = g / a.n_tiles, tile = g - vu * a.n_tiles;
-      const int unit = vu / a.vu_per_unit;
-      const int row0 = (vu - unit * a.vu_per_unit) * a.vu_rows;
+    int vu = vu_begin, tile = tile_begin, unit = vu_begin / a.vu_per_unit;
+    int row0 = (vu - unit * a.vu_per_unit) * a.vu_rows;
+    for (int i = 0; i < nt && ok; ++i, ++tile) {
+      if (tile == a.n_tiles) {
+        tile = 0; ++vu; unit = vu / a.vu_per_unit;
+        row0 = (vu - unit * a.vu_per_unit) * a.vu_rows;
+      }
       if (vu != cur_vu) {
         if (kVotes) {
           // this warp's copy of -lse2 of the unit's window rows (-inf for the padding rows); warps
