@@ -29,7 +29,7 @@ namespace {
 
 using namespace tc;
 
-constexpr int kGroups = 2;  // consumer warpgroups (4 warps each); group g consumes accumulator g
+constexpr int kGroups = 2;  // consumer warpgroups (4 warps each); both work on the same accumulator, half of its columns each
 constexpr int kProducerWarp = kGroups * 4;
 constexpr int kMmaWarp = kGroups * 4 + 1;
 constexpr int kThreads = kGroups * 128 + 64;
@@ -90,9 +90,10 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
   constexpr int TILE_KEYS = kVotes ? 128 : 256;
   constexpr uint32_t STAGE_BYTES = TILE_KEYS * 256;
   extern __shared__ unsigned char smem_raw[];
-  __shared__ __align__(8) unsigned long long bars[16];
+  __shared__ __align__(8) unsigned long long bars[18];
   __shared__ uint32_t tmem_slot;
   __shared__ Ctl ctl;
+  __shared__ float vx[2][128];  // votes: partial vote of the second column half, per accumulator
   __shared__ __align__(16) float nlse2_s[kVotes ? kGroups * 4 : 1][kVotes ? kMaxRows : 4];  // -lse2 per row, one copy per warp
   __shared__ float2 ml_s[kVotes ? 1 : kGroups][kVotes ? 1 : 2][kVotes ? 1 : 128];       // running (max, sum)
 
@@ -117,6 +118,8 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
   auto empty_k = [&](int s) { return bar0 + 8u * (6 + s); };
   auto t_full = [&](int b) { return bar0 + 8u * (10 + b); };
   auto t_empty = [&](int b) { return bar0 + 8u * (12 + b); };
+  auto vx_full = [&](int b) { return bar0 + 8u * (14 + b); };
+  auto vx_empty = [&](int b) { return bar0 + 8u * (16 + b); };
 
   if (tid == 0) {
     ctl.abort = 0;
@@ -124,7 +127,10 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
     mbar_init(q_full, 1);
     mbar_init(q_empty, 1);
     for (int s = 0; s < 4; ++s) { mbar_init(full_k(s), 1); mbar_init(empty_k(s), 1); }
-    for (int b = 0; b < 2; ++b) { mbar_init(t_full(b), 1); mbar_init(t_empty(b), 128); }
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(t_full(b), 1); mbar_init(t_empty(b), kGroups * 128);
+      mbar_init(vx_full(b), 128); mbar_init(vx_empty(b), 128);
+    }
     fence_mbar_init();
   }
   if (warp == kMmaWarp) {
@@ -204,10 +210,11 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
     }
   } else {
     // ------------------------------------------------------------ accumulator consumers
-    // Thread ct of warpgroup grp owns TMEM lane ct and consumes the jobs (key tile, row block) whose
-    // running index is congruent to grp mod 2, i.e. the accumulator buffer grp.
+    // Thread ct of warpgroup grp owns TMEM lane ct.  Both groups consume every job (key tile, row
+    // block), each one half of the accumulator's columns: a job is then drained at the full rate
+    // of the exponential unit while the MMAs of the next job fill the other accumulator.
     const int grp = warp >> 2, ct = tid & 127;
-    const uint32_t lane_addr = tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)(grp * kBufCols);
+    const uint32_t lane_base = tmem_base + ((uint32_t)((warp & 3) * 32) << 16);
     float acc0 = 0.f, acc1 = 0.f, acc2 = 0.f, acc3 = 0.f;  // votes: running vote of this thread's key
     int cur_vu = -1, j = 0;
     bool ok = true;
@@ -249,14 +256,17 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
       }
       const int tbase = tile * TILE_KEYS;
       for (int blk = 0; blk < a.n_blocks; ++blk, ++j) {
-        if ((j & 1) != grp) continue;
-        ok = mbar_wait(&ctl, t_full(grp), (j >> 1) & 1, (kVotes ? 35u : 15u) | ((unsigned)j << 8));
+        const int buf = j & 1;
+        const uint32_t lane_addr = lane_base + (uint32_t)(buf * kBufCols);
+        ok = mbar_wait(&ctl, t_full(buf), (j >> 1) & 1, (kVotes ? 35u : 15u) | ((unsigned)j << 8));
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) break;
         tc_fence_after_sync();
         uint32_t ra[32], rb[32];
         if (kVotes) {
-          const float* nl = nlse2_s[warp] + blk * a.block_rows;
+          const int cw = a.block_rows >> 1;  // columns (query rows) of this group: a multiple of 32
+          const float* nl = nlse2_s[warp] + blk * a.block_rows + grp * cw;
+          const uint32_t tcol = lane_addr + (uint32_t)(grp * cw);
           auto add32 = [&](const uint32_t (&r)[32], int c0) {
 #pragma unroll
             for (int e = 0; e < 32; e += 4) {
@@ -268,24 +278,39 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
             }
           };
           // block_rows is a multiple of 32: chunks alternate between the two register sets
-          tmem_ld32_issue(lane_addr, ra);
-          for (int c0 = 0; c0 < a.block_rows; c0 += 64) {
+          tmem_ld32_issue(tcol, ra);
+          for (int c0 = 0; c0 < cw; c0 += 64) {
             tmem_ld_wait(ra);
-            const bool more_b = c0 + 32 < a.block_rows;
-            if (more_b) tmem_ld32_issue(lane_addr + c0 + 32, rb);
+            const bool more_b = c0 + 32 < cw;
+            if (more_b) tmem_ld32_issue(tcol + c0 + 32, rb);
             add32(ra, c0);
             if (more_b) {
               tmem_ld_wait(rb);
-              if (c0 + 64 < a.block_rows) tmem_ld32_issue(lane_addr + c0 + 64, ra);
+              if (c0 + 64 < cw) tmem_ld32_issue(tcol + c0 + 64, ra);
               add32(rb, c0 + 32);
             }
           }
           tc_fence_before_sync();
-          mbar_arrive(t_empty(grp));
-          const int key = tbase + ct;
-          float* out = blk == 0 ? a.vote : a.vote2;
-          if (key < a.n_cand) out[(size_t)unit * a.n_cand + key] = (acc0 + acc1) + (acc2 + acc3);
+          mbar_arrive(t_empty(buf));
+          // the two halves of the key's vote meet in shared memory; group 0 stores the sum
+          const float part = (acc0 + acc1) + (acc2 + acc3);
           acc0 = acc1 = acc2 = acc3 = 0.f;
+          if (grp == 1) {
+            ok = mbar_wait(&ctl, vx_empty(buf), ((j >> 1) & 1) ^ 1, 37u | ((unsigned)j << 8));
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+            vx[buf][ct] = part;
+            mbar_arrive(vx_full(buf));
+          } else {
+            ok = mbar_wait(&ctl, vx_full(buf), (j >> 1) & 1, 38u | ((unsigned)j << 8));
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+            const float v = part + vx[buf][ct];
+            mbar_arrive(vx_empty(buf));
+            const int key = tbase + ct;
+            float* out = blk == 0 ? a.vote : a.vote2;
+            if (key < a.n_cand) out[(size_t)unit * a.n_cand + key] = v;
+          }
         } else {
           float2 ml = ml_s[grp][blk][ct];
           const int row = row0 + blk * 128 + ct;
@@ -304,18 +329,19 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
               ml.x = m_new;
             }
           };
-          tmem_ld32_issue(lane_addr, ra);
+          const int cbeg = grp * (TILE_KEYS / 2), cend = cbeg + TILE_KEYS / 2;  // this group's keys of the tile
+          tmem_ld32_issue(lane_addr + cbeg, ra);
 #pragma unroll 1
-          for (int c0 = 0; c0 < TILE_KEYS; c0 += 64) {
+          for (int c0 = cbeg; c0 < cend; c0 += 64) {
             tmem_ld_wait(ra);
             tmem_ld32_issue(lane_addr + c0 + 32, rb);
             fold32(ra, c0);
             tmem_ld_wait(rb);
-            if (c0 + 64 < TILE_KEYS) {
+            if (c0 + 64 < cend) {
               tmem_ld32_issue(lane_addr + c0 + 64, ra);
             } else {
               tc_fence_before_sync();
-              mbar_arrive(t_empty(grp));  // the accumulator is in registers: hand the buffer back early
+              mbar_arrive(t_empty(buf));  // the accumulator is in registers: hand the buffer back early
             }
             fold32(rb, c0 + 32);
           }
@@ -451,7 +477,7 @@ cudaError_t launch_votes_tc(const CompressGeom& g, const CompressWs& ws, const v
   // One accumulator of up to 256 row columns per (key tile, row block); with two row blocks each
   // warpgroup sums one block and the two partial votes are added afterwards.
   a.n_blocks = GW <= 256 ? 1 : 2;
-  a.block_rows = ((GW + a.n_blocks - 1) / a.n_blocks + 31) / 32 * 32;
+  a.block_rows = ((GW + a.n_blocks - 1) / a.n_blocks + 63) / 64 * 64;
   a.n_tiles = (g.n_cand + kTileKeys - 1) / kTileKeys;
   partition_tiles(a, g.units);
   const int q_bytes = a.n_blocks * a.block_rows * 256;
