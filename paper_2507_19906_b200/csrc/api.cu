@@ -139,7 +139,7 @@ DecodeWs make_decode_ws(const calidrop_params* p) {
   size_t off = 0;
   w.counters = off; off = align_up(off + (size_t)units * 4 * kDecodeMaxLayers, 256);
   w.part_ml = off;  off = align_up(off + (size_t)units * w.max_split * kMaxG * 2 * 4, 256);
-  w.rho = off;      off = align_up(off + (size_t)units * kMaxG * p->n_cal * 4, 256);
+  w.rho = off;      off = align_up(off + (size_t)units * kMaxG * w.max_split * 8, 256);
   w.part_o = off;   off = align_up(off + (size_t)units * w.max_split * kMaxG * kD * 4, 256);
   w.per_layer = off;
   return w;
@@ -278,9 +278,13 @@ int calidrop_decode_batched(const calidrop_params* p, int32_t n_layers, const ca
   a.units = p->B * p->Hkv; a.n_layers = n_layers;
   // the splits of a unit form one thread-block cluster: 1, 2, 4 or 8 CTAs
   int want = decode_nsplit(a.units * n_layers, n_kv);
+  if (want > w.max_split) want = w.max_split;
   a.nsplit = 1;
   while (a.nsplit * 2 <= want && a.nsplit < 8) a.nsplit *= 2;
-  a.rows_per_split = (n_kv + a.nsplit - 1) / a.nsplit;
+  // few units with a long cache: several clusters per unit, combined through the workspace
+  a.nclu = want / a.nsplit;
+  if (a.nclu < 1) a.nclu = 1;
+  a.rows_per_split = (n_kv + a.nsplit * a.nclu - 1) / (a.nsplit * a.nclu);
   a.scale2 = scale2_of(p);
   a.theta1 = p->theta1; a.theta2 = p->theta2; a.always_apply = p->theta2 <= -1.0f;
   // The workspace is laid out array by array with the layer index outermost inside each
@@ -289,8 +293,8 @@ int calidrop_decode_batched(const calidrop_params* p, int32_t n_layers, const ca
   const size_t nl = (size_t)n_layers;
   size_t off = 0;
   a.counters = (unsigned*)(base + off); off += align_up((size_t)a.units * 4 * kDecodeMaxLayers, 256);
-  a.part_ml = (float*)(base + off);     off += align_up((size_t)a.units * a.nsplit * kMaxG * 2 * 4 * nl, 256);
-  a.rho = (float*)(base + off);         off += align_up((size_t)a.units * kMaxG * p->n_cal * 4 * nl, 256);
+  a.part_ml = (float*)(base + off);     off += align_up((size_t)a.units * a.nclu * kMaxG * 2 * 4 * nl, 256);
+  a.part_best = (unsigned long long*)(base + off); off += align_up((size_t)a.units * a.nclu * kMaxG * 8 * nl, 256);
   a.part_o = (float*)(base + off);
   for (int i = 0; i < n_layers; ++i) {
     const calidrop_decode_layer& L = layers[i];

@@ -7,13 +7,17 @@
 // HBM traffic (about 2G flop per byte), so the contraction uses the warp-level mma.sync path
 // with G <= 8 rows of a 16-row tile; tcgen05 tiles (64 rows minimum) would add nothing here.
 //
-// Grid: (split, batch*kv-head, layer); the splits of one (unit, layer) form a thread-block
-// cluster of 1, 2, 4 or 8 CTAs.  Each CTA streams its slice of rows through shared memory with
+// Grid: (split, batch*kv-head, layer); the splits of one (unit, layer) form thread-block
+// clusters of 1, 2, 4 or 8 CTAs.  Each CTA streams its slice of rows through shared memory with
 // 16-byte cp.async copies (XOR-swizzled so ldmatrix is conflict-free), four warps each running
 // an independent online softmax over interleaved 16-row blocks.  The splits are combined inside
 // the cluster through distributed shared memory: every CTA finishes a slice of the 128 output
 // dimensions for all heads of the group, so there is no global-memory round trip, no ticket and
-// no CTA that works alone at the end.
+// no CTA that works alone at the end.  Only when very few units share a long cache (fewer than
+// 19 units per launch) does one cluster per unit leave most SMs idle; then a unit gets up to
+// eight clusters, each writes its combined partial, its (max, sum) pair and its best similarity
+// to the workspace, and the CTA that takes the last ticket of the unit's arrival counter merges
+// them and resets the counter.
 //
 // A launch moves only tens of MB, so its latency chain matters as much as its bandwidth:
 //   * the launch carries the programmatic-serialisation attribute and the kernel prefetches its
@@ -82,12 +86,42 @@ __device__ __forceinline__ void cluster_wait() {
   asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
 
+// Gate and merge of one output element (Eq. 1-2): (acc, M, Lsum) is the unnormalised partial of
+// the retained cache in the log2 domain, best the chosen (similarity, calibration row) key.
+__device__ __forceinline__ void merge_store(const DecodeArgs& a, const DecodeLayerPtrs& P, int hq, int d, float acc,
+                                            float M, float Lsum, unsigned long long best, float lse_c, float oc) {
+  const int cs = (int)(unsigned)(best & 0xffffffffull);
+  const float rho = rank_key_value(best);
+  float outv = acc / Lsum;       // O_a
+  float lse2 = M + log2f(Lsum);  // LSE_a (log2 domain)
+  const bool apply = (a.always_apply || rho > a.theta2) && (lse_c > -INFINITY);
+  if (apply) {
+    // alpha_i = e^{LSE_a - LSE}, alpha_j = e^{LSE_c - LSE}; out = alpha_i O_a + alpha_j O_c
+    const float lc2 = lse_c * kLog2e;
+    const float mx = fmaxf(lse2, lc2);
+    const float ea = exp2f(lse2 - mx), ec = exp2f(lc2 - mx);
+    const float tot = ea + ec;
+    outv = (ea / tot) * outv + (ec / tot) * oc;
+    lse2 = mx + log2f(tot);
+  }
+  reinterpret_cast<__nv_bfloat16*>(P.out)[(size_t)hq * kD + d] = __float2bfloat16_rn(outv);
+  if (d == 0) {
+    if (P.lse_out) P.lse_out[hq] = lse2 * kLn2;
+    if (P.flags)
+      P.flags[hq] = (uint8_t)((apply ? 1 : 0) | (rho < a.theta1 ? 2 : 0) | (a.n_cal <= 64 ? (cs << 2) : 0));
+  }
+}
+
 __global__ void __launch_bounds__(kThreads, 2) decode_kernel(const __grid_constant__ DecodeArgs a) {
   extern __shared__ __align__(128) unsigned char smem[];
   __shared__ unsigned long long s_best[kMaxG];  // best (similarity, row) of this CTA's calibration rows
 
   cg::cluster_group cluster = cg::this_cluster();
-  const int split = blockIdx.x, unit = blockIdx.y, layer = blockIdx.z;  // cluster rank == split
+  const int gs = blockIdx.x;             // split index over the whole unit
+  const int split = gs % a.nsplit;       // rank inside the cluster
+  const int clu = gs / a.nsplit;         // cluster of this unit
+  const int n_gs = a.nsplit * a.nclu;
+  const int unit = blockIdx.y, layer = blockIdx.z;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int gq = lane >> 2, tq = lane & 3;  // MMA fragment coordinates
   const DecodeLayerPtrs& P = a.layer[layer];
@@ -101,7 +135,7 @@ __global__ void __launch_bounds__(kThreads, 2) decode_kernel(const __grid_consta
   const unsigned char* k_new = (const unsigned char*)P.k_new + (size_t)unit * kRowBytes;
   const unsigned char* v_new = (const unsigned char*)P.v_new + (size_t)unit * kRowBytes;
 
-  const int r0 = split * a.rows_per_split;
+  const int r0 = min(a.n_kv, gs * a.rows_per_split);
   const int r1 = min(a.n_kv, r0 + a.rows_per_split);
   const int nblk = r1 > r0 ? (r1 - r0 + kBlkRows - 1) / kBlkRows : 0;
   const int my_blocks = nblk > warp ? (nblk - warp + kWarps - 1) / kWarps : 0;
@@ -125,8 +159,8 @@ __global__ void __launch_bounds__(kThreads, 2) decode_kernel(const __grid_consta
     }
   }
   // calibration rows of this CTA: the contiguous range [c_begin, c_begin + n_c)
-  const int c_per = (a.n_cal + a.nsplit - 1) / a.nsplit;
-  const int c_begin = min(a.n_cal, split * c_per);
+  const int c_per = (a.n_cal + n_gs - 1) / n_gs;
+  const int c_begin = min(a.n_cal, gs * c_per);
   const int n_c = min(a.n_cal, c_begin + c_per) - c_begin;
   if (tid >= 32 && tid < 32 + a.G && n_c > 0) {  // same for the small operands of the similarity
     const int g = tid - 32;
@@ -333,7 +367,8 @@ __global__ void __launch_bounds__(kThreads, 2) decode_kernel(const __grid_consta
   // ---- (7) finish.  This CTA owns 128 / nsplit output dimensions of every head of the group.
   const int dpc = kD / a.nsplit;
   const int n_items = a.G * dpc;
-  // Two items per thread at most would need nsplit >= G / ... ; in general loop over the items.
+  const bool single = a.nclu == 1;
+  const int lu = layer * a.units + unit;
   for (int item0 = 0; item0 < n_items; item0 += kThreads) {
     const int item = item0 + tid;
     const bool act = item < n_items;
@@ -348,11 +383,9 @@ __global__ void __launch_bounds__(kThreads, 2) decode_kernel(const __grid_consta
         best = k > best ? k : best;
       }
     }
-    const int cs = (int)(unsigned)(best & 0xffffffffull);
-    const float rho = rank_key_value(best);
-    const size_t crow = (size_t)hq * a.n_cal + cs;
     float lse_c = 0.f, oc = 0.f;
-    if (act) {  // in flight while the partials are exchanged
+    if (act && single) {  // in flight while the partials are exchanged
+      const size_t crow = (size_t)hq * a.n_cal + (unsigned)(best & 0xffffffffull);
       lse_c = __ldg(P.LSE_c + crow);
       oc = __ldg(P.O_c + crow * kD + d);
     }
@@ -377,28 +410,65 @@ __global__ void __launch_bounds__(kThreads, 2) decode_kernel(const __grid_consta
       Lsum = fmaf(ls[s], sc, Lsum);
       acc = fmaf(os[s], sc, acc);
     }
-    float outv = acc / Lsum;             // O_a
-    float lse2 = M + log2f(Lsum);        // LSE_a (log2 domain)
-    const bool apply = (a.always_apply || rho > a.theta2) && (lse_c > -INFINITY);
-    if (apply) {
-      // alpha_i = e^{LSE_a - LSE}, alpha_j = e^{LSE_c - LSE}; out = alpha_i O_a + alpha_j O_c (Eq. 1-2)
-      const float lc2 = lse_c * kLog2e;
-      const float mx = fmaxf(lse2, lc2);
-      const float ea = exp2f(lse2 - mx), ec = exp2f(lc2 - mx);
-      const float tot = ea + ec;
-      outv = (ea / tot) * outv + (ec / tot) * oc;
-      lse2 = mx + log2f(tot);
-    }
-    if (act) {
-      reinterpret_cast<__nv_bfloat16*>(P.out)[(size_t)hq * kD + d] = __float2bfloat16_rn(outv);
+    if (single) {
+      if (act) merge_store(a, P, hq, d, acc, M, Lsum, best, lse_c, oc);
+    } else if (act) {
+      // this cluster's partial goes to the workspace; (M, Lsum, best) are the same in all its CTAs
+      const size_t pc = ((size_t)lu * a.nclu + clu) * kMaxG + g;
+      a.part_o[pc * kD + d] = acc;
       if (d == 0) {
-        if (P.lse_out) P.lse_out[hq] = lse2 * kLn2;
-        if (P.flags)
-          P.flags[hq] = (uint8_t)((apply ? 1 : 0) | (rho < a.theta1 ? 2 : 0) | (a.n_cal <= 64 ? (cs << 2) : 0));
+        a.part_ml[pc * 2] = M;
+        a.part_ml[pc * 2 + 1] = Lsum;
+        a.part_best[pc] = best;
       }
     }
   }
   cluster_arrive();  // (C) no CTA leaves while another may still read its shared memory
+  if (!single) {
+    // ---- (8) several clusters per unit: the CTA that takes the unit's last ticket merges them
+    __shared__ unsigned s_ticket;
+    __threadfence();
+    __syncthreads();
+    if (tid == 0) s_ticket = atomicAdd(&a.counters[lu], 1u);
+    __syncthreads();
+    if (s_ticket == (unsigned)(n_gs - 1)) {
+      __threadfence();
+      const int d = tid;  // one output dimension per thread
+      for (int g = 0; g < a.G; ++g) {
+        const size_t pu = (size_t)lu * a.nclu * kMaxG + g;
+        unsigned long long best = 0ull;
+        float ms[8], ls[8], os[8];
+#pragma unroll
+        for (int c = 0; c < 8; ++c) {
+          ms[c] = -INFINITY; ls[c] = 0.f; os[c] = 0.f;
+          if (c < a.nclu) {
+            const size_t pc = pu + (size_t)c * kMaxG;
+            const unsigned long long k = __ldcg(a.part_best + pc);
+            best = k > best ? k : best;
+            const float2 ml2 = __ldcg(reinterpret_cast<const float2*>(a.part_ml + pc * 2));
+            ms[c] = ml2.x; ls[c] = ml2.y;
+            os[c] = __ldcg(a.part_o + pc * kD + d);
+          }
+        }
+        const int hq = hq0 + g;
+        const size_t crow = (size_t)hq * a.n_cal + (unsigned)(best & 0xffffffffull);
+        const float lse_c = __ldg(P.LSE_c + crow);
+        const float oc = __ldg(P.O_c + crow * kD + d);
+        float M = -INFINITY;
+#pragma unroll
+        for (int c = 0; c < 8; ++c) M = fmaxf(M, ms[c]);
+        float Lsum = 0.f, acc = 0.f;
+#pragma unroll
+        for (int c = 0; c < 8; ++c) {
+          const float sc = ms[c] > -INFINITY ? ex2_approx(ms[c] - M) : 0.f;
+          Lsum = fmaf(ls[c], sc, Lsum);
+          acc = fmaf(os[c], sc, acc);
+        }
+        merge_store(a, P, hq, d, acc, M, Lsum, best, lse_c, oc);
+      }
+      if (tid == 0) a.counters[lu] = 0u;  // ready for the next launch on this workspace
+    }
+  }
   cluster_wait();
 }
 
@@ -415,7 +485,7 @@ cudaError_t launch_decode(const DecodeArgs& a, cudaStream_t st) {
     if (dev >= 0 && dev < 64) attr_set[dev] = true;
   }
   cudaLaunchConfig_t cfg{};
-  cfg.gridDim = dim3(a.nsplit, a.units, a.n_layers);
+  cfg.gridDim = dim3(a.nsplit * a.nclu, a.units, a.n_layers);
   cfg.blockDim = dim3(kThreads);
   cfg.dynamicSmemBytes = kSmemBytes;
   cfg.stream = st;

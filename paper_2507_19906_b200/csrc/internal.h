@@ -46,14 +46,16 @@ constexpr int kDecodeTargetCtas = 296;  // two resident CTAs on each of the 148 
 
 struct DecodeArgs {
   int B, Hq, Hkv, G, n_cal, cap, kv_len, n_kv, has_new;
-  int units, n_layers, nsplit, rows_per_split;
+  int units, n_layers, rows_per_split;
+  int nsplit;  // CTAs per cluster (1, 2, 4 or 8): the splits combined through distributed shared memory
+  int nclu;    // clusters per (layer, unit); more than one only when few units share a long cache
   float scale2, theta1, theta2;
   int always_apply;
-  // per-layer workspace arrays (element strides are implied by units / nsplit / n_cal)
-  float* part_o;       // [layer][unit][nsplit][8][128]
-  float* part_ml;      // [layer][unit][nsplit][8][2]
-  float* rho;          // [layer][unit][8][n_cal]
-  unsigned* counters;  // [layer][unit]
+  // workspace arrays, used only when nclu > 1: per-cluster partials and the arrival counters
+  float* part_o;                  // [layer][unit][nclu][8][128]
+  float* part_ml;                 // [layer][unit][nclu][8][2]
+  unsigned long long* part_best;  // [layer][unit][nclu][8] best (similarity, row) keys
+  unsigned* counters;             // [layer][unit]
   DecodeLayerPtrs layer[kDecodeMaxLayers];
 };
 

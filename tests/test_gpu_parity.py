@@ -37,6 +37,8 @@ SMALL = [
     (1, 7, 1, 700, 64, 7, 160, 64),      # 448 window rows per kv head: two row blocks in the vote pass
     (1, 16, 2, 900, 64, 5, 200, 16),     # G = 8, W = 64: 512 window rows, four 128-row statistic blocks
     (1, 4, 1, 3000, 128, 7, 400, 128),   # W = 128: one query head per calibration row block
+    (1, 8, 1, 4000, 16, 7, 2100, 16),    # one unit, long cache: decode runs eight clusters per unit
+    (2, 8, 2, 2500, 16, 7, 1000, 7),     # four units: three clusters per unit, most CTAs without a C_q row
 ]
 
 
