@@ -45,6 +45,14 @@ constexpr int kStageBytes = 2 * kBlkRows * kRowBytes;  // K block then V block
 constexpr int kWarpSmem = kStages * kStageBytes;       // 24 KB
 constexpr int kSmemBytes = kWarps * kWarpSmem;         // 96 KB -> two CTAs per SM
 
+constexpr int kWoStride = kD + 4;  // row stride of the per-warp partial outputs: heads land in distinct banks
+
+__device__ __forceinline__ uint32_t movmatrix_trans(uint32_t x) {
+  uint32_t y;
+  asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(y) : "r"(x));
+  return y;
+}
+
 __device__ __forceinline__ uint32_t swz(int row, int chunk) {
   return (uint32_t)(row * kRowBytes + ((chunk ^ (row & 7)) << 4));
 }
@@ -266,11 +274,16 @@ __global__ void __launch_bounds__(kThreads, 2) decode_kernel(const __grid_consta
   }
   cluster_arrive();  // (A) this CTA's s_best is final
 
-  // ---- (5) main loop
-  float o[kD / 8][4];
+  // ---- (5) main loop.  The products are taken transposed, keys on the 16-row side of the MMA and
+  // the (at most eight) heads on its 8-column side, so that no half of a tile is padding:
+  //   S^T[16 keys x 8 heads]   = K_blk[16 x 128] . Q^T[128 x 8]          (8 MMAs)
+  //   O^T[128 dims x 8 heads] += V_blk^T[128 x 16 keys] . P^T[16 x 8]     (8 MMAs)
+  // A thread holds heads 2tq, 2tq+1 of keys gq, gq+8 (S^T) and of dims 16n+gq, 16n+gq+8 (O^T).
+  float o[kD / 16][4];
 #pragma unroll
-  for (int n = 0; n < kD / 8; ++n) { o[n][0] = o[n][1] = o[n][2] = o[n][3] = 0.f; }
-  float m = -INFINITY, l = 0.f;
+  for (int n = 0; n < kD / 16; ++n) { o[n][0] = o[n][1] = o[n][2] = o[n][3] = 0.f; }
+  float m0 = -INFINITY, m1 = -INFINITY, l0 = 0.f, l1 = 0.f;  // heads 2tq and 2tq+1
+  const int mid = lane >> 3;
 
   for (int i = 0; i < my_blocks; ++i) {
     const int nxt = i + kStages - 1;
@@ -283,66 +296,73 @@ __global__ void __launch_bounds__(kThreads, 2) decode_kernel(const __grid_consta
     const uint32_t sV = sK + kBlkRows * kRowBytes;
     const int row_base = r0 + (warp + i * kWarps) * kBlkRows;
 
-    // S = Q K^T for 16 keys: two n8 tiles
-    float s0[4] = {0.f, 0.f, 0.f, 0.f}, s1[4] = {0.f, 0.f, 0.f, 0.f};
+    // S^T: two accumulators (even and odd k-steps) halve the dependent chain
+    float sa[4] = {0.f, 0.f, 0.f, 0.f}, sb[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
     for (int kk = 0; kk < kD / 16; ++kk) {
-      const int mid = lane >> 3;
-      const int row = (lane & 7) + (mid >> 1) * 8;
-      const int chunk = kk * 2 + (mid & 1);
-      uint32_t b0, b1, b2, b3;
-      ldmatrix_x4(sK + swz(row, chunk), b0, b1, b2, b3);
-      mma_bf16_16816(s0, qa[kk][0], 0u, qa[kk][1], 0u, b0, b1);
-      mma_bf16_16816(s1, qa[kk][0], 0u, qa[kk][1], 0u, b2, b3);
+      uint32_t a0, a1, a2, a3;
+      ldmatrix_x4(sK + swz((lane & 7) + (mid & 1) * 8, kk * 2 + (mid >> 1)), a0, a1, a2, a3);
+      if (kk & 1) mma_bf16_16816(sb, a0, a1, a2, a3, qa[kk][0], qa[kk][1]);
+      else mma_bf16_16816(sa, a0, a1, a2, a3, qa[kk][0], qa[kk][1]);
     }
-    // online softmax on row gq (keys 2tq, 2tq+1, 8+2tq, 9+2tq of this block)
-    const int kb = row_base + 2 * tq;
-    float x0 = kb < r1 ? s0[0] * a.scale2 : -INFINITY;
-    float x1 = kb + 1 < r1 ? s0[1] * a.scale2 : -INFINITY;
-    float x2 = kb + 8 < r1 ? s1[0] * a.scale2 : -INFINITY;
-    float x3 = kb + 9 < r1 ? s1[1] * a.scale2 : -INFINITY;
-    float bm = fmaxf(fmaxf(x0, x1), fmaxf(x2, x3));
-    bm = fmaxf(bm, __shfl_xor_sync(0xffffffffu, bm, 1));
-    bm = fmaxf(bm, __shfl_xor_sync(0xffffffffu, bm, 2));
-    const float m_new = fmaxf(m, bm);  // finite: every processed block has a valid first row
-    const float corr = ex2_approx(m - m_new);
-    const float p0 = ex2_approx(x0 - m_new), p1 = ex2_approx(x1 - m_new);
-    const float p2 = ex2_approx(x2 - m_new), p3 = ex2_approx(x3 - m_new);
-    l = l * corr + (p0 + p1) + (p2 + p3);
-    m = m_new;
+    // online softmax per head over the 16 keys of the block (keys gq and gq + 8 live here)
+    const bool v0 = row_base + gq < r1, v1 = row_base + gq + 8 < r1;
+    const float x00 = v0 ? (sa[0] + sb[0]) * a.scale2 : -INFINITY;
+    const float x01 = v0 ? (sa[1] + sb[1]) * a.scale2 : -INFINITY;
+    const float x10 = v1 ? (sa[2] + sb[2]) * a.scale2 : -INFINITY;
+    const float x11 = v1 ? (sa[3] + sb[3]) * a.scale2 : -INFINITY;
+    float bm0 = fmaxf(x00, x10), bm1 = fmaxf(x01, x11);
 #pragma unroll
-    for (int n = 0; n < kD / 8; ++n) { o[n][0] *= corr; o[n][1] *= corr; }
-    const uint32_t pa0 = pack_bf16(p0, p1), pa2 = pack_bf16(p2, p3);
-    // O += P V
+    for (int off = 4; off < 32; off <<= 1) {
+      bm0 = fmaxf(bm0, __shfl_xor_sync(0xffffffffu, bm0, off));
+      bm1 = fmaxf(bm1, __shfl_xor_sync(0xffffffffu, bm1, off));
+    }
+    const float mn0 = fmaxf(m0, bm0), mn1 = fmaxf(m1, bm1);  // finite: the block's first key is valid
+    const float corr0 = ex2_approx(m0 - mn0), corr1 = ex2_approx(m1 - mn1);
+    const float p00 = ex2_approx(x00 - mn0), p01 = ex2_approx(x01 - mn1);
+    const float p10 = ex2_approx(x10 - mn0), p11 = ex2_approx(x11 - mn1);
+    l0 = l0 * corr0 + (p00 + p10);  // partial over this thread's keys, summed over gq at the end
+    l1 = l1 * corr1 + (p01 + p11);
+    m0 = mn0; m1 = mn1;
 #pragma unroll
-    for (int n = 0; n < kD / 8; n += 2) {
-      const int mid = lane >> 3;
-      const int row = (lane & 7) + (mid & 1) * 8;
-      const int chunk = n + (mid >> 1);
-      uint32_t b0, b1, b2, b3;
-      ldmatrix_x4_trans(sV + swz(row, chunk), b0, b1, b2, b3);
-      mma_bf16_16816(o[n], pa0, 0u, pa2, 0u, b0, b1);
-      mma_bf16_16816(o[n + 1], pa0, 0u, pa2, 0u, b2, b3);
+    for (int n = 0; n < kD / 16; ++n) { o[n][0] *= corr0; o[n][1] *= corr1; o[n][2] *= corr0; o[n][3] *= corr1; }
+    // P^T as the B operand: transpose the two 8x8 (key, head) fragments inside the warp
+    const uint32_t pb0 = movmatrix_trans(pack_bf16(p00, p01)), pb1 = movmatrix_trans(pack_bf16(p10, p11));
+#pragma unroll
+    for (int n = 0; n < kD / 16; ++n) {
+      uint32_t a0, a1, a2, a3;
+      ldmatrix_x4_trans(sV + swz((lane & 7) + (mid >> 1) * 8, n * 2 + (mid & 1)), a0, a1, a2, a3);
+      mma_bf16_16816(o[n], a0, a1, a2, a3, pb0, pb1);
     }
     __syncwarp();  // the stage is refilled by the next iteration's cp.async
   }
   cp_async_wait<0>();
-  l += __shfl_xor_sync(0xffffffffu, l, 1);
-  l += __shfl_xor_sync(0xffffffffu, l, 2);
+#pragma unroll
+  for (int off = 4; off < 32; off <<= 1) {
+    l0 += __shfl_xor_sync(0xffffffffu, l0, off);
+    l1 += __shfl_xor_sync(0xffffffffu, l1, off);
+  }
   __syncthreads();  // all warps are done with their stages: reuse them for the combine
 
   // ---- (6) CTA combine of the four warps into this split's partial: xo[g][d], xml[g] = (m, l)
-  float* wo = reinterpret_cast<float*>(smem);             // [warp][8][128]
-  float* wml = wo + kWarps * kMaxG * kD;                   // [warp][8][2]
+  float* wo = reinterpret_cast<float*>(smem);             // [warp][8][kWoStride]
+  float* wml = wo + kWarps * kMaxG * kWoStride;            // [warp][8][2]
   float* xo = wml + kWarps * kMaxG * 2;                    // [8][128]
   float* xml = xo + kMaxG * kD;                            // [8][2]
+  if (2 * tq < a.G) {
 #pragma unroll
-  for (int n = 0; n < kD / 8; ++n)
-    *reinterpret_cast<float2*>(wo + ((warp * kMaxG + gq) * kD + n * 8 + 2 * tq)) = make_float2(o[n][0], o[n][1]);
-  if (tq == 0) { wml[(warp * kMaxG + gq) * 2] = m; wml[(warp * kMaxG + gq) * 2 + 1] = l; }
+    for (int n = 0; n < kD / 16; ++n) {
+      float* w0 = wo + (warp * kMaxG + 2 * tq) * kWoStride + n * 16 + gq;
+      w0[0] = o[n][0]; w0[8] = o[n][2];
+      w0[kWoStride] = o[n][1]; w0[kWoStride + 8] = o[n][3];
+    }
+    if (gq == 0) {
+      wml[(warp * kMaxG + 2 * tq) * 2] = m0; wml[(warp * kMaxG + 2 * tq) * 2 + 1] = l0;
+      wml[(warp * kMaxG + 2 * tq + 1) * 2] = m1; wml[(warp * kMaxG + 2 * tq + 1) * 2 + 1] = l1;
+    }
+  }
   __syncthreads();
-  {
-    const int d = tid;  // one output dimension per thread
+  for (int d = tid; d < kD; d += kThreads) {
 #pragma unroll
     for (int g = 0; g < kMaxG; ++g) {
       if (g >= a.G) break;
@@ -355,7 +375,7 @@ __global__ void __launch_bounds__(kThreads, 2) decode_kernel(const __grid_consta
         const float mw = wml[(w * kMaxG + g) * 2];
         const float sc = mw > -INFINITY ? ex2_approx(mw - M) : 0.f;
         Lsum += wml[(w * kMaxG + g) * 2 + 1] * sc;
-        acc += wo[(w * kMaxG + g) * kD + d] * sc;
+        acc += wo[(w * kMaxG + g) * kWoStride + d] * sc;
       }
       xo[g * kD + d] = acc;
       if (d == 0) { xml[g * 2] = M; xml[g * 2 + 1] = Lsum; }
@@ -433,8 +453,8 @@ __global__ void __launch_bounds__(kThreads, 2) decode_kernel(const __grid_consta
     __syncthreads();
     if (s_ticket == (unsigned)(n_gs - 1)) {
       __threadfence();
-      const int d = tid;  // one output dimension per thread
-      for (int g = 0; g < a.G; ++g) {
+      for (int gd = tid; gd < a.G * kD; gd += kThreads) {
+        const int g = gd / kD, d = gd % kD;
         const size_t pu = (size_t)lu * a.nclu * kMaxG + g;
         unsigned long long best = 0ull;
         float ms[8], ls[8], os[8];
