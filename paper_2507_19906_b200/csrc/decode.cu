@@ -37,13 +37,13 @@ namespace {
 
 namespace cg = cooperative_groups;
 
-constexpr int kWarps = 4;
+constexpr int kWarps = 8;
 constexpr int kThreads = kWarps * 32;
 constexpr int kBlkRows = 16;                           // rows per pipeline stage of one warp
 constexpr int kStages = 3;
 constexpr int kStageBytes = 2 * kBlkRows * kRowBytes;  // K block then V block
 constexpr int kWarpSmem = kStages * kStageBytes;       // 24 KB
-constexpr int kSmemBytes = kWarps * kWarpSmem;         // 96 KB -> two CTAs per SM
+constexpr int kSmemBytes = kWarps * kWarpSmem;         // 192 KB -> one CTA per SM
 
 constexpr int kWoStride = kD + 4;  // row stride of the per-warp partial outputs: heads land in distinct banks
 
@@ -120,7 +120,7 @@ __device__ __forceinline__ void merge_store(const DecodeArgs& a, const DecodeLay
   }
 }
 
-__global__ void __launch_bounds__(kThreads, 2) decode_kernel(const __grid_constant__ DecodeArgs a) {
+__global__ void __launch_bounds__(kThreads, 1) decode_kernel(const __grid_constant__ DecodeArgs a) {
   extern __shared__ __align__(128) unsigned char smem[];
   __shared__ unsigned long long s_best[kMaxG];  // best (similarity, row) of this CTA's calibration rows
 

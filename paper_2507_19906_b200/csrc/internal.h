@@ -42,7 +42,7 @@ struct DecodeLayerPtrs {
 
 constexpr int kDecodeMaxLayers = 32;
 constexpr int kDecodeMaxSplit = 64;
-constexpr int kDecodeTargetCtas = 296;  // two resident CTAs on each of the 148 SMs
+constexpr int kDecodeTargetCtas = 148;  // one resident CTA on each of the 148 SMs
 
 struct DecodeArgs {
   int B, Hq, Hkv, G, n_cal, cap, kv_len, n_kv, has_new;
