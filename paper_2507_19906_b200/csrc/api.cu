@@ -128,7 +128,7 @@ int decode_nsplit(int units_total, int n_kv) {
 }
 
 struct DecodeWs {
-  size_t part_o, part_ml, rho, counters, per_layer;
+  size_t part_o, part_ml, rho, counters, status, per_layer;
   int max_split;
 };
 
@@ -138,6 +138,7 @@ DecodeWs make_decode_ws(const calidrop_params* p) {
   w.max_split = decode_nsplit(units, 1 << 30);
   size_t off = 0;
   w.counters = off; off = align_up(off + (size_t)units * 4 * kDecodeMaxLayers, 256);
+  w.status = off;   off += 256;  // error word: nonzero after a bounded wait of the kernel ran out
   w.part_ml = off;  off = align_up(off + (size_t)units * w.max_split * kMaxG * 2 * 4, 256);
   w.rho = off;      off = align_up(off + (size_t)units * kMaxG * w.max_split * 8, 256);
   w.part_o = off;   off = align_up(off + (size_t)units * w.max_split * kMaxG * kD * 4, 256);
@@ -272,7 +273,7 @@ int calidrop_decode_batched(const calidrop_params* p, int32_t n_layers, const ca
   if (workspace_bytes < w.per_layer * (size_t)n_layers) return CALIDROP_WORKSPACE_TOO_SMALL;
   if (!device_supported()) return CALIDROP_UNSUPPORTED;
 
-  DecodeArgs a{};
+  DecodeCommon a{};
   a.B = p->B; a.Hq = p->Hq; a.Hkv = p->Hkv; a.G = p->Hq / p->Hkv; a.n_cal = p->n_cal; a.cap = p->cap;
   a.kv_len = kv_len; a.n_kv = n_kv; a.has_new = has_new ? 1 : 0;
   a.units = p->B * p->Hkv; a.n_layers = n_layers;
@@ -293,15 +294,30 @@ int calidrop_decode_batched(const calidrop_params* p, int32_t n_layers, const ca
   const size_t nl = (size_t)n_layers;
   size_t off = 0;
   a.counters = (unsigned*)(base + off); off += align_up((size_t)a.units * 4 * kDecodeMaxLayers, 256);
+  a.status = (unsigned*)(base + off);   off += 256;
   a.part_ml = (float*)(base + off);     off += align_up((size_t)a.units * a.nclu * kMaxG * 2 * 4 * nl, 256);
   a.part_best = (unsigned long long*)(base + off); off += align_up((size_t)a.units * a.nclu * kMaxG * 8 * nl, 256);
   a.part_o = (float*)(base + off);
-  for (int i = 0; i < n_layers; ++i) {
-    const calidrop_decode_layer& L = layers[i];
-    a.layer[i] = DecodeLayerPtrs{L.q, L.k_new, L.v_new, L.K_kept, L.V_kept, L.O_c, L.LSE_c, L.C_q,
-                                 L.out, L.lse_out, L.flags};
+  cudaError_t e;
+  if (n_layers == 1) {
+    DecodeArgsT<1> args{};
+    args.c = a;
+    const calidrop_decode_layer& L = layers[0];
+    args.layer[0] = DecodeLayerPtrs{L.q, L.k_new, L.v_new, L.K_kept, L.V_kept, L.O_c, L.LSE_c, L.C_q,
+                                    L.out, L.lse_out, L.flags};
+    if (!make_decode_maps(a, args.layer[0], &args.maps[0])) return CALIDROP_CUDA_ERROR;
+    e = launch_decode(args, (cudaStream_t)stream);
+  } else {
+    static thread_local DecodeArgsT<kDecodeMaxLayers> args;
+    args.c = a;
+    for (int i = 0; i < n_layers; ++i) {
+      const calidrop_decode_layer& L = layers[i];
+      args.layer[i] = DecodeLayerPtrs{L.q, L.k_new, L.v_new, L.K_kept, L.V_kept, L.O_c, L.LSE_c, L.C_q,
+                                      L.out, L.lse_out, L.flags};
+      if (!make_decode_maps(a, args.layer[i], &args.maps[i])) return CALIDROP_CUDA_ERROR;
+    }
+    e = launch_decode(args, (cudaStream_t)stream);
   }
-  cudaError_t e = launch_decode(a, (cudaStream_t)stream);
   return e == cudaSuccess ? CALIDROP_OK : cuda_fail(e);
 }
 

@@ -4,32 +4,38 @@
 // retained rows with the G query heads of a kv group packed into one MMA tile (so every K/V
 // byte is read once for all of them), the cosine similarity of the query with the stored
 // calibration queries, the threshold gate, and the merge of Eq. 1-2.  The work is bound by
-// HBM traffic (about 2G flop per byte), so the contraction uses the warp-level mma.sync path
-// with G <= 8 rows of a 16-row tile; tcgen05 tiles (64 rows minimum) would add nothing here.
+// HBM traffic (about 2G flop per byte), so the contraction uses the warp-level mma.sync path;
+// what matters is how the bytes get to the SM and how short the chain after the last byte is.
 //
 // Grid: (split, batch*kv-head, layer); the splits of one (unit, layer) form thread-block
-// clusters of 1, 2, 4 or 8 CTAs.  Each CTA streams its slice of rows through shared memory with
-// 16-byte cp.async copies (XOR-swizzled so ldmatrix is conflict-free), four warps each running
-// an independent online softmax over interleaved 16-row blocks.  The splits are combined inside
-// the cluster through distributed shared memory: every CTA finishes a slice of the 128 output
-// dimensions for all heads of the group, so there is no global-memory round trip, no ticket and
-// no CTA that works alone at the end.  Only when very few units share a long cache (fewer than
-// 19 units per launch) does one cluster per unit leave most SMs idle; then a unit gets up to
-// eight clusters, each writes its combined partial, its (max, sum) pair and its best similarity
-// to the workspace, and the CTA that takes the last ticket of the unit's arrival counter merges
-// them and resets the counter.
+// clusters of 1, 2, 4 or 8 CTAs.  A CTA has one producer warp and eight stream warps.  The
+// producer moves the CTA's slice of K and V through a ring of three 64-row slots with TMA
+// (128-byte swizzle, so ldmatrix is conflict-free and no load instruction per 16 bytes is
+// spent on the stream); each slot is consumed by four stream warps, 16 rows each, with their
+// own online softmax.  The products are taken transposed, keys on the 16-row side of the MMA and
+// the (at most eight) heads on its 8-column side, so that no half of a tile is padding:
+//   S^T[16 keys x 8 heads]   = K_blk[16 x 128] . Q^T[128 x 8]          (8 MMAs)
+//   O^T[128 dims x 8 heads] += V_blk^T[128 x 16 keys] . P^T[16 x 8]     (8 MMAs)
+// The splits are combined inside the cluster through distributed shared memory: every CTA
+// finishes a slice of the 128 output dimensions for all heads of the group, and each CTA pushes
+// its partial of a slice into the shared memory of the slice's owner, so that after one cluster
+// barrier every CTA reduces local data only.  Only when very few units share a long cache does
+// one cluster per unit leave most SMs idle; then a unit gets up to eight clusters, each writes
+// its combined partial, its (max, sum) pair and its best similarity to the workspace, and the
+// CTA that takes the last ticket of the unit's arrival counter merges them and resets the counter.
 //
 // A launch moves only tens of MB, so its latency chain matters as much as its bandwidth:
 //   * the launch carries the programmatic-serialisation attribute and the kernel prefetches its
-//     K/V slice into L2 before the dependency wait, so the HBM reads of one decode call overlap
-//     the tail of whatever runs ahead of it in the stream;
-//   * the K/V copies are issued first, the similarity work (which needs only q and C_q) runs while
-//     they are in flight, and the cluster exchanges each CTA's best (similarity, row) pair early,
-//     so the chosen O_c row is already being fetched while the partial outputs are combined.
+//     K/V slice into L2 before the dependency wait; a CTA takes less than half an SM, so the
+//     CTAs of the next decode call are resident, and prefetching, while this one finishes;
+//   * the similarity work (which needs only q and C_q) runs while the first slots are in flight,
+//     and the cluster exchanges each CTA's best (similarity, row) pair early, so the chosen O_c
+//     row is already being fetched while the partial outputs are combined.
 #include <cooperative_groups.h>
 
 #include "common.cuh"
 #include "internal.h"
+#include "tc_common.cuh"
 
 namespace calidrop {
 
@@ -37,15 +43,23 @@ namespace {
 
 namespace cg = cooperative_groups;
 
-constexpr int kWarps = 8;
-constexpr int kThreads = kWarps * 32;
-constexpr int kBlkRows = 16;                           // rows per pipeline stage of one warp
-constexpr int kStages = 3;
-constexpr int kStageBytes = 2 * kBlkRows * kRowBytes;  // K block then V block
-constexpr int kWarpSmem = kStages * kStageBytes;       // 24 KB
-constexpr int kSmemBytes = kWarps * kWarpSmem;         // 192 KB -> one CTA per SM
-
+constexpr int kStreamWarps = 8;
+constexpr int kThreads = (kStreamWarps + 1) * 32;  // the last warp is the producer
+constexpr int kBlkRows = 16;                        // rows of one warp's MMA block
+constexpr int kSlotRows = 64;                       // rows per ring slot: four blocks
+constexpr int kSlots = 6;
+constexpr int kPlaneBytes = kSlotRows * 128;        // 64 rows x 64 columns of bf16 (one TMA box)
+constexpr int kSlotBytes = 4 * kPlaneBytes;         // K low / K high / V low / V high column halves
+constexpr int kRingBytes = kSlots * kSlotBytes;     // 192 KB -> one CTA per SM
+constexpr int kSmemBytes = kRingBytes + 1024;       // + slack for the 1024-byte alignment
 constexpr int kWoStride = kD + 4;  // row stride of the per-warp partial outputs: heads land in distinct banks
+constexpr long long kWaitLimitCycles = 2000000000ll;  // about a second: a wait this long has failed
+
+// Byte offset of 16-byte chunk `chunk` (0..15) of row `row` (0..63) inside the K or V part of a
+// slot: two column halves, each a [64 rows][128 bytes] plane in the 128-byte swizzle TMA writes.
+__device__ __forceinline__ uint32_t plane_off(int row, int chunk) {
+  return (uint32_t)((chunk >> 3) * kPlaneBytes + row * 128 + (((chunk & 7) ^ (row & 7)) << 4));
+}
 
 __device__ __forceinline__ uint32_t movmatrix_trans(uint32_t x) {
   uint32_t y;
@@ -53,8 +67,57 @@ __device__ __forceinline__ uint32_t movmatrix_trans(uint32_t x) {
   return y;
 }
 
-__device__ __forceinline__ uint32_t swz(int row, int chunk) {
-  return (uint32_t)(row * kRowBytes + ((chunk ^ (row & 7)) << 4));
+// ---- mbarrier / TMA helpers (no cluster multicast anywhere: every copy lands in this CTA)
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n"
+      ".reg .pred p;\n"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+      "selp.u32 %0, 1, 0, p;\n"
+      "}\n"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// Bounded wait: when it runs out the CTA's abort flag is raised, the workspace's error word is
+// set and every later wait of the CTA returns at once; the CTA still walks through all its
+// barriers, so nothing hangs, but its output is not valid.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                          unsigned* status, unsigned code) {
+  if (mbar_try_wait(bar, parity)) return true;
+  long long t0 = 0;
+  unsigned polls = 0;
+  while (!mbar_try_wait(bar, parity)) {
+    if ((++polls & 255u) == 0u) {
+      if (*abort_flag) return false;
+      const long long now = clock64();
+      if (t0 == 0) t0 = now;
+      if (now - t0 > kWaitLimitCycles) {
+        *abort_flag = 1;
+        atomicCAS(status, 0u, code);
+        return false;
+      }
+    }
+  }
+  return true;
+}
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1,
+                                            int c2) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+      ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2)
+      : "memory");
 }
 
 struct RhoLoad {
@@ -96,7 +159,7 @@ __device__ __forceinline__ void cluster_wait() {
 
 // Gate and merge of one output element (Eq. 1-2): (acc, M, Lsum) is the unnormalised partial of
 // the retained cache in the log2 domain, best the chosen (similarity, calibration row) key.
-__device__ __forceinline__ void merge_store(const DecodeArgs& a, const DecodeLayerPtrs& P, int hq, int d, float acc,
+__device__ __forceinline__ void merge_store(const DecodeCommon& a, const DecodeLayerPtrs& P, int hq, int d, float acc,
                                             float M, float Lsum, unsigned long long best, float lse_c, float oc) {
   const int cs = (int)(unsigned)(best & 0xffffffffull);
   const float rho = rank_key_value(best);
@@ -120,10 +183,18 @@ __device__ __forceinline__ void merge_store(const DecodeArgs& a, const DecodeLay
   }
 }
 
-__global__ void __launch_bounds__(kThreads, 1) decode_kernel(const __grid_constant__ DecodeArgs a) {
-  extern __shared__ __align__(128) unsigned char smem[];
-  __shared__ unsigned long long s_best[kMaxG];  // best (similarity, row) of this CTA's calibration rows
+template <int NL>
+__global__ void __launch_bounds__(kThreads, 1) decode_kernel(const __grid_constant__ DecodeArgsT<NL> args) {
+  extern __shared__ unsigned char smem_raw[];
+  __shared__ __align__(8) unsigned long long s_full[kSlots][2], s_empty[kSlots][2];
+  __shared__ unsigned long long s_best[kMaxG];     // best (similarity, row) of this CTA's calibration rows
+  __shared__ unsigned long long s_bestall[kMaxG];  // ... of the whole cluster
+  __shared__ float s_xpart[kMaxG * kD];            // [source split][head][dim of this CTA's slice]
+  __shared__ float s_xml[8][kMaxG][2];             // [source split][head] (max, sum)
+  __shared__ int s_abort;
+  __shared__ unsigned s_ticket;
 
+  const DecodeCommon& a = args.c;
   cg::cluster_group cluster = cg::this_cluster();
   const int gs = blockIdx.x;             // split index over the whole unit
   const int split = gs % a.nsplit;       // rank inside the cluster
@@ -132,7 +203,8 @@ __global__ void __launch_bounds__(kThreads, 1) decode_kernel(const __grid_consta
   const int unit = blockIdx.y, layer = blockIdx.z;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int gq = lane >> 2, tq = lane & 3;  // MMA fragment coordinates
-  const DecodeLayerPtrs& P = a.layer[layer];
+  const DecodeLayerPtrs& P = args.layer[layer];
+  const DecodeLayerMaps& TM = args.maps[layer];
   const int b = unit / a.Hkv, h = unit % a.Hkv;
   const int hq0 = b * a.Hq + h * a.G;  // first query head of this kv group
 
@@ -140,23 +212,34 @@ __global__ void __launch_bounds__(kThreads, 1) decode_kernel(const __grid_consta
   const __nv_bfloat16* Cq = (const __nv_bfloat16*)P.C_q;
   const unsigned char* Kc = (const unsigned char*)P.K + (size_t)unit * a.cap * kRowBytes;
   const unsigned char* Vc = (const unsigned char*)P.V + (size_t)unit * a.cap * kRowBytes;
-  const unsigned char* k_new = (const unsigned char*)P.k_new + (size_t)unit * kRowBytes;
-  const unsigned char* v_new = (const unsigned char*)P.v_new + (size_t)unit * kRowBytes;
 
   const int r0 = min(a.n_kv, gs * a.rows_per_split);
   const int r1 = min(a.n_kv, r0 + a.rows_per_split);
-  const int nblk = r1 > r0 ? (r1 - r0 + kBlkRows - 1) / kBlkRows : 0;
-  const int my_blocks = nblk > warp ? (nblk - warp + kWarps - 1) / kWarps : 0;
+  const int n_sb = (r1 - r0 + kSlotRows - 1) / kSlotRows;  // ring fills of this CTA
 
-  unsigned char* wsm = smem + warp * kWarpSmem;
-  const uint32_t wsm_u32 = smem_u32(wsm);
+  const uint32_t ring = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  unsigned char* ring_ptr = smem_raw + (ring - smem_u32(smem_raw));
+  volatile int* abort_flag = &s_abort;
 
   // ---- (0) overlap with the kernel ahead of this one in the stream.  Until the dependency wait
-  // nothing the predecessor may have written is read and nothing is written; the only early work
-  // is an L2 prefetch of this CTA's slice of the retained cache, which cannot observe stale data
-  // (L2 is the point of coherence) and turns the later cp.async stream into L2 hits.
+  // nothing the predecessor may have written is read and nothing global is written; the only
+  // early global work is an L2 prefetch of this CTA's slice of the retained cache, which cannot
+  // observe stale data (L2 is the point of coherence) and turns the later TMA stream into L2 hits.
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  // calibration rows of this CTA: the contiguous range [c_begin, c_begin + n_c)
+  const int c_per = (a.n_cal + n_gs - 1) / n_gs;
+  const int c_begin = min(a.n_cal, gs * c_per);
+  const int n_c = min(a.n_cal, c_begin + c_per) - c_begin;
   if (tid == 0) {
+    for (int s = 0; s < kSlots; ++s)
+      for (int p = 0; p < 2; ++p) {
+        mbar_init(smem_u32(&s_full[s][p]), 1);    // the producer's arrive with the byte count
+        mbar_init(smem_u32(&s_empty[s][p]), 4);   // one lane of each of the slot's four warps
+      }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    s_abort = 0;
+  }
+  if (warp == kStreamWarps && lane == 0) {
     const int n_old = min(r1, a.kv_len) - r0;  // rows already in the cache (the appended row is not)
     if (n_old > 0) {
       const unsigned bytes = (unsigned)n_old * kRowBytes;
@@ -165,11 +248,11 @@ __global__ void __launch_bounds__(kThreads, 1) decode_kernel(const __grid_consta
       asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(Vc + (size_t)r0 * kRowBytes), "r"(bytes)
                    : "memory");
     }
+    asm volatile("prefetch.tensormap [%0];" ::"l"(&TM.k64) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(&TM.v64) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(&TM.k16) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(&TM.v16) : "memory");
   }
-  // calibration rows of this CTA: the contiguous range [c_begin, c_begin + n_c)
-  const int c_per = (a.n_cal + n_gs - 1) / n_gs;
-  const int c_begin = min(a.n_cal, gs * c_per);
-  const int n_c = min(a.n_cal, c_begin + c_per) - c_begin;
   if (tid >= 32 && tid < 32 + a.G && n_c > 0) {  // same for the small operands of the similarity
     const int g = tid - 32;
     asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(Cq + ((size_t)(hq0 + g) * a.n_cal + c_begin) * kD),
@@ -184,18 +267,51 @@ __global__ void __launch_bounds__(kThreads, 1) decode_kernel(const __grid_consta
   asm volatile("griddepcontrol.wait;" ::: "memory");
   __syncthreads();
 
-  // ---- (1) loads of the similarity operands go out ahead of the K/V burst so that they are not
-  // queued behind it: four lanes per (head, calibration row) pair, 32 pairs per pass, the first
-  // two passes in flight at once
+  // One ring fill: rows [r0 + sb * 64, ...) of K and V into slot sb % 3.  Whole slots take four
+  // 64-row boxes; the ragged last slot takes 16-row boxes for the row groups that hold valid rows,
+  // so a split never pulls more than 15 rows of its neighbour.  Rows at or beyond kv_len lie
+  // outside the tensor and arrive as zeros.
+  auto fill = [&](int sb) {
+    const int s = sb % kSlots, k = sb / kSlots;
+    const uint32_t bar = smem_u32(&s_full[s][k & 1]);
+    const uint32_t dst = ring + s * kSlotBytes;
+    const int row0 = r0 + sb * kSlotRows;
+    const int nrows = min(kSlotRows, r1 - row0);
+    if (nrows == kSlotRows) {
+      mbar_expect_tx(bar, kSlotBytes);
+      tma_load_3d(dst, &TM.k64, bar, 0, row0, unit);
+      tma_load_3d(dst + kPlaneBytes, &TM.k64, bar, 64, row0, unit);
+      tma_load_3d(dst + 2 * kPlaneBytes, &TM.v64, bar, 0, row0, unit);
+      tma_load_3d(dst + 3 * kPlaneBytes, &TM.v64, bar, 64, row0, unit);
+    } else {
+      const int nb = (nrows + kBlkRows - 1) / kBlkRows;
+      mbar_expect_tx(bar, (uint32_t)nb * 4u * kBlkRows * 128u);
+      for (int j = 0; j < nb; ++j) {
+        const uint32_t dj = dst + j * kBlkRows * 128;
+        tma_load_3d(dj, &TM.k16, bar, 0, row0 + j * kBlkRows, unit);
+        tma_load_3d(dj + kPlaneBytes, &TM.k16, bar, 64, row0 + j * kBlkRows, unit);
+        tma_load_3d(dj + 2 * kPlaneBytes, &TM.v16, bar, 0, row0 + j * kBlkRows, unit);
+        tma_load_3d(dj + 3 * kPlaneBytes, &TM.v16, bar, 64, row0 + j * kBlkRows, unit);
+      }
+    }
+  };
+  if (warp == kStreamWarps) {
+    if (lane == 0)
+      for (int sb = 0; sb < min(n_sb, kSlots); ++sb) fill(sb);
+    __syncwarp();
+  }
+
+  // ---- (1) cosine similarities of this CTA's calibration rows: four lanes per (head, row) pair,
+  // 72 pairs per pass; the best pair per head goes to s_best while the first slots are in flight
   constexpr int kPairsPerPass = kThreads / 4;
   const int pairs = n_c * a.G;
-  const int sub = tid & 3;
+  const int sub4 = tid & 3;
   auto rho_load = [&](int pi, RhoLoad (&r)[2]) {
     r[0] = RhoLoad{}; r[1] = RhoLoad{};
     if (pi < pairs) {
       const int g = pi % a.G, c = c_begin + pi / a.G;
-      const uint4* qp = reinterpret_cast<const uint4*>(q + (size_t)(hq0 + g) * kD + sub * 32);
-      const uint4* cp = reinterpret_cast<const uint4*>(Cq + ((size_t)(hq0 + g) * a.n_cal + c) * kD + sub * 32);
+      const uint4* qp = reinterpret_cast<const uint4*>(q + (size_t)(hq0 + g) * kD + sub4 * 32);
+      const uint4* cp = reinterpret_cast<const uint4*>(Cq + ((size_t)(hq0 + g) * a.n_cal + c) * kD + sub4 * 32);
       r[0].q0 = __ldg(qp); r[0].q1 = __ldg(qp + 1); r[0].c0 = __ldg(cp); r[0].c1 = __ldg(cp + 1);
       r[1].q0 = __ldg(qp + 2); r[1].q1 = __ldg(qp + 3); r[1].c0 = __ldg(cp + 2); r[1].c1 = __ldg(cp + 3);
     }
@@ -209,147 +325,163 @@ __global__ void __launch_bounds__(kThreads, 1) decode_kernel(const __grid_consta
       qq += __shfl_xor_sync(0xffffffffu, qq, o);
       cc += __shfl_xor_sync(0xffffffffu, cc, o);
     }
-    if (sub == 0 && pi < pairs) {
+    if (sub4 == 0 && pi < pairs) {
       const int g = pi % a.G, c = c_begin + pi / a.G;
       const float rho = (qq > 0.f && cc > 0.f) ? dot / (sqrtf(qq) * sqrtf(cc)) : 0.f;
       atomicMax(&s_best[g], rank_key(rho, c));
     }
   };
-  RhoLoad rl0[2], rl1[2];
-  rho_load(tid >> 2, rl0);
-  rho_load(kPairsPerPass + (tid >> 2), rl1);
-
-  // ---- (2) the K/V stream: issue one 16-row block (K and V) of this warp into a stage
-  auto issue = [&](int i, int stage) {
-    const int row_base = r0 + (warp + i * kWarps) * kBlkRows;
-    const uint32_t dstK = wsm_u32 + stage * kStageBytes;
-    const uint32_t dstV = dstK + kBlkRows * kRowBytes;
-#pragma unroll
-    for (int it = 0; it < 8; ++it) {
-      const int idx = it * 32 + lane;
-      const int row = idx >> 4, chunk = idx & 15;
-      const int rg = row_base + row;
-      const bool valid = rg < r1;
-      const bool fresh = a.has_new && rg == a.kv_len;
-      const unsigned char* sk = fresh ? k_new + chunk * 16 : Kc + (size_t)(valid ? rg : 0) * kRowBytes + chunk * 16;
-      const unsigned char* sv = fresh ? v_new + chunk * 16 : Vc + (size_t)(valid ? rg : 0) * kRowBytes + chunk * 16;
-      cp_async_16(dstK + swz(row, chunk), sk, valid ? 16 : 0);
-      cp_async_16(dstV + swz(row, chunk), sv, valid ? 16 : 0);
-    }
-  };
-#pragma unroll
-  for (int s = 0; s < kStages - 1; ++s) {
-    if (s < my_blocks) issue(s, s);
-    cp_async_commit();
-  }
-
-  // ---- (3) query fragments (rows 0..G-1 of a 16-row A tile, the rest zero)
+  // query fragments of the stream warps (B operand of S^T, heads on the 8-column side): their
+  // loads go out together with those of the similarity
   uint32_t qa[kD / 16][2];
 #pragma unroll
   for (int kk = 0; kk < kD / 16; ++kk) {
     qa[kk][0] = 0u; qa[kk][1] = 0u;
-    if (gq < a.G) {
+    if (warp < kStreamWarps && gq < a.G) {
       const uint32_t* qr = reinterpret_cast<const uint32_t*>(q + (size_t)(hq0 + gq) * kD + kk * 16);
       qa[kk][0] = __ldg(qr + tq);
       qa[kk][1] = __ldg(qr + 4 + tq);
     }
   }
-
-  // ---- (3b) append: the CTA whose slice holds row kv_len stores the new K/V row into the cache
-  if (a.has_new && a.kv_len >= r0 && a.kv_len < r1 && warp == 0) {
-    const int chunk = lane & 15;
-    const unsigned char* src = (lane < 16 ? k_new : v_new) + chunk * 16;
-    unsigned char* dst = (unsigned char*)(lane < 16 ? P.K : P.V) +
-                         ((size_t)unit * a.cap + a.kv_len) * kRowBytes + chunk * 16;
-    *reinterpret_cast<uint4*>(dst) = *reinterpret_cast<const uint4*>(src);
-  }
-
-  // ---- (4) cosine similarities of this CTA's calibration rows; the best pair per head goes to
-  // s_best (the K/V copies are in flight meanwhile)
-  rho_finish(tid >> 2, rl0);
-  rho_finish(kPairsPerPass + (tid >> 2), rl1);
-  for (int base = 2 * kPairsPerPass; base < pairs; base += kPairsPerPass) {
-    rho_load(base + (tid >> 2), rl0);
-    rho_finish(base + (tid >> 2), rl0);
+  {
+    RhoLoad rl[2];
+    rho_load(tid >> 2, rl);
+    rho_finish(tid >> 2, rl);
+    for (int base = kPairsPerPass; base < pairs; base += kPairsPerPass) {
+      rho_load(base + (tid >> 2), rl);
+      rho_finish(base + (tid >> 2), rl);
+    }
   }
   cluster_arrive();  // (A) this CTA's s_best is final
 
-  // ---- (5) main loop.  The products are taken transposed, keys on the 16-row side of the MMA and
-  // the (at most eight) heads on its 8-column side, so that no half of a tile is padding:
-  //   S^T[16 keys x 8 heads]   = K_blk[16 x 128] . Q^T[128 x 8]          (8 MMAs)
-  //   O^T[128 dims x 8 heads] += V_blk^T[128 x 16 keys] . P^T[16 x 8]     (8 MMAs)
-  // A thread holds heads 2tq, 2tq+1 of keys gq, gq+8 (S^T) and of dims 16n+gq, 16n+gq+8 (O^T).
   float o[kD / 16][4];
 #pragma unroll
   for (int n = 0; n < kD / 16; ++n) { o[n][0] = o[n][1] = o[n][2] = o[n][3] = 0.f; }
   float m0 = -INFINITY, m1 = -INFINITY, l0 = 0.f, l1 = 0.f;  // heads 2tq and 2tq+1
-  const int mid = lane >> 3;
 
-  for (int i = 0; i < my_blocks; ++i) {
-    const int nxt = i + kStages - 1;
-    if (nxt < my_blocks) issue(nxt, nxt % kStages);
-    cp_async_commit();
-    cp_async_wait<kStages - 1>();
-    __syncwarp();
-
-    const uint32_t sK = wsm_u32 + (i % kStages) * kStageBytes;
-    const uint32_t sV = sK + kBlkRows * kRowBytes;
-    const int row_base = r0 + (warp + i * kWarps) * kBlkRows;
-
-    // S^T: two accumulators (even and odd k-steps) halve the dependent chain
-    float sa[4] = {0.f, 0.f, 0.f, 0.f}, sb[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll
-    for (int kk = 0; kk < kD / 16; ++kk) {
-      uint32_t a0, a1, a2, a3;
-      ldmatrix_x4(sK + swz((lane & 7) + (mid & 1) * 8, kk * 2 + (mid >> 1)), a0, a1, a2, a3);
-      if (kk & 1) mma_bf16_16816(sb, a0, a1, a2, a3, qa[kk][0], qa[kk][1]);
-      else mma_bf16_16816(sa, a0, a1, a2, a3, qa[kk][0], qa[kk][1]);
+  if (warp == kStreamWarps) {
+    // ---- (2) producer: refill a slot as soon as its four warps have released it
+    if (lane == 0) {
+      for (int sb = kSlots; sb < n_sb; ++sb) {
+        const int s = sb % kSlots, kp = sb / kSlots - 1;  // the fill that occupies the slot
+        if (!mbar_wait(smem_u32(&s_empty[s][kp & 1]), (kp >> 1) & 1, abort_flag, a.status, 0x100u + sb)) break;
+        fill(sb);
+      }
     }
-    // online softmax per head over the 16 keys of the block (keys gq and gq + 8 live here)
-    const bool v0 = row_base + gq < r1, v1 = row_base + gq + 8 < r1;
-    const float x00 = v0 ? (sa[0] + sb[0]) * a.scale2 : -INFINITY;
-    const float x01 = v0 ? (sa[1] + sb[1]) * a.scale2 : -INFINITY;
-    const float x10 = v1 ? (sa[2] + sb[2]) * a.scale2 : -INFINITY;
-    const float x11 = v1 ? (sa[3] + sb[3]) * a.scale2 : -INFINITY;
-    float bm0 = fmaxf(x00, x10), bm1 = fmaxf(x01, x11);
+    __syncwarp();
+  } else {
+    // ---- (3) stream warps
+    const int group = warp >> 2, sub = warp & 3;
+    const int mid = lane >> 3;
+    for (int sb = group; sb < n_sb; sb += 2) {
+      const int s = sb % kSlots, k = sb / kSlots;
+      const bool ok = mbar_wait(smem_u32(&s_full[s][k & 1]), (k >> 1) & 1, abort_flag, a.status, 0x200u + sb);
+      const int row_base = r0 + sb * kSlotRows + sub * kBlkRows;
+      if (ok && row_base < r1) {
+        const uint32_t sK = ring + s * kSlotBytes;
+        const uint32_t sV = sK + 2 * kPlaneBytes;
+        // D1: the warp that meets row kv_len takes it from k_new / v_new (the cache row is
+        // outside the TMA tensor and arrived as zeros) and appends it to the cache
+        if (a.has_new && a.kv_len >= row_base && a.kv_len < row_base + kBlkRows) {
+          const int chunk = lane & 15;
+          const int rs = a.kv_len - (r0 + sb * kSlotRows);  // row inside the slot
+          const unsigned char* src = (const unsigned char*)(lane < 16 ? P.k_new : P.v_new) +
+                                     (size_t)unit * kRowBytes + chunk * 16;
+          const uint4 v = *reinterpret_cast<const uint4*>(src);
+          unsigned char* dstg = (unsigned char*)(lane < 16 ? P.K : P.V) +
+                                ((size_t)unit * a.cap + a.kv_len) * kRowBytes + chunk * 16;
+          *reinterpret_cast<uint4*>(dstg) = v;
+          *reinterpret_cast<uint4*>(ring_ptr + s * kSlotBytes + (lane < 16 ? 0 : 2 * kPlaneBytes) +
+                                    plane_off(rs, chunk)) = v;
+          __syncwarp();
+        }
+        // S^T: two accumulators (even and odd k-steps) halve the dependent chain
+        float sa[4] = {0.f, 0.f, 0.f, 0.f}, sb2[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+        for (int kk = 0; kk < kD / 16; ++kk) {
+          uint32_t a0, a1, a2, a3;
+          ldmatrix_x4(sK + plane_off(sub * kBlkRows + (lane & 7) + (mid & 1) * 8, kk * 2 + (mid >> 1)), a0, a1, a2, a3);
+          if (kk & 1) mma_bf16_16816(sb2, a0, a1, a2, a3, qa[kk][0], qa[kk][1]);
+          else mma_bf16_16816(sa, a0, a1, a2, a3, qa[kk][0], qa[kk][1]);
+        }
+        // online softmax per head over the 16 keys of the block (keys gq and gq + 8 live here)
+        const bool v0 = row_base + gq < r1, v1 = row_base + gq + 8 < r1;
+        const float x00 = v0 ? (sa[0] + sb2[0]) * a.scale2 : -INFINITY;
+        const float x01 = v0 ? (sa[1] + sb2[1]) * a.scale2 : -INFINITY;
+        const float x10 = v1 ? (sa[2] + sb2[2]) * a.scale2 : -INFINITY;
+        const float x11 = v1 ? (sa[3] + sb2[3]) * a.scale2 : -INFINITY;
+        float bm0 = fmaxf(x00, x10), bm1 = fmaxf(x01, x11);
+#pragma unroll
+        for (int off = 4; off < 32; off <<= 1) {
+          bm0 = fmaxf(bm0, __shfl_xor_sync(0xffffffffu, bm0, off));
+          bm1 = fmaxf(bm1, __shfl_xor_sync(0xffffffffu, bm1, off));
+        }
+        const float mn0 = fmaxf(m0, bm0), mn1 = fmaxf(m1, bm1);  // finite: the block's first key is valid
+        const float corr0 = ex2_approx(m0 - mn0), corr1 = ex2_approx(m1 - mn1);
+        const float p00 = ex2_approx(x00 - mn0), p01 = ex2_approx(x01 - mn1);
+        const float p10 = ex2_approx(x10 - mn0), p11 = ex2_approx(x11 - mn1);
+        l0 = l0 * corr0 + (p00 + p10);  // partial over this thread's keys, summed over gq at the end
+        l1 = l1 * corr1 + (p01 + p11);
+        m0 = mn0; m1 = mn1;
+#pragma unroll
+        for (int n = 0; n < kD / 16; ++n) { o[n][0] *= corr0; o[n][1] *= corr1; o[n][2] *= corr0; o[n][3] *= corr1; }
+        // P^T as the B operand: transpose the two 8x8 (key, head) fragments inside the warp
+        const uint32_t pb0 = movmatrix_trans(pack_bf16(p00, p01)), pb1 = movmatrix_trans(pack_bf16(p10, p11));
+#pragma unroll
+        for (int n = 0; n < kD / 16; ++n) {
+          uint32_t a0, a1, a2, a3;
+          ldmatrix_x4_trans(sV + plane_off(sub * kBlkRows + (lane & 7) + (mid >> 1) * 8, n * 2 + (mid & 1)), a0, a1, a2, a3);
+          mma_bf16_16816(o[n], a0, a1, a2, a3, pb0, pb1);
+        }
+      }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(smem_u32(&s_empty[s][k & 1]));  // the slot may be refilled
+    }
 #pragma unroll
     for (int off = 4; off < 32; off <<= 1) {
-      bm0 = fmaxf(bm0, __shfl_xor_sync(0xffffffffu, bm0, off));
-      bm1 = fmaxf(bm1, __shfl_xor_sync(0xffffffffu, bm1, off));
+      l0 += __shfl_xor_sync(0xffffffffu, l0, off);
+      l1 += __shfl_xor_sync(0xffffffffu, l1, off);
     }
-    const float mn0 = fmaxf(m0, bm0), mn1 = fmaxf(m1, bm1);  // finite: the block's first key is valid
-    const float corr0 = ex2_approx(m0 - mn0), corr1 = ex2_approx(m1 - mn1);
-    const float p00 = ex2_approx(x00 - mn0), p01 = ex2_approx(x01 - mn1);
-    const float p10 = ex2_approx(x10 - mn0), p11 = ex2_approx(x11 - mn1);
-    l0 = l0 * corr0 + (p00 + p10);  // partial over this thread's keys, summed over gq at the end
-    l1 = l1 * corr1 + (p01 + p11);
-    m0 = mn0; m1 = mn1;
-#pragma unroll
-    for (int n = 0; n < kD / 16; ++n) { o[n][0] *= corr0; o[n][1] *= corr1; o[n][2] *= corr0; o[n][3] *= corr1; }
-    // P^T as the B operand: transpose the two 8x8 (key, head) fragments inside the warp
-    const uint32_t pb0 = movmatrix_trans(pack_bf16(p00, p01)), pb1 = movmatrix_trans(pack_bf16(p10, p11));
-#pragma unroll
-    for (int n = 0; n < kD / 16; ++n) {
-      uint32_t a0, a1, a2, a3;
-      ldmatrix_x4_trans(sV + swz((lane & 7) + (mid >> 1) * 8, n * 2 + (mid & 1)), a0, a1, a2, a3);
-      mma_bf16_16816(o[n], a0, a1, a2, a3, pb0, pb1);
-    }
-    __syncwarp();  // the stage is refilled by the next iteration's cp.async
   }
-  cp_async_wait<0>();
-#pragma unroll
-  for (int off = 4; off < 32; off <<= 1) {
-    l0 += __shfl_xor_sync(0xffffffffu, l0, off);
-    l1 += __shfl_xor_sync(0xffffffffu, l1, off);
-  }
-  __syncthreads();  // all warps are done with their stages: reuse them for the combine
 
-  // ---- (6) CTA combine of the four warps into this split's partial: xo[g][d], xml[g] = (m, l)
-  float* wo = reinterpret_cast<float*>(smem);             // [warp][8][kWoStride]
-  float* wml = wo + kWarps * kMaxG * kWoStride;            // [warp][8][2]
-  float* xo = wml + kWarps * kMaxG * 2;                    // [8][128]
-  float* xml = xo + kMaxG * kD;                            // [8][2]
-  if (2 * tq < a.G) {
+  // ---- (4) the calibration row: best similarity over the cluster, ties to the largest row
+  // index; the chosen O_c row and LSE_c start their way into L2 while the partials are combined
+  cluster_wait();  // (A) every CTA's s_best can be read
+  if (tid < a.G) {
+    unsigned long long best = 0ull;
+    for (int s = 0; s < a.nsplit; ++s) {
+      const unsigned long long k = *cluster.map_shared_rank(&s_best[tid], s);
+      best = k > best ? k : best;
+    }
+    s_bestall[tid] = best;
+    if (a.nclu == 1 && a.G * (kD / a.nsplit) > kThreads) {
+      const size_t crow = (size_t)(hq0 + tid) * a.n_cal + (unsigned)(best & 0xffffffffull);
+      const float* orow = P.O_c + crow * kD;
+#pragma unroll
+      for (int i = 0; i < 4; ++i) asm volatile("prefetch.global.L2 [%0];" ::"l"(orow + i * 32));
+      asm volatile("prefetch.global.L2 [%0];" ::"l"(P.LSE_c + crow));
+    }
+  }
+  __syncthreads();  // all warps are done with the ring: reuse it for the combine
+  const int dpc = kD / a.nsplit;
+  const int n_items = a.G * dpc;
+  const bool single = a.nclu == 1;
+  // the common case has one output element per thread at most: its O_c element and LSE_c are
+  // loaded now and arrive while the partials are combined
+  const bool early = single && n_items <= kThreads;
+  float lse_c_early = 0.f, oc_early = 0.f;
+  if (early && tid < n_items) {
+    const int g = tid / dpc, d = split * dpc + tid % dpc;
+    const size_t crow = (size_t)(hq0 + g) * a.n_cal + (unsigned)(s_bestall[g] & 0xffffffffull);
+    lse_c_early = __ldg(P.LSE_c + crow);
+    oc_early = __ldg(P.O_c + crow * kD + d);
+  }
+
+  // ---- (5) CTA combine of the eight stream warps, pushed to the owners of the output slices:
+  // CTA r of the cluster owns dimensions [r * dpc, (r + 1) * dpc) of every head of the group
+  float* wo = reinterpret_cast<float*>(ring_ptr);          // [warp][8][kWoStride]
+  float* wml = wo + kStreamWarps * kMaxG * kWoStride;       // [warp][8][2]
+  if (warp < kStreamWarps && 2 * tq < a.G) {
 #pragma unroll
     for (int n = 0; n < kD / 16; ++n) {
       float* w0 = wo + (warp * kMaxG + 2 * tq) * kWoStride + n * 16 + gq;
@@ -362,77 +494,54 @@ __global__ void __launch_bounds__(kThreads, 1) decode_kernel(const __grid_consta
     }
   }
   __syncthreads();
-  for (int d = tid; d < kD; d += kThreads) {
-#pragma unroll
-    for (int g = 0; g < kMaxG; ++g) {
-      if (g >= a.G) break;
-      float M = -INFINITY;
-#pragma unroll
-      for (int w = 0; w < kWarps; ++w) M = fmaxf(M, wml[(w * kMaxG + g) * 2]);
-      float Lsum = 0.f, acc = 0.f;
-#pragma unroll
-      for (int w = 0; w < kWarps; ++w) {
-        const float mw = wml[(w * kMaxG + g) * 2];
-        const float sc = mw > -INFINITY ? ex2_approx(mw - M) : 0.f;
-        Lsum += wml[(w * kMaxG + g) * 2 + 1] * sc;
-        acc += wo[(w * kMaxG + g) * kWoStride + d] * sc;
-      }
-      xo[g * kD + d] = acc;
-      if (d == 0) { xml[g * 2] = M; xml[g * 2 + 1] = Lsum; }
-    }
-  }
-  cluster_wait();    // (A) every CTA's s_best can be read
-  cluster_arrive();  // (B) this CTA's partial (xo, xml) is final
-
-  // ---- (7) finish.  This CTA owns 128 / nsplit output dimensions of every head of the group.
-  const int dpc = kD / a.nsplit;
-  const int n_items = a.G * dpc;
-  const bool single = a.nclu == 1;
-  const int lu = layer * a.units + unit;
-  for (int item0 = 0; item0 < n_items; item0 += kThreads) {
-    const int item = item0 + tid;
-    const bool act = item < n_items;
-    const int g = act ? item / dpc : 0, d = split * dpc + (act ? item % dpc : 0);
-    const int hq = hq0 + g;
-    // the calibration row: best similarity over all CTAs, ties to the largest row index
-    unsigned long long best = 0ull;
-#pragma unroll
-    for (int s = 0; s < 8; ++s) {
-      if (s < a.nsplit) {
-        const unsigned long long k = *cluster.map_shared_rank(&s_best[g], s);
-        best = k > best ? k : best;
-      }
-    }
-    float lse_c = 0.f, oc = 0.f;
-    if (act && single) {  // in flight while the partials are exchanged
-      const size_t crow = (size_t)hq * a.n_cal + (unsigned)(best & 0xffffffffull);
-      lse_c = __ldg(P.LSE_c + crow);
-      oc = __ldg(P.O_c + crow * kD + d);
-    }
-    if (item0 == 0) cluster_wait();  // (B) every CTA's partial can be read
-    float ms[8], ls[8], os[8];
-#pragma unroll
-    for (int s = 0; s < 8; ++s) {  // all remote reads in flight together
-      ms[s] = -INFINITY; ls[s] = 0.f; os[s] = 0.f;
-      if (s < a.nsplit) {
-        const float2 ml2 = *reinterpret_cast<const float2*>(cluster.map_shared_rank(xml, s) + g * 2);
-        ms[s] = ml2.x; ls[s] = ml2.y;
-        os[s] = cluster.map_shared_rank(xo, s)[g * kD + d];
-      }
-    }
+  for (int idx = tid; idx < a.G * kD; idx += kThreads) {
+    const int g = idx / kD, d = idx % kD;
     float M = -INFINITY;
 #pragma unroll
-    for (int s = 0; s < 8; ++s) M = fmaxf(M, ms[s]);
+    for (int w = 0; w < kStreamWarps; ++w) M = fmaxf(M, wml[(w * kMaxG + g) * 2]);
     float Lsum = 0.f, acc = 0.f;
 #pragma unroll
-    for (int s = 0; s < 8; ++s) {
-      const float sc = ms[s] > -INFINITY ? ex2_approx(ms[s] - M) : 0.f;
-      Lsum = fmaf(ls[s], sc, Lsum);
-      acc = fmaf(os[s], sc, acc);
+    for (int w = 0; w < kStreamWarps; ++w) {
+      const float mw = wml[(w * kMaxG + g) * 2];
+      const float sc = mw > -INFINITY ? ex2_approx(mw - M) : 0.f;
+      Lsum += wml[(w * kMaxG + g) * 2 + 1] * sc;
+      acc += wo[(w * kMaxG + g) * kWoStride + d] * sc;
+    }
+    const int owner = d / dpc;
+    cluster.map_shared_rank(s_xpart, owner)[(split * kMaxG + g) * dpc + (d - owner * dpc)] = acc;
+    if (d < a.nsplit) {  // the (max, sum) pair of this split goes to every CTA of the cluster
+      float* xm = &cluster.map_shared_rank(&s_xml[0][0][0], d)[(split * kMaxG + g) * 2];
+      xm[0] = M; xm[1] = Lsum;
+    }
+  }
+  cluster_arrive();  // (B) this CTA's pushes are done
+  cluster_wait();    //     and everything pushed to this CTA has arrived
+
+  // ---- (6) finish: reduce the splits for this CTA's output slice (local data only from here on,
+  // so no CTA has to wait for another before it leaves)
+  const int lu = layer * a.units + unit;
+  for (int item = tid; item < n_items; item += kThreads) {
+    const int g = item / dpc, dl = item % dpc, d = split * dpc + dl;
+    const int hq = hq0 + g;
+    const unsigned long long best = s_bestall[g];
+    float M = -INFINITY;
+    for (int s = 0; s < a.nsplit; ++s) M = fmaxf(M, s_xml[s][g][0]);
+    float Lsum = 0.f, acc = 0.f;
+    for (int s = 0; s < a.nsplit; ++s) {
+      const float ms = s_xml[s][g][0];
+      const float sc = ms > -INFINITY ? ex2_approx(ms - M) : 0.f;
+      Lsum = fmaf(s_xml[s][g][1], sc, Lsum);
+      acc = fmaf(s_xpart[(s * kMaxG + g) * dpc + dl], sc, acc);
     }
     if (single) {
-      if (act) merge_store(a, P, hq, d, acc, M, Lsum, best, lse_c, oc);
-    } else if (act) {
+      float lse_c = lse_c_early, oc = oc_early;
+      if (!early) {
+        const size_t crow = (size_t)hq * a.n_cal + (unsigned)(best & 0xffffffffull);
+        lse_c = __ldg(P.LSE_c + crow);
+        oc = __ldg(P.O_c + crow * kD + d);
+      }
+      merge_store(a, P, hq, d, acc, M, Lsum, best, lse_c, oc);
+    } else {
       // this cluster's partial goes to the workspace; (M, Lsum, best) are the same in all its CTAs
       const size_t pc = ((size_t)lu * a.nclu + clu) * kMaxG + g;
       a.part_o[pc * kD + d] = acc;
@@ -443,10 +552,8 @@ __global__ void __launch_bounds__(kThreads, 1) decode_kernel(const __grid_consta
       }
     }
   }
-  cluster_arrive();  // (C) no CTA leaves while another may still read its shared memory
   if (!single) {
-    // ---- (8) several clusters per unit: the CTA that takes the unit's last ticket merges them
-    __shared__ unsigned s_ticket;
+    // ---- (7) several clusters per unit: the CTA that takes the unit's last ticket merges them
     __threadfence();
     __syncthreads();
     if (tid == 0) s_ticket = atomicAdd(&a.counters[lu], 1u);
@@ -489,39 +596,60 @@ __global__ void __launch_bounds__(kThreads, 1) decode_kernel(const __grid_consta
       if (tid == 0) a.counters[lu] = 0u;  // ready for the next launch on this workspace
     }
   }
-  cluster_wait();
 }
 
 }  // namespace
 
-cudaError_t launch_decode(const DecodeArgs& a, cudaStream_t st) {
+bool make_decode_maps(const DecodeCommon& c, const DecodeLayerPtrs& L, DecodeLayerMaps* out) {
+  // rows at or beyond kv_len are outside the tensor: the TMA unit delivers zeros for them
+  const uint64_t rows = (uint64_t)(c.kv_len > 0 ? c.kv_len : 1);
+  const uint64_t dims[2] = {rows, (uint64_t)c.units};
+  const uint64_t strides[2] = {(uint64_t)kRowBytes, (uint64_t)c.cap * kRowBytes};
+  const uint32_t box64[2] = {(uint32_t)kSlotRows, 1}, box16[2] = {(uint32_t)kBlkRows, 1};
+  return make_tensor_map_bf16(&out->k64, L.K, 3, dims, strides, box64) &&
+         make_tensor_map_bf16(&out->v64, L.V, 3, dims, strides, box64) &&
+         make_tensor_map_bf16(&out->k16, L.K, 3, dims, strides, box16) &&
+         make_tensor_map_bf16(&out->v16, L.V, 3, dims, strides, box16);
+}
+
+namespace {
+
+template <int NL>
+cudaError_t launch_decode_t(const DecodeArgsT<NL>& a, cudaStream_t st) {
   static bool attr_set[64] = {};
   int dev = 0;
   cudaError_t e = cudaGetDevice(&dev);
   if (e != cudaSuccess) return e;
   if (dev < 0 || dev >= 64 || !attr_set[dev]) {
-    e = cudaFuncSetAttribute(decode_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+    e = cudaFuncSetAttribute(decode_kernel<NL>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
     if (e != cudaSuccess) return e;
     if (dev >= 0 && dev < 64) attr_set[dev] = true;
   }
   cudaLaunchConfig_t cfg{};
-  cfg.gridDim = dim3(a.nsplit * a.nclu, a.units, a.n_layers);
+  cfg.gridDim = dim3(a.c.nsplit * a.c.nclu, a.c.units, a.c.n_layers);
   cfg.blockDim = dim3(kThreads);
   cfg.dynamicSmemBytes = kSmemBytes;
   cfg.stream = st;
   cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeClusterDimension;  // the splits of a unit are one cluster
-  attr[0].val.clusterDim.x = a.nsplit;
+  attr[0].val.clusterDim.x = a.c.nsplit;
   attr[0].val.clusterDim.y = 1;
   attr[0].val.clusterDim.z = 1;
   attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 2;
-  e = cudaLaunchKernelEx(&cfg, decode_kernel, a);
+  e = cudaLaunchKernelEx(&cfg, decode_kernel<NL>, a);
   if (e != cudaSuccess) return e;
   count_launch(1);
   return cudaGetLastError();
+}
+
+}  // namespace
+
+cudaError_t launch_decode(const DecodeArgsT<1>& a, cudaStream_t st) { return launch_decode_t<1>(a, st); }
+cudaError_t launch_decode(const DecodeArgsT<kDecodeMaxLayers>& a, cudaStream_t st) {
+  return launch_decode_t<kDecodeMaxLayers>(a, st);
 }
 
 }  // namespace calidrop

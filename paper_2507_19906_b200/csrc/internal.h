@@ -1,6 +1,7 @@
 // Internal launcher interface between the C-ABI layer (api.cu) and the kernels.
 #pragma once
 
+#include <cuda.h>
 #include <cuda_runtime.h>
 #include <stddef.h>
 #include <stdint.h>
@@ -40,11 +41,17 @@ struct DecodeLayerPtrs {
   uint8_t* flags;
 };
 
+// TMA views of one layer's retained cache, [unit][row < kv_len][128] bf16 with 128-byte swizzle:
+// boxes of 64 rows for whole ring slots and of 16 rows for the ragged end of a split.
+struct alignas(64) DecodeLayerMaps {
+  CUtensorMap k64, v64, k16, v16;
+};
+
 constexpr int kDecodeMaxLayers = 32;
 constexpr int kDecodeMaxSplit = 64;
-constexpr int kDecodeTargetCtas = 148;  // one resident CTA on each of the 148 SMs
+constexpr int kDecodeTargetCtas = 148;  // one CTA of a launch on each of the 148 SMs
 
-struct DecodeArgs {
+struct DecodeCommon {
   int B, Hq, Hkv, G, n_cal, cap, kv_len, n_kv, has_new;
   int units, n_layers, rows_per_split;
   int nsplit;  // CTAs per cluster (1, 2, 4 or 8): the splits combined through distributed shared memory
@@ -56,7 +63,16 @@ struct DecodeArgs {
   float* part_ml;                 // [layer][unit][nclu][8][2]
   unsigned long long* part_best;  // [layer][unit][nclu][8] best (similarity, row) keys
   unsigned* counters;             // [layer][unit]
-  DecodeLayerPtrs layer[kDecodeMaxLayers];
+  unsigned* status;               // error word of the workspace: nonzero after a wait ran out
+};
+
+// Kernel argument block for NL layers (1 for the single-layer entry points, 32 for the batched one:
+// the block travels with every launch, so the common case keeps it small).
+template <int NL>
+struct DecodeArgsT {
+  DecodeCommon c;
+  DecodeLayerPtrs layer[NL];
+  DecodeLayerMaps maps[NL];
 };
 
 // compress_simt.cu
@@ -90,7 +106,10 @@ cudaError_t launch_pool_select_cluster(const CompressGeom& g, const CompressWs& 
 cudaError_t launch_gather(const CompressGeom& g, const void* K, const void* V, const int32_t* kept_idx,
                           void* K_kept, void* V_kept, cudaStream_t st);
 // decode.cu
-cudaError_t launch_decode(const DecodeArgs& a, cudaStream_t st);
+// Fills the TMA views of one layer; false when the driver refuses the encoding.
+bool make_decode_maps(const DecodeCommon& c, const DecodeLayerPtrs& L, DecodeLayerMaps* out);
+cudaError_t launch_decode(const DecodeArgsT<1>& a, cudaStream_t st);
+cudaError_t launch_decode(const DecodeArgsT<kDecodeMaxLayers>& a, cudaStream_t st);
 
 void count_launch(int n = 1);
 
