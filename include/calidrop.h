@@ -142,6 +142,15 @@ size_t calidrop_decode_workspace_bytes(const calidrop_params* p, int32_t kv_len_
 int calidrop_decode_workspace_init(void* workspace, size_t workspace_bytes, void* stream);
 
 /*
+ * Byte offset, from the base of a decode workspace, of its 32-bit error word (the same offset
+ * for every layer count).  The decode kernel waits on its copy pipeline with a time limit; a
+ * wait that expires (a bug or a failing device, not bad input) stores a non-zero code there and
+ * the kernel runs to its end without hanging, with undefined outputs for that call.  The word
+ * stays 0 otherwise.  Returns (size_t)-1 if the parameters are invalid.
+ */
+size_t calidrop_decode_workspace_status_offset(const calidrop_params* p);
+
+/*
  * One decode step for one layer (Algorithm 2, lines 1-2 and 9-14).
  *
  * Per (b, query head hq of kv head h):

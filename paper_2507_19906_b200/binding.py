@@ -24,7 +24,8 @@ MAX_LAYERS = 32
 
 EXPORTS = [
     "calidrop_compress_workspace_bytes", "calidrop_compress", "calidrop_compress_workspace_layout",
-    "calidrop_decode_workspace_bytes", "calidrop_decode_workspace_init", "calidrop_decode",
+    "calidrop_decode_workspace_bytes", "calidrop_decode_workspace_init",
+    "calidrop_decode_workspace_status_offset", "calidrop_decode",
     "calidrop_decode_batched", "calidrop_decode_static", "calidrop_compress_host", "calidrop_decode_host",
     "calidrop_status_string", "calidrop_version", "calidrop_launch_count",
 ]
@@ -70,6 +71,8 @@ def load():
     vp = C.c_void_p
     lib.calidrop_compress.restype = C.c_int
     lib.calidrop_compress.argtypes = [C.POINTER(Params)] + [vp] * 11 + [C.c_size_t, vp]
+    lib.calidrop_decode_workspace_status_offset.restype = C.c_size_t
+    lib.calidrop_decode_workspace_status_offset.argtypes = [C.POINTER(Params)]
     lib.calidrop_decode_workspace_init.restype = C.c_int
     lib.calidrop_decode_workspace_init.argtypes = [vp, C.c_size_t, vp]
     lib.calidrop_decode.restype = C.c_int
@@ -133,6 +136,10 @@ def calidrop_compress_workspace_bytes(p: Params) -> int:
 
 def calidrop_decode_workspace_bytes(p: Params, kv_len_max: int) -> int:
     return int(load().calidrop_decode_workspace_bytes(C.byref(p), kv_len_max))
+
+
+def calidrop_decode_workspace_status_offset(p: Params) -> int:
+    return int(load().calidrop_decode_workspace_status_offset(C.byref(p)))
 
 
 def calidrop_compress_workspace_layout(p: Params) -> CompressLayout:

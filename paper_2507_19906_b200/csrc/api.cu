@@ -245,6 +245,11 @@ size_t calidrop_decode_workspace_bytes(const calidrop_params* p, int32_t kv_len_
   return make_decode_ws(p).per_layer;
 }
 
+size_t calidrop_decode_workspace_status_offset(const calidrop_params* p) {
+  if (check_common(p) != CALIDROP_OK) return (size_t)-1;
+  return make_decode_ws(p).status;
+}
+
 int calidrop_decode_workspace_init(void* workspace, size_t workspace_bytes, void* stream) {
   if (!workspace) return CALIDROP_INVALID_ARG;
   cudaError_t e = cudaMemsetAsync(workspace, 0, workspace_bytes, (cudaStream_t)stream);

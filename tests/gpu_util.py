@@ -141,6 +141,8 @@ def decode_steps_compare(g, ref, q, kn, vn, *, theta1=0.7, theta2=0.85, steps=No
         cd.calidrop_decode(p, dq, dk, dv, st.K_kept, st.V_kept, kv_len, st.O_c, st.LSE_c, st.C_q, out, lse,
                            flags, st.ws_decode)
         torch.cuda.synchronize()
+        off = cd.calidrop_decode_workspace_status_offset(p)
+        assert int(st.ws_decode[off:off + 4].view(torch.int32).item()) == 0, "a wait of the decode kernel ran out"
         gout = wl.bf16_bits_to_f64(to_bits(out))
         gflags = flags.cpu().numpy()
         o = oracle.decode(q[t], kn[t] if append else None, vn[t] if append else None, Kk, Vk, kv_len,

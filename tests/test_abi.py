@@ -46,6 +46,8 @@ def test_size_queries_and_status_strings(lib):
     assert ws >= 2 * 4 * 8 * (32768 - 64) * 4          # votes and pooled votes at least
     assert ws % 256 == 0
     assert cd.calidrop_decode_workspace_bytes(p, 2176) > 0
+    off = cd.calidrop_decode_workspace_status_offset(p)
+    assert off % 256 == 0 and off + 4 <= cd.calidrop_decode_workspace_bytes(p, 2176)
     lay = cd.calidrop_compress_workspace_layout(p)
     assert lay.vote_offset % 256 == 0 and lay.pooled_offset > lay.vote_offset
     bad = cd.make_params(B=4, Hq=32, Hkv=8, L=32768, window=64, pool=6, budget=2048, n_cal=64, cap=2176)
