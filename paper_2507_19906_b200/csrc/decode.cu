@@ -113,11 +113,40 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
   return true;
 }
 __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1,
-                                            int c2) {
+                                            int c2, uint64_t pol) {
   asm volatile(
-      "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
-      ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2)
+      "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes.L2::cache_hint "
+      "[%0], [%1, {%3, %4, %5}], [%2], %6;"
+      ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "l"(pol)
       : "memory");
+}
+
+// L2 eviction policies.  The retained cache is read once per call and is far larger than what the
+// next call on the same state finds in L2 again, so its lines are marked to go first; the
+// calibration state (C_q, the chosen O_c rows, LSE_c) is small and read by every call, so its
+// lines are marked to stay.  With that the similarity loads are L2 hits and do not queue behind
+// the stream in the memory system.
+__device__ __forceinline__ uint64_t policy_evict_first() {
+  uint64_t p;
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
+  return p;
+}
+__device__ __forceinline__ uint64_t policy_evict_last() {
+  uint64_t p;
+  asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(p));
+  return p;
+}
+__device__ __forceinline__ uint4 ldg_keep(const uint4* ptr, uint64_t pol) {
+  uint4 v;
+  asm volatile("ld.global.nc.L2::cache_hint.v4.u32 {%0, %1, %2, %3}, [%4], %5;"
+               : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+               : "l"(ptr), "l"(pol));
+  return v;
+}
+__device__ __forceinline__ float ldg_keep(const float* ptr, uint64_t pol) {
+  float v;
+  asm volatile("ld.global.nc.L2::cache_hint.f32 %0, [%1], %2;" : "=f"(v) : "l"(ptr), "l"(pol));
+  return v;
 }
 
 struct RhoLoad {
@@ -217,6 +246,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_kernel(const __grid_consta
   const int r1 = min(a.n_kv, r0 + a.rows_per_split);
   const int n_sb = (r1 - r0 + kSlotRows - 1) / kSlotRows;  // ring fills of this CTA
 
+  const uint64_t pol_stream = policy_evict_first(), pol_keep = policy_evict_last();
   const uint32_t ring = (smem_u32(smem_raw) + 1023u) & ~1023u;
   unsigned char* ring_ptr = smem_raw + (ring - smem_u32(smem_raw));
   volatile int* abort_flag = &s_abort;
@@ -243,9 +273,11 @@ __global__ void __launch_bounds__(kThreads, 1) decode_kernel(const __grid_consta
     const int n_old = min(r1, a.kv_len) - r0;  // rows already in the cache (the appended row is not)
     if (n_old > 0) {
       const unsigned bytes = (unsigned)n_old * kRowBytes;
-      asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(Kc + (size_t)r0 * kRowBytes), "r"(bytes)
+      asm volatile("cp.async.bulk.prefetch.L2.global.L2::cache_hint [%0], %1, %2;" ::"l"(Kc + (size_t)r0 * kRowBytes),
+                   "r"(bytes), "l"(pol_stream)
                    : "memory");
-      asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(Vc + (size_t)r0 * kRowBytes), "r"(bytes)
+      asm volatile("cp.async.bulk.prefetch.L2.global.L2::cache_hint [%0], %1, %2;" ::"l"(Vc + (size_t)r0 * kRowBytes),
+                   "r"(bytes), "l"(pol_stream)
                    : "memory");
     }
     asm volatile("prefetch.tensormap [%0];" ::"l"(&TM.k64) : "memory");
@@ -255,8 +287,9 @@ __global__ void __launch_bounds__(kThreads, 1) decode_kernel(const __grid_consta
   }
   if (tid >= 32 && tid < 32 + a.G && n_c > 0) {  // same for the small operands of the similarity
     const int g = tid - 32;
-    asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(Cq + ((size_t)(hq0 + g) * a.n_cal + c_begin) * kD),
-                 "r"((unsigned)n_c * kRowBytes)
+    asm volatile("cp.async.bulk.prefetch.L2.global.L2::cache_hint [%0], %1, %2;" ::"l"(
+                     Cq + ((size_t)(hq0 + g) * a.n_cal + c_begin) * kD),
+                 "r"((unsigned)n_c * kRowBytes), "l"(pol_keep)
                  : "memory");
     if (g == 0)
       asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(q + (size_t)hq0 * kD),
@@ -279,27 +312,22 @@ __global__ void __launch_bounds__(kThreads, 1) decode_kernel(const __grid_consta
     const int nrows = min(kSlotRows, r1 - row0);
     if (nrows == kSlotRows) {
       mbar_expect_tx(bar, kSlotBytes);
-      tma_load_3d(dst, &TM.k64, bar, 0, row0, unit);
-      tma_load_3d(dst + kPlaneBytes, &TM.k64, bar, 64, row0, unit);
-      tma_load_3d(dst + 2 * kPlaneBytes, &TM.v64, bar, 0, row0, unit);
-      tma_load_3d(dst + 3 * kPlaneBytes, &TM.v64, bar, 64, row0, unit);
+      tma_load_3d(dst, &TM.k64, bar, 0, row0, unit, pol_stream);
+      tma_load_3d(dst + kPlaneBytes, &TM.k64, bar, 64, row0, unit, pol_stream);
+      tma_load_3d(dst + 2 * kPlaneBytes, &TM.v64, bar, 0, row0, unit, pol_stream);
+      tma_load_3d(dst + 3 * kPlaneBytes, &TM.v64, bar, 64, row0, unit, pol_stream);
     } else {
       const int nb = (nrows + kBlkRows - 1) / kBlkRows;
       mbar_expect_tx(bar, (uint32_t)nb * 4u * kBlkRows * 128u);
       for (int j = 0; j < nb; ++j) {
         const uint32_t dj = dst + j * kBlkRows * 128;
-        tma_load_3d(dj, &TM.k16, bar, 0, row0 + j * kBlkRows, unit);
-        tma_load_3d(dj + kPlaneBytes, &TM.k16, bar, 64, row0 + j * kBlkRows, unit);
-        tma_load_3d(dj + 2 * kPlaneBytes, &TM.v16, bar, 0, row0 + j * kBlkRows, unit);
-        tma_load_3d(dj + 3 * kPlaneBytes, &TM.v16, bar, 64, row0 + j * kBlkRows, unit);
+        tma_load_3d(dj, &TM.k16, bar, 0, row0 + j * kBlkRows, unit, pol_stream);
+        tma_load_3d(dj + kPlaneBytes, &TM.k16, bar, 64, row0 + j * kBlkRows, unit, pol_stream);
+        tma_load_3d(dj + 2 * kPlaneBytes, &TM.v16, bar, 0, row0 + j * kBlkRows, unit, pol_stream);
+        tma_load_3d(dj + 3 * kPlaneBytes, &TM.v16, bar, 64, row0 + j * kBlkRows, unit, pol_stream);
       }
     }
   };
-  if (warp == kStreamWarps) {
-    if (lane == 0)
-      for (int sb = 0; sb < min(n_sb, kSlots); ++sb) fill(sb);
-    __syncwarp();
-  }
 
   // ---- (1) cosine similarities of this CTA's calibration rows: four lanes per (head, row) pair,
   // 72 pairs per pass; the best pair per head goes to s_best while the first slots are in flight
@@ -312,8 +340,10 @@ __global__ void __launch_bounds__(kThreads, 1) decode_kernel(const __grid_consta
       const int g = pi % a.G, c = c_begin + pi / a.G;
       const uint4* qp = reinterpret_cast<const uint4*>(q + (size_t)(hq0 + g) * kD + sub4 * 32);
       const uint4* cp = reinterpret_cast<const uint4*>(Cq + ((size_t)(hq0 + g) * a.n_cal + c) * kD + sub4 * 32);
-      r[0].q0 = __ldg(qp); r[0].q1 = __ldg(qp + 1); r[0].c0 = __ldg(cp); r[0].c1 = __ldg(cp + 1);
-      r[1].q0 = __ldg(qp + 2); r[1].q1 = __ldg(qp + 3); r[1].c0 = __ldg(cp + 2); r[1].c1 = __ldg(cp + 3);
+      r[0].q0 = __ldg(qp); r[0].q1 = __ldg(qp + 1);
+      r[0].c0 = ldg_keep(cp, pol_keep); r[0].c1 = ldg_keep(cp + 1, pol_keep);
+      r[1].q0 = __ldg(qp + 2); r[1].q1 = __ldg(qp + 3);
+      r[1].c0 = ldg_keep(cp + 2, pol_keep); r[1].c1 = ldg_keep(cp + 3, pol_keep);
     }
   };
   auto rho_finish = [&](int pi, const RhoLoad (&r)[2]) {
@@ -346,13 +376,29 @@ __global__ void __launch_bounds__(kThreads, 1) decode_kernel(const __grid_consta
   {
     RhoLoad rl[2];
     rho_load(tid >> 2, rl);
+    // the first ring fills go out behind the (small) similarity loads, not ahead of them
+    if (warp == kStreamWarps) {
+      if (lane == 0)
+        for (int sb = 0; sb < min(n_sb, kSlots); ++sb) fill(sb);
+      __syncwarp();
+    }
     rho_finish(tid >> 2, rl);
     for (int base = kPairsPerPass; base < pairs; base += kPairsPerPass) {
       rho_load(base + (tid >> 2), rl);
       rho_finish(base + (tid >> 2), rl);
     }
   }
-  cluster_arrive();  // (A) this CTA's s_best is final
+  // (A) this CTA's s_best is final.  Publishing it to the cluster takes a release fence, which is
+  // slow while the stream is in flight; the stream warps therefore only hand their updates to the
+  // producer warp through a CTA barrier and arrive relaxed, and the producer warp, which has time,
+  // makes the one release for the CTA.
+  if (warp == kStreamWarps) {
+    asm volatile("barrier.cta.sync 1, %0;" ::"n"(kThreads) : "memory");
+    cluster_arrive();
+  } else {
+    asm volatile("barrier.cta.arrive 1, %0;" ::"n"(kThreads) : "memory");
+    asm volatile("barrier.cluster.arrive.relaxed.aligned;" ::: "memory");
+  }
 
   float o[kD / 16][4];
 #pragma unroll
@@ -473,8 +519,8 @@ __global__ void __launch_bounds__(kThreads, 1) decode_kernel(const __grid_consta
   if (early && tid < n_items) {
     const int g = tid / dpc, d = split * dpc + tid % dpc;
     const size_t crow = (size_t)(hq0 + g) * a.n_cal + (unsigned)(s_bestall[g] & 0xffffffffull);
-    lse_c_early = __ldg(P.LSE_c + crow);
-    oc_early = __ldg(P.O_c + crow * kD + d);
+    lse_c_early = ldg_keep(P.LSE_c + crow, pol_keep);
+    oc_early = ldg_keep(P.O_c + crow * kD + d, pol_keep);
   }
 
   // ---- (5) CTA combine of the eight stream warps, pushed to the owners of the output slices:
