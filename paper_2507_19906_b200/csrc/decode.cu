@@ -253,7 +253,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_kernel(const __grid_consta
 
   // ---- (0) overlap with the kernel ahead of this one in the stream.  Until the dependency wait
   // nothing the predecessor may have written is read and nothing global is written; the only
-  // early global work is an L2 prefetch of this CTA's slice of the retained cache, which cannot
+  // early global work is an L2 prefetch of the head of this CTA's slice of the retained cache, which cannot
   // observe stale data (L2 is the point of coherence) and turns the later TMA stream into L2 hits.
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   // calibration rows of this CTA: the contiguous range [c_begin, c_begin + n_c)
@@ -270,7 +270,10 @@ __global__ void __launch_bounds__(kThreads, 1) decode_kernel(const __grid_consta
     s_abort = 0;
   }
   if (warp == kStreamWarps && lane == 0) {
-    const int n_old = min(r1, a.kv_len) - r0;  // rows already in the cache (the appended row is not)
+    // Only the head of the slice is prefetched, about what HBM delivers until the dependency wait
+    // is released: a deeper prefetch queues so much in the memory system that the small, latency-
+    // critical loads of q and C_q behind it come back late (measured: 3/8 of the slice is best).
+    const int n_old = min(min(r1, a.kv_len) - r0, (3 * a.rows_per_split + 7) / 8);
     if (n_old > 0) {
       const unsigned bytes = (unsigned)n_old * kRowBytes;
       asm volatile("cp.async.bulk.prefetch.L2.global.L2::cache_hint [%0], %1, %2;" ::"l"(Kc + (size_t)r0 * kRowBytes),
@@ -415,6 +418,18 @@ __global__ void __launch_bounds__(kThreads, 1) decode_kernel(const __grid_consta
       }
     }
     __syncwarp();
+    // with the last fill under way the producer has nothing left to move: it settles the
+    // calibration row (best similarity over the cluster, ties to the largest row index) while the
+    // stream warps are still busy
+    cluster_wait();  // (A) every CTA's s_best can be read
+    if (lane < a.G) {
+      unsigned long long best = 0ull;
+      for (int s = 0; s < a.nsplit; ++s) {
+        const unsigned long long k = *cluster.map_shared_rank(&s_best[lane], s);
+        best = k > best ? k : best;
+      }
+      s_bestall[lane] = best;
+    }
   } else {
     // ---- (3) stream warps
     const int group = warp >> 2, sub = warp & 3;
@@ -490,30 +505,23 @@ __global__ void __launch_bounds__(kThreads, 1) decode_kernel(const __grid_consta
     }
   }
 
-  // ---- (4) the calibration row: best similarity over the cluster, ties to the largest row
-  // index; the chosen O_c row and LSE_c start their way into L2 while the partials are combined
-  cluster_wait();  // (A) every CTA's s_best can be read
-  if (tid < a.G) {
-    unsigned long long best = 0ull;
-    for (int s = 0; s < a.nsplit; ++s) {
-      const unsigned long long k = *cluster.map_shared_rank(&s_best[tid], s);
-      best = k > best ? k : best;
-    }
-    s_bestall[tid] = best;
-    if (a.nclu == 1 && a.G * (kD / a.nsplit) > kThreads) {
-      const size_t crow = (size_t)(hq0 + tid) * a.n_cal + (unsigned)(best & 0xffffffffull);
-      const float* orow = P.O_c + crow * kD;
-#pragma unroll
-      for (int i = 0; i < 4; ++i) asm volatile("prefetch.global.L2 [%0];" ::"l"(orow + i * 32));
-      asm volatile("prefetch.global.L2 [%0];" ::"l"(P.LSE_c + crow));
-    }
-  }
+  // ---- (4) the chosen O_c elements and LSE_c start their way while the partials are combined
+  if (warp < kStreamWarps) cluster_wait();  // (A): the stream warps only pass it
   __syncthreads();  // all warps are done with the ring: reuse it for the combine
   const int dpc = kD / a.nsplit;
   const int n_items = a.G * dpc;
   const bool single = a.nclu == 1;
   // the common case has one output element per thread at most: its O_c element and LSE_c are
   // loaded now and arrive while the partials are combined
+  if (!single || n_items > kThreads) {
+    if (tid < a.G && single) {
+      const size_t crow = (size_t)(hq0 + tid) * a.n_cal + (unsigned)(s_bestall[tid] & 0xffffffffull);
+      const float* orow = P.O_c + crow * kD;
+#pragma unroll
+      for (int i = 0; i < 4; ++i) asm volatile("prefetch.global.L2 [%0];" ::"l"(orow + i * 32));
+      asm volatile("prefetch.global.L2 [%0];" ::"l"(P.LSE_c + crow));
+    }
+  }
   const bool early = single && n_items <= kThreads;
   float lse_c_early = 0.f, oc_early = 0.f;
   if (early && tid < n_items) {
