@@ -64,7 +64,10 @@ calib_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
   __shared__ Ctl ctl;
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int cta = blockIdx.x;
+  // CTAs come in groups of n_cblocks: the members of a group walk the same (kv unit, key tile)
+  // range at the same pace, one calibration row block each, so that a K/V tile fetched for one
+  // of them is still in L2 when the others ask for it and crosses the HBM interface once.
+  const int cta = blockIdx.x / a.n_cblocks, cb = blockIdx.x % a.n_cblocks;
   const int g_begin = cta * a.tiles_per_cta;
   const int g_end = min(a.total_tiles, g_begin + a.tiles_per_cta);
   const int nt = g_end - g_begin;
@@ -114,7 +117,8 @@ calib_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
 
   // first tile of a run of tiles of one virtual unit inside this CTA's range
   // (the position inside the tile space is tracked incrementally: no division per tile)
-  const int vu_begin = g_begin / a.n_tiles, tile_begin = g_begin - vu_begin * a.n_tiles;
+  const int unit_begin = g_begin / a.n_tiles, tile_begin = g_begin - unit_begin * a.n_tiles;
+  const int vu_begin = unit_begin * a.n_cblocks + cb;
   auto seg_first = [&](int i, int tile) { return i == 0 || tile == 0; };
   auto seg_last = [&](int i, int tile) { return i == nt - 1 || tile == a.n_tiles - 1; };
 
@@ -124,9 +128,9 @@ calib_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
       tma_prefetch_desc(&q_map);
       tma_prefetch_desc(&k_map);
       tma_prefetch_desc(&v_map);
-      int seg = 0, vu = vu_begin, tile = tile_begin, unit = vu_begin / a.n_cblocks;
+      int seg = 0, vu = vu_begin, tile = tile_begin, unit = unit_begin;
       for (int i = 0; i < nt; ++i, ++tile) {
-        if (tile == a.n_tiles) { tile = 0; ++vu; unit = vu / a.n_cblocks; }
+        if (tile == a.n_tiles) { tile = 0; ++unit; vu += a.n_cblocks; }
         if (seg_first(i, tile)) {
           // the Q_c block of the next virtual unit replaces the current one once its MMAs are done
           if (seg > 0 && !mbar_wait(&ctl, q_empty, (seg - 1) & 1, 20u | ((unsigned)i << 8))) break;
@@ -238,7 +242,7 @@ calib_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
       w = __all_sync(0xffffffffu, w);
       if (!w) return false;
       tc_fence_after_sync();
-      const int slot = cta - (vu * a.n_tiles) / a.tiles_per_cta;
+      const int slot = cta - ((vu / a.n_cblocks) * a.n_tiles) / a.tiles_per_cta;
       const size_t part = (size_t)vu * a.max_slots + slot;
       float* orow = a.o_part + (part * 128 + r) * kD;
 #pragma unroll 1
@@ -271,9 +275,9 @@ calib_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
     };
 
     const uint32_t* bm_all = a.bitmap;
-    int vu = vu_begin, tile = tile_begin, unit = vu_begin / a.n_cblocks;
+    int vu = vu_begin, tile = tile_begin, unit = unit_begin;
     for (int i = 0; i < nt; ++i, ++tile) {
-      if (tile == a.n_tiles) { tile = 0; ++vu; unit = vu / a.n_cblocks; }
+      if (tile == a.n_tiles) { tile = 0; ++unit; vu += a.n_cblocks; }
       if (vu != cur_vu) {
         if (cur_vu >= 0) {
           ok = store_partial(cur_vu);
@@ -364,7 +368,7 @@ calib_reduce_kernel(const __nv_bfloat16* __restrict__ Q_obs, const float* __rest
   const int Hkv = Hq / G, h = hq / G, g = hq % G;
   const int unit = b * Hkv + h, cb = g / gpb, r = (g % gpb) * n_cal + c;
   const int vu = unit * n_cblocks + cb;
-  const int first = (vu * n_tiles) / tiles_per_cta, last = ((vu + 1) * n_tiles - 1) / tiles_per_cta;
+  const int first = (unit * n_tiles) / tiles_per_cta, last = ((unit + 1) * n_tiles - 1) / tiles_per_cta;
   const size_t part0 = (size_t)vu * max_slots;
   float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
   float l = 0.f;
@@ -400,9 +404,12 @@ void calib_tc_plan(const CompressGeom& g, int* gpb, int* n_cblocks, int* tiles_p
   *gpb = per;
   *n_cblocks = (g.G + per - 1) / per;
   const int n_tiles = (g.n_cand + kTileKeys - 1) / kTileKeys;
-  const int total = g.units * *n_cblocks * n_tiles;
-  const int ctas = total < kSms ? total : kSms;
-  *tiles_per_cta = (total + ctas - 1) / ctas;
+  // the (kv unit, tile) space is shared out over groups of n_cblocks CTAs
+  const int total = g.units * n_tiles;
+  int groups = kSms / *n_cblocks;
+  if (groups < 1) groups = 1;
+  if (groups > total) groups = total;
+  *tiles_per_cta = (total + groups - 1) / groups;
   *max_slots = (n_tiles + *tiles_per_cta - 1) / *tiles_per_cta + 1;
   *parts = (size_t)g.units * *n_cblocks * *max_slots;
 }
@@ -415,7 +422,7 @@ cudaError_t launch_calib_tc(const CompressGeom& g, const CompressWs& ws, const v
   size_t parts;
   calib_tc_plan(g, &a.gpb, &a.n_cblocks, &a.tiles_per_cta, &a.max_slots, &parts);
   a.n_tiles = (g.n_cand + kTileKeys - 1) / kTileKeys;
-  a.total_tiles = g.units * a.n_cblocks * a.n_tiles;
+  a.total_tiles = g.units * a.n_tiles;
   a.bitmap_words = g.bitmap_words;
   a.scale2 = g.scale2;
   a.row_lse = row_lse;
@@ -443,7 +450,7 @@ cudaError_t launch_calib_tc(const CompressGeom& g, const CompressWs& ws, const v
     if (e != cudaSuccess) return e;
     if (dev >= 0 && dev < 64) attr_set[dev] = true;
   }
-  const int grid = (a.total_tiles + a.tiles_per_cta - 1) / a.tiles_per_cta;
+  const int grid = (a.total_tiles + a.tiles_per_cta - 1) / a.tiles_per_cta * a.n_cblocks;
   calib_tc_kernel<<<grid, kThreads, kSmemBytes, st>>>(qm, km, vm, a);
   const int total = g.B * g.Hq * g.n_cal;
   calib_reduce_kernel<<<(total + 3) / 4, 128, 0, st>>>((const __nv_bfloat16*)Q_obs, row_lse, a.o_part, a.l_part, O_c,
