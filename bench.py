@@ -37,7 +37,7 @@ UNIT = "GB/s"
 FALLBACK_HBM_GBS, FALLBACK_BF16_TFLOPS = 6650.0, 1590.0
 # dram__bytes_read.sum + dram__bytes_write.sum per decode launch at config 3 from the committed ncu
 # capture (profiles/decode_kernel_config3.md); reported only for that workload.
-DECODE_DRAM_TRAFFIC_PER_LAUNCH = 35854080
+DECODE_DRAM_TRAFFIC_PER_LAUNCH = 35865216
 
 
 def load_peaks():
@@ -63,6 +63,35 @@ def compress_flops(cfg, n_cal):
     P.V (the logits of the calibration rows are already part of the scoring)."""
     E = cfg.L - cfg.budget
     return 2 * cfg.B * cfg.Hq * cfg.window * cfg.L * cfg.D + 2 * cfg.B * cfg.Hq * n_cal * E * cfg.D
+
+
+def max_over_ranks(values, world, device):
+    """Multi-GPU timing rule: every rank contributes its device-measured times and all of them
+    continue with the maximum over the ranks (one all-reduce on the job's process group)."""
+    import torch
+    t = torch.tensor(list(values), dtype=torch.float64, device=device)
+    if world > 1:
+        import torch.distributed as dist
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(x) for x in t.cpu()]
+
+
+def whole_job_rate(units_per_rank, world, time_ms):
+    """Replicas only: every rank processes the same number of units, the job's rate is all of them
+    over the slowest rank's time."""
+    return units_per_rank * world / (time_ms * 1e-3)
+
+
+def compress_exps(cfg, n_cal):
+    """Exponentials the path evaluates per layer when the caller supplies no row LSE: one per
+    logit in the statistics pass and in the vote pass, one per (calibration row, candidate)."""
+    E = cfg.L - cfg.budget
+    return 2 * cfg.B * cfg.Hq * cfg.window * cfg.L + cfg.B * cfg.Hq * n_cal * E
+
+
+# special-function pipe: 16 results per clock per SM (measured with a dependent-free ex2 loop),
+# 148 SMs, at the maximum SM clock
+XU_PER_CLK_PER_SM, N_SMS, SM_MAX_HZ = 16, 148, 1.965e9
 
 
 def compress_bytes(cfg):
@@ -242,10 +271,7 @@ def run_gpu(args):
     t_comp = sum(e[0].elapsed_time(e[1]) for e in ev)   # ms over all timed steps
     t_dec = sum(e[1].elapsed_time(e[2]) for e in ev)
     t_tot = sum(e[0].elapsed_time(e[2]) for e in ev)
-    times = torch.tensor([t_comp, t_dec, t_tot], dtype=torch.float64, device="cuda")
-    if world > 1:
-        dist.all_reduce(times, op=dist.ReduceOp.MAX)
-    t_comp, t_dec, t_tot = (float(x) for x in times.cpu())
+    t_comp, t_dec, t_tot = max_over_ranks([t_comp, t_dec, t_tot], world, "cuda")
 
     dec_bytes_step = sum(decode_bytes(cfg, n_cal, cfg.budget + t + 1) for t in range(T)) * S
     dec_launches = T * (1 if args.batched_decode else S) * args.steps
@@ -286,14 +312,11 @@ def run_gpu(args):
         e1.record()
         barrier()
         tot_ms = e0.elapsed_time(e1)
-        tt = torch.tensor([tot_ms], dtype=torch.float64, device="cuda")
-        if world > 1:
-            dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        tot_ms = float(tt.cpu())
+        tot_ms = max_over_ranks([tot_ms], world, "cuda")[0]
         h2d = S * (cfg.B * cfg.Hq * cfg.window * cfg.D * 2 + 2 * cfg.B * cfg.Hkv * cfg.L * cfg.D * 2) + \
             T * S * (cfg.B * cfg.Hq * cfg.D * 2 + 2 * cfg.B * cfg.Hkv * cfg.D * 2)
         d2h = S * (kept_h.numel() * 4 + Oc_h.numel() * 4 + Lc_h.numel() * 4) + T * S * out_h.numel() * 2
-        e2e = {"value": dec_bytes_step * args.e2e_steps / (tot_ms * 1e-3) / 1e9 * world, "unit": UNIT,
+        e2e = {"value": whole_job_rate(dec_bytes_step * args.e2e_steps, world, tot_ms) / 1e9, "unit": UNIT,
                "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h),
                "ms_per_step": tot_ms / args.e2e_steps,
                "note": "decode algorithmic bytes / whole end-to-end step time (host copies of the prompt "
@@ -312,7 +335,7 @@ def run_gpu(args):
     avg_launch_s = t_dec * 1e-3 / dec_launches
     bytes_per_launch = dec_bytes_step / (T * (1 if args.batched_decode else S))
     result = {
-        "metric": METRIC, "value": dec_gbs * world, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "metric": METRIC, "value": whole_job_rate(dec_bytes_step * args.steps, world, t_dec) / 1e9, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": t_tot / args.steps, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
         "config": {"workload": f"config {args.config}: B{cfg.B} {cfg.Hq}q/{cfg.Hkv}kv D128 prefix {cfg.L} "
@@ -332,7 +355,10 @@ def run_gpu(args):
         "compress": {"ms_per_layer": comp_ms_layer, "algorithmic_tflops": comp_tflops,
                      "frac_of_bf16_peak_burst": comp_tflops / peaks["bf16_tflops"],
                      "frac_of_bf16_peak_sustained": comp_tflops / peaks["bf16_tflops_sustained"],
-                     "min_bytes_gbs": comp_gbs, "frac_of_measured_hbm": comp_gbs / peaks["hbm_gbs"]},
+                     "min_bytes_gbs": comp_gbs, "frac_of_measured_hbm": comp_gbs / peaks["hbm_gbs"],
+                     "exp_per_s": compress_exps(cfg, n_cal) / (comp_ms_layer * 1e-3),
+                     "frac_of_xu_peak": compress_exps(cfg, n_cal) / (comp_ms_layer * 1e-3)
+                     / (XU_PER_CLK_PER_SM * N_SMS * SM_MAX_HZ)},
         "roofline": {"bound": "hbm", "kernel": "decode_kernel", "achieved": dec_gbs, "peak": peaks["hbm_gbs"],
                      "unit": "GB/s", "frac": dec_gbs / peaks["hbm_gbs"], "peak_source": peaks["source"],
                      "traffic": DECODE_DRAM_TRAFFIC_PER_LAUNCH
