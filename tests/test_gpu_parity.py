@@ -319,3 +319,53 @@ def test_config4_layers_sampled_units(cuda_lib):
 def test_config5_sampled_unit(cuda_lib):
     cfg = wl.CONFIGS[5]
     _sampled_units_check(cfg, 0, n_cal=64, units=[(0, 2)], steps=4, step_ids={3})
+
+
+# ---------------------------------------------------------------- decode on hand-built states
+@pytest.mark.parametrize("B,Hq,Hkv,kv0,steps,n_cal", [
+    (1, 4, 2, 0, 6, 3),       # the cache starts empty: the first step attends to its own row alone
+    (2, 8, 2, 60, 8, 2),      # the appended row crosses the first 64-row slot boundary
+    (1, 7, 1, 1020, 10, 5),   # ... and a 16-row block boundary deep in a long slice (one unit: eight clusters)
+    (3, 8, 8, 250, 4, 1),     # 24 units: clusters of 4, slices of about 64 rows
+])
+def test_decode_ignores_cache_rows_beyond_kv_len(cuda_lib, B, Hq, Hkv, kv0, steps, n_cal):
+    """The cache rows at and beyond kv_len belong to the caller and may hold anything; here they
+    hold NaN bit patterns.  Every step must still match the oracle, which never reads them."""
+    from paper_2507_19906_b200 import binding as cd
+    rng = np.random.Generator(np.random.Philox(key=[77, B * 1000 + kv0]))
+    D, cap = 128, max(kv0 + steps, 64)
+    bits = lambda x: wl.f32_to_bf16_bits(np.ascontiguousarray(x, dtype=np.float32))
+    budget = min(cap, max(kv0, 16))
+    p = cd.make_params(B=B, Hq=Hq, Hkv=Hkv, L=budget + 64, window=8, pool=7, budget=budget, n_cal=n_cal, cap=cap)
+    st = cd.alloc_layer_state(p)
+    Kk = np.full((B, Hkv, cap, D), 0x7FC0, dtype=np.uint16)   # quiet NaN everywhere ...
+    Vk = np.full((B, Hkv, cap, D), 0x7FC0, dtype=np.uint16)
+    Kk[:, :, :kv0] = bits(rng.standard_normal((B, Hkv, kv0, D)))   # ... except the valid rows
+    Vk[:, :, :kv0] = bits(rng.standard_normal((B, Hkv, kv0, D)))
+    Cq = bits(rng.standard_normal((B, Hq, n_cal, D)))
+    Oc = rng.standard_normal((B, Hq, n_cal, D)).astype(np.float32)
+    Lc = (rng.standard_normal((B, Hq, n_cal)) + 3.0).astype(np.float32)
+    st.K_kept.copy_(to_dev(Kk)); st.V_kept.copy_(to_dev(Vk)); st.C_q.copy_(to_dev(Cq))
+    st.O_c.copy_(torch.from_numpy(Oc)); st.LSE_c.copy_(torch.from_numpy(Lc))
+    out = torch.empty((B, Hq, D), dtype=torch.bfloat16, device="cuda")
+    lse = torch.empty((B, Hq), dtype=torch.float32, device="cuda")
+    flags = torch.empty((B, Hq), dtype=torch.uint8, device="cuda")
+    p.theta1, p.theta2 = 0.7, -1.0                                  # always merge: O_c and LSE_c matter
+    for t in range(steps):
+        # queries close to a calibration query half of the time, so that both rows get chosen
+        q = bits(wl.bf16_bits_to_f32(Cq[:, :, t % n_cal]) + 0.5 * rng.standard_normal((B, Hq, D)).astype(np.float32))
+        kn, vn = bits(rng.standard_normal((B, Hkv, D))), bits(rng.standard_normal((B, Hkv, D)))
+        cd.calidrop_decode(p, to_dev(q), to_dev(kn), to_dev(vn), st.K_kept, st.V_kept, kv0 + t, st.O_c, st.LSE_c,
+                           st.C_q, out, lse, flags, st.ws_decode)
+        torch.cuda.synchronize()
+        o = oracle.decode(q, kn, vn, Kk, Vk, kv0 + t, Oc, Lc, Cq, theta1=0.7, theta2=-1.0)
+        got = wl.bf16_bits_to_f64(to_bits(out))
+        gf = flags.cpu().numpy()
+        same = (gf >> 2) == (o.flags >> 2)
+        assert same.mean() > 0.9                                    # row choice may differ only at near-ties
+        assert_close_out(got[same], o.out[same], f"step {t}")
+        assert_close_lse(lse.cpu().numpy()[same], o.lse[same], f"step {t} lse")
+        # the appended row reached the cache, bit for bit, and nothing else was written
+        np.testing.assert_array_equal(to_bits(st.K_kept)[:, :, :kv0 + t + 1], Kk[:, :, :kv0 + t + 1])
+        np.testing.assert_array_equal(to_bits(st.V_kept)[:, :, :kv0 + t + 1], Vk[:, :, :kv0 + t + 1])
+        np.testing.assert_array_equal(to_bits(st.K_kept)[:, :, kv0 + t + 1:], Kk[:, :, kv0 + t + 1:])
