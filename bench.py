@@ -82,11 +82,12 @@ def whole_job_rate(units_per_rank, world, time_ms):
     return units_per_rank * world / (time_ms * 1e-3)
 
 
-def compress_exps(cfg, n_cal):
-    """Exponentials the path evaluates per layer when the caller supplies no row LSE: one per
-    logit in the statistics pass and in the vote pass, one per (calibration row, candidate)."""
+def compress_exps(cfg, n_cal, lse_supplied=False):
+    """Exponentials the path evaluates per layer: one per logit in the vote pass (and in the
+    statistics pass when the caller supplies no row LSE), one per (calibration row, candidate)."""
     E = cfg.L - cfg.budget
-    return 2 * cfg.B * cfg.Hq * cfg.window * cfg.L + cfg.B * cfg.Hq * n_cal * E
+    passes = 1 if lse_supplied else 2
+    return passes * cfg.B * cfg.Hq * cfg.window * cfg.L + cfg.B * cfg.Hq * n_cal * E
 
 
 # special-function pipe: 16 results per clock per SM (measured with a dependent-free ex2 loop),
@@ -201,11 +202,24 @@ def run_gpu(args):
     lses = [torch.empty((cfg.B, cfg.Hq), dtype=torch.float32, device="cuda") for _ in range(S)]
     flgs = [torch.empty((cfg.B, cfg.Hq), dtype=torch.uint8, device="cuda") for _ in range(S)]
 
+    lse_in = [None] * NI
+    if args.lse_obs:
+        # what a prefill attention kernel would hand over: here taken from an untimed compress call
+        lay = cd.calidrop_compress_workspace_layout(p)
+        n_lse = cfg.B * cfg.Hq * cfg.window
+        for i in range(NI):
+            Qd, Kd, Vd = inputs[i]
+            st = states[0]
+            cd.calidrop_compress(p, Qd, Kd, Vd, None, st.kept_idx, st.K_kept, st.V_kept, st.O_c, st.LSE_c,
+                                 st.C_q, st.ws_compress)
+            torch.cuda.synchronize()
+            lse_in[i] = st.ws_compress[lay.row_lse_offset:lay.row_lse_offset + 4 * n_lse].view(torch.float32).clone()
+
     def compress_phase():
         for s, st in enumerate(states):
             Qd, Kd, Vd = inputs[s % NI]
-            cd.calidrop_compress(p, Qd, Kd, Vd, None, st.kept_idx, st.K_kept, st.V_kept, st.O_c, st.LSE_c,
-                                 st.C_q, st.ws_compress)
+            cd.calidrop_compress(p, Qd, Kd, Vd, lse_in[s % NI], st.kept_idx, st.K_kept, st.V_kept, st.O_c,
+                                 st.LSE_c, st.C_q, st.ws_compress)
 
     if args.batched_decode:
         # one launch per decode step covering all layer states (calidrop_decode_batched)
@@ -344,7 +358,8 @@ def run_gpu(args):
                    "layer_states": S, "prompt_inputs": NI,
                    "l2": f"inputs larger than L2: {S} retained caches ({S * bytes_per_launch / 1e6:.0f} MB) "
                          f"visited round-robin, prompts of {2 * cfg.B * cfg.Hkv * cfg.L * cfg.D * 2 / 1e6:.0f} MB",
-                   "lse_obs": "not supplied (row statistics recomputed inside the step)",
+                   "lse_obs": "supplied by the caller (statistics pass skipped)" if args.lse_obs
+                   else "not supplied (row statistics recomputed inside the step)",
                    "launch": "eager C-ABI calls" if args.no_graph else "CUDA-graph replay of the captured C-ABI calls",
                    "decode_entry": "calidrop_decode_batched over the layer states" if args.batched_decode
                    else "calidrop_decode per layer state",
@@ -356,8 +371,8 @@ def run_gpu(args):
                      "frac_of_bf16_peak_burst": comp_tflops / peaks["bf16_tflops"],
                      "frac_of_bf16_peak_sustained": comp_tflops / peaks["bf16_tflops_sustained"],
                      "min_bytes_gbs": comp_gbs, "frac_of_measured_hbm": comp_gbs / peaks["hbm_gbs"],
-                     "exp_per_s": compress_exps(cfg, n_cal) / (comp_ms_layer * 1e-3),
-                     "frac_of_xu_peak": compress_exps(cfg, n_cal) / (comp_ms_layer * 1e-3)
+                     "exp_per_s": compress_exps(cfg, n_cal, args.lse_obs) / (comp_ms_layer * 1e-3),
+                     "frac_of_xu_peak": compress_exps(cfg, n_cal, args.lse_obs) / (comp_ms_layer * 1e-3)
                      / (XU_PER_CLK_PER_SM * N_SMS * SM_MAX_HZ)},
         "roofline": {"bound": "hbm", "kernel": "decode_kernel", "achieved": dec_gbs, "peak": peaks["hbm_gbs"],
                      "unit": "GB/s", "frac": dec_gbs / peaks["hbm_gbs"], "peak_source": peaks["source"],
@@ -481,6 +496,9 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--batched-decode", action="store_true",
                     help="one calidrop_decode_batched launch per decode step over all layer states")
+    ap.add_argument("--lse-obs", action="store_true",
+                    help="supply the row log-sum-exp of the prefill attention to calidrop_compress (as a prefill "
+                         "kernel would), so the statistics pass is skipped; not the default workload")
     ap.add_argument("--no-graph", action="store_true", help="launch every call eagerly instead of replaying CUDA graphs")
     args = ap.parse_args()
     if args.impl == "reference":

@@ -116,8 +116,8 @@ bool scalar_path_forced() {
   return forced;
 }
 
-// Split-K factor of the decode launch: enough CTAs to fill the machine twice over, never
-// fewer than 32 rows per split.
+// Split-K factor of the decode launch: one CTA per SM at most (a CTA's ring takes most of an SM's
+// shared memory), never fewer than 32 rows per split.
 int decode_nsplit(int units_total, int n_kv) {
   int ns = kDecodeTargetCtas / units_total;
   if (ns < 1) ns = 1;
@@ -128,7 +128,7 @@ int decode_nsplit(int units_total, int n_kv) {
 }
 
 struct DecodeWs {
-  size_t part_o, part_ml, rho, counters, status, per_layer;
+  size_t part_o, part_ml, part_best, counters, status, per_layer;
   int max_split;
 };
 
@@ -140,7 +140,7 @@ DecodeWs make_decode_ws(const calidrop_params* p) {
   w.counters = off; off = align_up(off + (size_t)units * 4 * kDecodeMaxLayers, 256);
   w.status = off;   off += 256;  // error word: nonzero after a bounded wait of the kernel ran out
   w.part_ml = off;  off = align_up(off + (size_t)units * w.max_split * kMaxG * 2 * 4, 256);
-  w.rho = off;      off = align_up(off + (size_t)units * kMaxG * w.max_split * 8, 256);
+  w.part_best = off; off = align_up(off + (size_t)units * kMaxG * w.max_split * 8, 256);
   w.part_o = off;   off = align_up(off + (size_t)units * w.max_split * kMaxG * kD * 4, 256);
   w.per_layer = off;
   return w;
