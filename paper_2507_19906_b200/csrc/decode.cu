@@ -300,6 +300,26 @@ __global__ void __launch_bounds__(kThreads, 1) decode_kernel(const __grid_consta
                    : "memory");
   }
   if (tid < kMaxG) s_best[tid] = 0ull;
+  // Address arithmetic of everything that is loaded right after the dependency wait, and of the
+  // finish, is done here: a single warp runs a dependent chain of scalar instructions at a few
+  // cycles each, and at this kernel's scale a hundred of them behind the wait are a measurable
+  // part of a launch (0.4 us each for the similarity loads and for the O_c loads, measured).
+  constexpr int kPairsPerPass = kThreads / 4;
+  const int pairs = n_c * a.G;
+  const int sub4 = tid & 3;
+  const int pi0 = tid >> 2;
+  const int pg0 = pi0 < pairs ? pi0 % a.G : 0, pc0 = c_begin + (pi0 < pairs ? pi0 / a.G : 0);
+  const uint4* qp0 = reinterpret_cast<const uint4*>(q + (size_t)(hq0 + pg0) * kD + sub4 * 32);
+  const uint4* cp0 = reinterpret_cast<const uint4*>(Cq + ((size_t)(hq0 + pg0) * a.n_cal + pc0) * kD + sub4 * 32);
+  const uint32_t* qr0 = reinterpret_cast<const uint32_t*>(q + (size_t)(hq0 + min(gq, a.G - 1)) * kD) + tq;
+  const int dpc = kD / a.nsplit, lg_dpc = 31 - __clz(dpc);  // nsplit is a power of two
+  const int n_items = a.G * dpc;
+  const bool single = a.nclu == 1;
+  const bool early = single && n_items <= kThreads;  // one output element per thread at most
+  const int eg = min(tid >> lg_dpc, a.G - 1), ed = split * dpc + (tid & (dpc - 1));
+  const float* oc_base = P.O_c + (size_t)(hq0 + eg) * a.n_cal * kD + ed;
+  const float* lsec_base = P.LSE_c + (size_t)(hq0 + eg) * a.n_cal;
+  asm volatile("" ::"l"(qp0), "l"(cp0), "l"(qr0), "l"(oc_base), "l"(lsec_base), "r"(pg0), "r"(pc0));
   asm volatile("griddepcontrol.wait;" ::: "memory");
   __syncthreads();
 
@@ -334,9 +354,6 @@ __global__ void __launch_bounds__(kThreads, 1) decode_kernel(const __grid_consta
 
   // ---- (1) cosine similarities of this CTA's calibration rows: four lanes per (head, row) pair,
   // 72 pairs per pass; the best pair per head goes to s_best while the first slots are in flight
-  constexpr int kPairsPerPass = kThreads / 4;
-  const int pairs = n_c * a.G;
-  const int sub4 = tid & 3;
   auto rho_load = [&](int pi, RhoLoad (&r)[2]) {
     r[0] = RhoLoad{}; r[1] = RhoLoad{};
     if (pi < pairs) {
@@ -349,7 +366,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_kernel(const __grid_consta
       r[1].c0 = ldg_keep(cp + 2, pol_keep); r[1].c1 = ldg_keep(cp + 3, pol_keep);
     }
   };
-  auto rho_finish = [&](int pi, const RhoLoad (&r)[2]) {
+  auto rho_finish = [&](int pi, int g, int c, const RhoLoad (&r)[2]) {
     float dot = 0.f, qq = 0.f, cc = 0.f;
     if (pi < pairs) { rho_accumulate(r[0], dot, qq, cc); rho_accumulate(r[1], dot, qq, cc); }
 #pragma unroll
@@ -359,7 +376,6 @@ __global__ void __launch_bounds__(kThreads, 1) decode_kernel(const __grid_consta
       cc += __shfl_xor_sync(0xffffffffu, cc, o);
     }
     if (sub4 == 0 && pi < pairs) {
-      const int g = pi % a.G, c = c_begin + pi / a.G;
       const float rho = (qq > 0.f && cc > 0.f) ? dot / (sqrtf(qq) * sqrtf(cc)) : 0.f;
       atomicMax(&s_best[g], rank_key(rho, c));
     }
@@ -371,24 +387,30 @@ __global__ void __launch_bounds__(kThreads, 1) decode_kernel(const __grid_consta
   for (int kk = 0; kk < kD / 16; ++kk) {
     qa[kk][0] = 0u; qa[kk][1] = 0u;
     if (warp < kStreamWarps && gq < a.G) {
-      const uint32_t* qr = reinterpret_cast<const uint32_t*>(q + (size_t)(hq0 + gq) * kD + kk * 16);
-      qa[kk][0] = __ldg(qr + tq);
-      qa[kk][1] = __ldg(qr + 4 + tq);
+      qa[kk][0] = __ldg(qr0 + kk * 8);
+      qa[kk][1] = __ldg(qr0 + kk * 8 + 4);
     }
   }
   {
     RhoLoad rl[2];
-    rho_load(tid >> 2, rl);
+    rl[0] = RhoLoad{}; rl[1] = RhoLoad{};
+    if (pi0 < pairs) {
+      rl[0].q0 = __ldg(qp0); rl[0].q1 = __ldg(qp0 + 1);
+      rl[0].c0 = ldg_keep(cp0, pol_keep); rl[0].c1 = ldg_keep(cp0 + 1, pol_keep);
+      rl[1].q0 = __ldg(qp0 + 2); rl[1].q1 = __ldg(qp0 + 3);
+      rl[1].c0 = ldg_keep(cp0 + 2, pol_keep); rl[1].c1 = ldg_keep(cp0 + 3, pol_keep);
+    }
     // the first ring fills go out behind the (small) similarity loads, not ahead of them
     if (warp == kStreamWarps) {
       if (lane == 0)
         for (int sb = 0; sb < min(n_sb, kSlots); ++sb) fill(sb);
       __syncwarp();
     }
-    rho_finish(tid >> 2, rl);
+    rho_finish(pi0, pg0, pc0, rl);
     for (int base = kPairsPerPass; base < pairs; base += kPairsPerPass) {
-      rho_load(base + (tid >> 2), rl);
-      rho_finish(base + (tid >> 2), rl);
+      const int pi = base + pi0;
+      rho_load(pi, rl);
+      rho_finish(pi, pi < pairs ? pi % a.G : 0, c_begin + (pi < pairs ? pi / a.G : 0), rl);
     }
   }
   // (A) this CTA's s_best is final.  Publishing it to the cluster takes a release fence, which is
@@ -508,9 +530,6 @@ __global__ void __launch_bounds__(kThreads, 1) decode_kernel(const __grid_consta
   // ---- (4) the chosen O_c elements and LSE_c start their way while the partials are combined
   if (warp < kStreamWarps) cluster_wait();  // (A): the stream warps only pass it
   __syncthreads();  // all warps are done with the ring: reuse it for the combine
-  const int dpc = kD / a.nsplit;
-  const int n_items = a.G * dpc;
-  const bool single = a.nclu == 1;
   // the common case has one output element per thread at most: its O_c element and LSE_c are
   // loaded now and arrive while the partials are combined
   if (!single || n_items > kThreads) {
@@ -522,13 +541,11 @@ __global__ void __launch_bounds__(kThreads, 1) decode_kernel(const __grid_consta
       asm volatile("prefetch.global.L2 [%0];" ::"l"(P.LSE_c + crow));
     }
   }
-  const bool early = single && n_items <= kThreads;
   float lse_c_early = 0.f, oc_early = 0.f;
   if (early && tid < n_items) {
-    const int g = tid / dpc, d = split * dpc + tid % dpc;
-    const size_t crow = (size_t)(hq0 + g) * a.n_cal + (unsigned)(s_bestall[g] & 0xffffffffull);
-    lse_c_early = ldg_keep(P.LSE_c + crow, pol_keep);
-    oc_early = ldg_keep(P.O_c + crow * kD + d, pol_keep);
+    const unsigned cs = (unsigned)(s_bestall[eg] & 0xffffffffull);
+    lse_c_early = ldg_keep(lsec_base + cs, pol_keep);
+    oc_early = ldg_keep(oc_base + (size_t)cs * kD, pol_keep);
   }
 
   // ---- (5) CTA combine of the eight stream warps, pushed to the owners of the output slices:
@@ -561,7 +578,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_kernel(const __grid_consta
       Lsum += wml[(w * kMaxG + g) * 2 + 1] * sc;
       acc += wo[(w * kMaxG + g) * kWoStride + d] * sc;
     }
-    const int owner = d / dpc;
+    const int owner = d >> lg_dpc;
     cluster.map_shared_rank(s_xpart, owner)[(split * kMaxG + g) * dpc + (d - owner * dpc)] = acc;
     if (d < a.nsplit) {  // the (max, sum) pair of this split goes to every CTA of the cluster
       float* xm = &cluster.map_shared_rank(&s_xml[0][0][0], d)[(split * kMaxG + g) * 2];
@@ -575,7 +592,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_kernel(const __grid_consta
   // so no CTA has to wait for another before it leaves)
   const int lu = layer * a.units + unit;
   for (int item = tid; item < n_items; item += kThreads) {
-    const int g = item / dpc, dl = item % dpc, d = split * dpc + dl;
+    const int g = item >> lg_dpc, dl = item & (dpc - 1), d = split * dpc + dl;
     const int hq = hq0 + g;
     const unsigned long long best = s_bestall[g];
     float M = -INFINITY;
