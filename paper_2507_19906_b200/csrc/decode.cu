@@ -320,8 +320,8 @@ __global__ void __launch_bounds__(kThreads, 1) decode_kernel(const __grid_consta
   const float* oc_base = P.O_c + (size_t)(hq0 + eg) * a.n_cal * kD + ed;
   const float* lsec_base = P.LSE_c + (size_t)(hq0 + eg) * a.n_cal;
   asm volatile("" ::"l"(qp0), "l"(cp0), "l"(qr0), "l"(oc_base), "l"(lsec_base), "r"(pg0), "r"(pc0));
+  __syncthreads();  // barriers initialised, s_best cleared: nothing of this needs the predecessor
   asm volatile("griddepcontrol.wait;" ::: "memory");
-  __syncthreads();
 
   // One ring fill: rows [r0 + sb * 64, ...) of K and V into slot sb % 3.  Whole slots take four
   // 64-row boxes; the ragged last slot takes 16-row boxes for the row groups that hold valid rows,
@@ -391,39 +391,38 @@ __global__ void __launch_bounds__(kThreads, 1) decode_kernel(const __grid_consta
       qa[kk][1] = __ldg(qr0 + kk * 8 + 4);
     }
   }
-  {
-    RhoLoad rl[2];
-    rl[0] = RhoLoad{}; rl[1] = RhoLoad{};
-    if (pi0 < pairs) {
-      rl[0].q0 = __ldg(qp0); rl[0].q1 = __ldg(qp0 + 1);
-      rl[0].c0 = ldg_keep(cp0, pol_keep); rl[0].c1 = ldg_keep(cp0 + 1, pol_keep);
-      rl[1].q0 = __ldg(qp0 + 2); rl[1].q1 = __ldg(qp0 + 3);
-      rl[1].c0 = ldg_keep(cp0 + 2, pol_keep); rl[1].c1 = ldg_keep(cp0 + 3, pol_keep);
-    }
-    // the first ring fills go out behind the (small) similarity loads, not ahead of them
-    if (warp == kStreamWarps) {
-      if (lane == 0)
-        for (int sb = 0; sb < min(n_sb, kSlots); ++sb) fill(sb);
-      __syncwarp();
-    }
+  RhoLoad rl[2];
+  rl[0] = RhoLoad{}; rl[1] = RhoLoad{};
+  if (pi0 < pairs) {
+    rl[0].q0 = __ldg(qp0); rl[0].q1 = __ldg(qp0 + 1);
+    rl[0].c0 = ldg_keep(cp0, pol_keep); rl[0].c1 = ldg_keep(cp0 + 1, pol_keep);
+    rl[1].q0 = __ldg(qp0 + 2); rl[1].q1 = __ldg(qp0 + 3);
+    rl[1].c0 = ldg_keep(cp0 + 2, pol_keep); rl[1].c1 = ldg_keep(cp0 + 3, pol_keep);
+  }
+  // the first ring fills go out behind the (small) similarity loads, not ahead of them
+  if (warp == kStreamWarps) {
+    if (lane == 0)
+      for (int sb = 0; sb < min(n_sb, kSlots); ++sb) fill(sb);
+    __syncwarp();
+  }
+  // The similarities are finished by the producer warp at once and by a stream warp after its first
+  // slot, whose data is already there when the query arrives.  (A) then says this CTA's s_best is
+  // final.  Publishing it to the cluster takes a release fence, which is slow while the stream is
+  // in flight; the stream warps therefore only hand their updates to the producer warp through a
+  // CTA barrier and arrive relaxed, and the producer warp, which has time, makes the one release
+  // for the CTA.
+  auto rho_rest = [&]() {
     rho_finish(pi0, pg0, pc0, rl);
     for (int base = kPairsPerPass; base < pairs; base += kPairsPerPass) {
       const int pi = base + pi0;
       rho_load(pi, rl);
       rho_finish(pi, pi < pairs ? pi % a.G : 0, c_begin + (pi < pairs ? pi / a.G : 0), rl);
     }
-  }
-  // (A) this CTA's s_best is final.  Publishing it to the cluster takes a release fence, which is
-  // slow while the stream is in flight; the stream warps therefore only hand their updates to the
-  // producer warp through a CTA barrier and arrive relaxed, and the producer warp, which has time,
-  // makes the one release for the CTA.
-  if (warp == kStreamWarps) {
-    asm volatile("barrier.cta.sync 1, %0;" ::"n"(kThreads) : "memory");
-    cluster_arrive();
-  } else {
-    asm volatile("barrier.cta.arrive 1, %0;" ::"n"(kThreads) : "memory");
-    asm volatile("barrier.cluster.arrive.relaxed.aligned;" ::: "memory");
-  }
+    if (warp != kStreamWarps) {
+      asm volatile("barrier.cta.arrive 1, %0;" ::"n"(kThreads) : "memory");
+      asm volatile("barrier.cluster.arrive.relaxed.aligned;" ::: "memory");
+    }
+  };
 
   float o[kD / 16][4];
 #pragma unroll
@@ -431,6 +430,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_kernel(const __grid_consta
   float m0 = -INFINITY, m1 = -INFINITY, l0 = 0.f, l1 = 0.f;  // heads 2tq and 2tq+1
 
   if (warp == kStreamWarps) {
+    rho_rest();
     // ---- (2) producer: refill a slot as soon as its four warps have released it
     if (lane == 0) {
       for (int sb = kSlots; sb < n_sb; ++sb) {
@@ -443,7 +443,9 @@ __global__ void __launch_bounds__(kThreads, 1) decode_kernel(const __grid_consta
     // with the last fill under way the producer has nothing left to move: it settles the
     // calibration row (best similarity over the cluster, ties to the largest row index) while the
     // stream warps are still busy
-    cluster_wait();  // (A) every CTA's s_best can be read
+    asm volatile("barrier.cta.sync 1, %0;" ::"n"(kThreads) : "memory");  // the stream warps' updates of s_best
+    cluster_arrive();  // (A) with the release for the whole CTA
+    cluster_wait();    //     every CTA's s_best can be read
     if (lane < a.G) {
       unsigned long long best = 0ull;
       for (int s = 0; s < a.nsplit; ++s) {
@@ -456,6 +458,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_kernel(const __grid_consta
     // ---- (3) stream warps
     const int group = warp >> 2, sub = warp & 3;
     const int mid = lane >> 3;
+    bool rho_done = false;
     for (int sb = group; sb < n_sb; sb += 2) {
       const int s = sb % kSlots, k = sb / kSlots;
       const bool ok = mbar_wait(smem_u32(&s_full[s][k & 1]), (k >> 1) & 1, abort_flag, a.status, 0x200u + sb);
@@ -519,7 +522,9 @@ __global__ void __launch_bounds__(kThreads, 1) decode_kernel(const __grid_consta
       }
       __syncwarp();
       if (lane == 0) mbar_arrive(smem_u32(&s_empty[s][k & 1]));  // the slot may be refilled
+      if (!rho_done) { rho_rest(); rho_done = true; }
     }
+    if (!rho_done) rho_rest();
 #pragma unroll
     for (int off = 4; off < 32; off <<= 1) {
       l0 += __shfl_xor_sync(0xffffffffu, l0, off);
