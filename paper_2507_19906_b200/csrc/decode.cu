@@ -570,12 +570,14 @@ __global__ void __launch_bounds__(kThreads, 1) decode_kernel(const __grid_consta
     }
   }
   __syncthreads();
-  for (int idx = tid; idx < a.G * kD; idx += kThreads) {
+  // two elements per thread and pass, their loads and arithmetic interleaved (the pushes are
+  // stores through generic pointers, which the compiler will not move loads across)
+  auto combine_one = [&](int idx, float& M, float& Lsum, float& acc) {
     const int g = idx / kD, d = idx % kD;
-    float M = -INFINITY;
+    M = -INFINITY;
 #pragma unroll
     for (int w = 0; w < kStreamWarps; ++w) M = fmaxf(M, wml[(w * kMaxG + g) * 2]);
-    float Lsum = 0.f, acc = 0.f;
+    Lsum = 0.f; acc = 0.f;
 #pragma unroll
     for (int w = 0; w < kStreamWarps; ++w) {
       const float mw = wml[(w * kMaxG + g) * 2];
@@ -583,12 +585,24 @@ __global__ void __launch_bounds__(kThreads, 1) decode_kernel(const __grid_consta
       Lsum += wml[(w * kMaxG + g) * 2 + 1] * sc;
       acc += wo[(w * kMaxG + g) * kWoStride + d] * sc;
     }
+  };
+  auto push_one = [&](int idx, float M, float Lsum, float acc) {
+    const int g = idx / kD, d = idx % kD;
     const int owner = d >> lg_dpc;
     cluster.map_shared_rank(s_xpart, owner)[(split * kMaxG + g) * dpc + (d - owner * dpc)] = acc;
     if (d < a.nsplit) {  // the (max, sum) pair of this split goes to every CTA of the cluster
       float* xm = &cluster.map_shared_rank(&s_xml[0][0][0], d)[(split * kMaxG + g) * 2];
       xm[0] = M; xm[1] = Lsum;
     }
+  };
+  for (int idx = tid; idx < a.G * kD; idx += 2 * kThreads) {
+    const int idx2 = idx + kThreads;
+    const bool two = idx2 < a.G * kD;
+    float M0, L0, A0, M1 = 0.f, L1 = 0.f, A1 = 0.f;
+    combine_one(idx, M0, L0, A0);
+    if (two) combine_one(idx2, M1, L1, A1);
+    push_one(idx, M0, L0, A0);
+    if (two) push_one(idx2, M1, L1, A1);
   }
   cluster_arrive();  // (B) this CTA's pushes are done
   cluster_wait();    //     and everything pushed to this CTA has arrived
