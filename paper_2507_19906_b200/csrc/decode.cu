@@ -192,17 +192,17 @@ __device__ __forceinline__ void merge_store(const DecodeCommon& a, const DecodeL
                                             float M, float Lsum, unsigned long long best, float lse_c, float oc) {
   const int cs = (int)(unsigned)(best & 0xffffffffull);
   const float rho = rank_key_value(best);
-  float outv = acc / Lsum;       // O_a
-  float lse2 = M + log2f(Lsum);  // LSE_a (log2 domain)
+  float outv = __fdividef(acc, Lsum);  // O_a
+  float lse2 = M + __log2f(Lsum);      // LSE_a (log2 domain)
   const bool apply = (a.always_apply || rho > a.theta2) && (lse_c > -INFINITY);
   if (apply) {
     // alpha_i = e^{LSE_a - LSE}, alpha_j = e^{LSE_c - LSE}; out = alpha_i O_a + alpha_j O_c
     const float lc2 = lse_c * kLog2e;
     const float mx = fmaxf(lse2, lc2);
-    const float ea = exp2f(lse2 - mx), ec = exp2f(lc2 - mx);
-    const float tot = ea + ec;
-    outv = (ea / tot) * outv + (ec / tot) * oc;
-    lse2 = mx + log2f(tot);
+    const float ea = ex2_approx(lse2 - mx), ec = ex2_approx(lc2 - mx);
+    const float inv = __fdividef(1.f, ea + ec);  // the sum is in [1, 2]
+    outv = (ea * inv) * outv + (ec * inv) * oc;
+    lse2 = mx + __log2f(ea + ec);
   }
   reinterpret_cast<__nv_bfloat16*>(P.out)[(size_t)hq * kD + d] = __float2bfloat16_rn(outv);
   if (d == 0) {
