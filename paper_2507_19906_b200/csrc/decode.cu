@@ -570,39 +570,32 @@ __global__ void __launch_bounds__(kThreads, 1) decode_kernel(const __grid_consta
     }
   }
   __syncthreads();
-  // two elements per thread and pass, their loads and arithmetic interleaved (the pushes are
-  // stores through generic pointers, which the compiler will not move loads across)
-  auto combine_one = [&](int idx, float& M, float& Lsum, float& acc) {
-    const int g = idx / kD, d = idx % kD;
-    M = -INFINITY;
+  // 256 threads: thread t owns dimensions (t & 63) and (t & 63) + 64 of head (t >> 6) + 4k, so the
+  // scale factors of the eight warps are worked out once for two elements, and all loads are done
+  // before the pushes (stores through generic pointers, which the compiler will not move loads across)
+  if (tid < 256) {
+    const int dlo = tid & 63;
+    for (int g = tid >> 6; g < a.G; g += 4) {
+      float mw[kStreamWarps], M = -INFINITY;
 #pragma unroll
-    for (int w = 0; w < kStreamWarps; ++w) M = fmaxf(M, wml[(w * kMaxG + g) * 2]);
-    Lsum = 0.f; acc = 0.f;
+      for (int w = 0; w < kStreamWarps; ++w) { mw[w] = wml[(w * kMaxG + g) * 2]; M = fmaxf(M, mw[w]); }
+      float Lsum = 0.f, acc0 = 0.f, acc1 = 0.f;
 #pragma unroll
-    for (int w = 0; w < kStreamWarps; ++w) {
-      const float mw = wml[(w * kMaxG + g) * 2];
-      const float sc = mw > -INFINITY ? ex2_approx(mw - M) : 0.f;
-      Lsum += wml[(w * kMaxG + g) * 2 + 1] * sc;
-      acc += wo[(w * kMaxG + g) * kWoStride + d] * sc;
+      for (int w = 0; w < kStreamWarps; ++w) {
+        const float sc = mw[w] > -INFINITY ? ex2_approx(mw[w] - M) : 0.f;
+        const float* wrow = wo + (w * kMaxG + g) * kWoStride + dlo;
+        Lsum = fmaf(wml[(w * kMaxG + g) * 2 + 1], sc, Lsum);
+        acc0 = fmaf(wrow[0], sc, acc0);
+        acc1 = fmaf(wrow[64], sc, acc1);
+      }
+      const int own0 = dlo >> lg_dpc, own1 = (dlo + 64) >> lg_dpc;
+      cluster.map_shared_rank(s_xpart, own0)[(split * kMaxG + g) * dpc + (dlo - own0 * dpc)] = acc0;
+      cluster.map_shared_rank(s_xpart, own1)[(split * kMaxG + g) * dpc + (dlo + 64 - own1 * dpc)] = acc1;
+      if (dlo < a.nsplit) {  // the (max, sum) pair of this split goes to every CTA of the cluster
+        float* xm = &cluster.map_shared_rank(&s_xml[0][0][0], dlo)[(split * kMaxG + g) * 2];
+        xm[0] = M; xm[1] = Lsum;
+      }
     }
-  };
-  auto push_one = [&](int idx, float M, float Lsum, float acc) {
-    const int g = idx / kD, d = idx % kD;
-    const int owner = d >> lg_dpc;
-    cluster.map_shared_rank(s_xpart, owner)[(split * kMaxG + g) * dpc + (d - owner * dpc)] = acc;
-    if (d < a.nsplit) {  // the (max, sum) pair of this split goes to every CTA of the cluster
-      float* xm = &cluster.map_shared_rank(&s_xml[0][0][0], d)[(split * kMaxG + g) * 2];
-      xm[0] = M; xm[1] = Lsum;
-    }
-  };
-  for (int idx = tid; idx < a.G * kD; idx += 2 * kThreads) {
-    const int idx2 = idx + kThreads;
-    const bool two = idx2 < a.G * kD;
-    float M0, L0, A0, M1 = 0.f, L1 = 0.f, A1 = 0.f;
-    combine_one(idx, M0, L0, A0);
-    if (two) combine_one(idx2, M1, L1, A1);
-    push_one(idx, M0, L0, A0);
-    if (two) push_one(idx2, M1, L1, A1);
   }
   cluster_arrive();  // (B) this CTA's pushes are done
   cluster_wait();    //     and everything pushed to this CTA has arrived
