@@ -224,6 +224,32 @@ __global__ void __launch_bounds__(kThreads, 1) decode_kernel(const __grid_consta
   __shared__ unsigned s_ticket;
 
   const DecodeCommon& a = args.c;
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  // ---- (0) overlap with the kernel ahead of this one in the stream, first thing in the kernel: an
+  // L2 prefetch of the head of this CTA's slice of the retained cache.  Until the dependency wait
+  // nothing the predecessor may have written is read and nothing global is written; a prefetch
+  // cannot observe stale data (L2 is the point of coherence) and turns the head of the later TMA
+  // stream into L2 hits.  Only the head: about what HBM delivers until the dependency wait is
+  // released.  A deeper prefetch queues so much in the memory system that the small, latency-
+  // critical loads of q and C_q behind it come back late (measured: 3/8 of the slice is best).
+  if (threadIdx.x == kStreamWarps * 32) {
+    const int pr0 = min(a.n_kv, (int)blockIdx.x * a.rows_per_split);
+    const int pr1 = min(a.n_kv, pr0 + a.rows_per_split);
+    const int n_old = min(min(pr1, a.kv_len) - pr0, (3 * a.rows_per_split + 7) / 8);
+    if (n_old > 0) {
+      const uint64_t pol = policy_evict_first();
+      const size_t off = ((size_t)blockIdx.y * a.cap + pr0) * kRowBytes;
+      const unsigned bytes = (unsigned)n_old * kRowBytes;
+      asm volatile("cp.async.bulk.prefetch.L2.global.L2::cache_hint [%0], %1, %2;" ::"l"(
+                       (const unsigned char*)args.layer[blockIdx.z].K + off),
+                   "r"(bytes), "l"(pol)
+                   : "memory");
+      asm volatile("cp.async.bulk.prefetch.L2.global.L2::cache_hint [%0], %1, %2;" ::"l"(
+                       (const unsigned char*)args.layer[blockIdx.z].V + off),
+                   "r"(bytes), "l"(pol)
+                   : "memory");
+    }
+  }
   cg::cluster_group cluster = cg::this_cluster();
   const int gs = blockIdx.x;             // split index over the whole unit
   const int split = gs % a.nsplit;       // rank inside the cluster
@@ -251,11 +277,6 @@ __global__ void __launch_bounds__(kThreads, 1) decode_kernel(const __grid_consta
   unsigned char* ring_ptr = smem_raw + (ring - smem_u32(smem_raw));
   volatile int* abort_flag = &s_abort;
 
-  // ---- (0) overlap with the kernel ahead of this one in the stream.  Until the dependency wait
-  // nothing the predecessor may have written is read and nothing global is written; the only
-  // early global work is an L2 prefetch of the head of this CTA's slice of the retained cache, which cannot
-  // observe stale data (L2 is the point of coherence) and turns the later TMA stream into L2 hits.
-  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   // calibration rows of this CTA: the contiguous range [c_begin, c_begin + n_c)
   const int c_per = (a.n_cal + n_gs - 1) / n_gs;
   const int c_begin = min(a.n_cal, gs * c_per);
@@ -270,19 +291,6 @@ __global__ void __launch_bounds__(kThreads, 1) decode_kernel(const __grid_consta
     s_abort = 0;
   }
   if (warp == kStreamWarps && lane == 0) {
-    // Only the head of the slice is prefetched, about what HBM delivers until the dependency wait
-    // is released: a deeper prefetch queues so much in the memory system that the small, latency-
-    // critical loads of q and C_q behind it come back late (measured: 3/8 of the slice is best).
-    const int n_old = min(min(r1, a.kv_len) - r0, (3 * a.rows_per_split + 7) / 8);
-    if (n_old > 0) {
-      const unsigned bytes = (unsigned)n_old * kRowBytes;
-      asm volatile("cp.async.bulk.prefetch.L2.global.L2::cache_hint [%0], %1, %2;" ::"l"(Kc + (size_t)r0 * kRowBytes),
-                   "r"(bytes), "l"(pol_stream)
-                   : "memory");
-      asm volatile("cp.async.bulk.prefetch.L2.global.L2::cache_hint [%0], %1, %2;" ::"l"(Vc + (size_t)r0 * kRowBytes),
-                   "r"(bytes), "l"(pol_stream)
-                   : "memory");
-    }
     asm volatile("prefetch.tensormap [%0];" ::"l"(&TM.k64) : "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(&TM.v64) : "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(&TM.k16) : "memory");
@@ -607,14 +615,21 @@ __global__ void __launch_bounds__(kThreads, 1) decode_kernel(const __grid_consta
     const int g = item >> lg_dpc, dl = item & (dpc - 1), d = split * dpc + dl;
     const int hq = hq0 + g;
     const unsigned long long best = s_bestall[g];
-    float M = -INFINITY;
-    for (int s = 0; s < a.nsplit; ++s) M = fmaxf(M, s_xml[s][g][0]);
+    float ms[8], ls[8], xs[8], M = -INFINITY;
+#pragma unroll
+    for (int s = 0; s < 8; ++s) {  // all loads first (nsplit <= 8)
+      const bool on = s < a.nsplit;
+      ms[s] = on ? s_xml[s][g][0] : -INFINITY;
+      ls[s] = on ? s_xml[s][g][1] : 0.f;
+      xs[s] = on ? s_xpart[(s * kMaxG + g) * dpc + dl] : 0.f;
+      M = fmaxf(M, ms[s]);
+    }
     float Lsum = 0.f, acc = 0.f;
-    for (int s = 0; s < a.nsplit; ++s) {
-      const float ms = s_xml[s][g][0];
-      const float sc = ms > -INFINITY ? ex2_approx(ms - M) : 0.f;
-      Lsum = fmaf(s_xml[s][g][1], sc, Lsum);
-      acc = fmaf(s_xpart[(s * kMaxG + g) * dpc + dl], sc, acc);
+#pragma unroll
+    for (int s = 0; s < 8; ++s) {
+      const float sc = ms[s] > -INFINITY ? ex2_approx(ms[s] - M) : 0.f;
+      Lsum = fmaf(ls[s], sc, Lsum);
+      acc = fmaf(xs[s], sc, acc);
     }
     if (single) {
       float lse_c = lse_c_early, oc = oc_early;
