@@ -218,8 +218,8 @@ __global__ void __launch_bounds__(kThreads, 1) decode_kernel(const __grid_consta
   __shared__ __align__(8) unsigned long long s_full[kSlots][2], s_empty[kSlots][2];
   __shared__ unsigned long long s_best[kMaxG];     // best (similarity, row) of this CTA's calibration rows
   __shared__ unsigned long long s_bestall[kMaxG];  // ... of the whole cluster
-  __shared__ float s_xpart[kMaxG * kD];            // [source split][head][dim of this CTA's slice]
-  __shared__ float s_xml[8][kMaxG][2];             // [source split][head] (max, sum)
+  __shared__ __align__(16) float s_xpart[kMaxG * kD];  // [source split][head][dim of this CTA's slice]
+  __shared__ __align__(16) float s_xml[8][kMaxG][2];   // [source split][head] (max, sum)
   __shared__ int s_abort;
   __shared__ unsigned s_ticket;
 
@@ -265,8 +265,6 @@ __global__ void __launch_bounds__(kThreads, 1) decode_kernel(const __grid_consta
 
   const __nv_bfloat16* q = (const __nv_bfloat16*)P.q;
   const __nv_bfloat16* Cq = (const __nv_bfloat16*)P.C_q;
-  const unsigned char* Kc = (const unsigned char*)P.K + (size_t)unit * a.cap * kRowBytes;
-  const unsigned char* Vc = (const unsigned char*)P.V + (size_t)unit * a.cap * kRowBytes;
 
   const int r0 = min(a.n_kv, gs * a.rows_per_split);
   const int r1 = min(a.n_kv, r0 + a.rows_per_split);
@@ -578,11 +576,12 @@ __global__ void __launch_bounds__(kThreads, 1) decode_kernel(const __grid_consta
     }
   }
   __syncthreads();
-  // 256 threads: thread t owns dimensions (t & 63) and (t & 63) + 64 of head (t >> 6) + 4k, so the
-  // scale factors of the eight warps are worked out once for two elements, and all loads are done
-  // before the pushes (stores through generic pointers, which the compiler will not move loads across)
+  // 256 threads: thread t owns dimensions 2 (t & 63) and 2 (t & 63) + 1 of head (t >> 6) + 4k, so the
+  // scale factors of the eight warps are worked out once for two elements, which go to their owner
+  // in one 8-byte store; all loads are done before the pushes (stores through generic pointers,
+  // which the compiler will not move loads across)
   if (tid < 256) {
-    const int dlo = tid & 63;
+    const int d0 = 2 * (tid & 63);
     for (int g = tid >> 6; g < a.G; g += 4) {
       float mw[kStreamWarps], M = -INFINITY;
 #pragma unroll
@@ -591,17 +590,17 @@ __global__ void __launch_bounds__(kThreads, 1) decode_kernel(const __grid_consta
 #pragma unroll
       for (int w = 0; w < kStreamWarps; ++w) {
         const float sc = mw[w] > -INFINITY ? ex2_approx(mw[w] - M) : 0.f;
-        const float* wrow = wo + (w * kMaxG + g) * kWoStride + dlo;
+        const float2 wv = *reinterpret_cast<const float2*>(wo + (w * kMaxG + g) * kWoStride + d0);
         Lsum = fmaf(wml[(w * kMaxG + g) * 2 + 1], sc, Lsum);
-        acc0 = fmaf(wrow[0], sc, acc0);
-        acc1 = fmaf(wrow[64], sc, acc1);
+        acc0 = fmaf(wv.x, sc, acc0);
+        acc1 = fmaf(wv.y, sc, acc1);
       }
-      const int own0 = dlo >> lg_dpc, own1 = (dlo + 64) >> lg_dpc;
-      cluster.map_shared_rank(s_xpart, own0)[(split * kMaxG + g) * dpc + (dlo - own0 * dpc)] = acc0;
-      cluster.map_shared_rank(s_xpart, own1)[(split * kMaxG + g) * dpc + (dlo + 64 - own1 * dpc)] = acc1;
-      if (dlo < a.nsplit) {  // the (max, sum) pair of this split goes to every CTA of the cluster
-        float* xm = &cluster.map_shared_rank(&s_xml[0][0][0], dlo)[(split * kMaxG + g) * 2];
-        xm[0] = M; xm[1] = Lsum;
+      const int own = d0 >> lg_dpc;  // dpc is even: both dimensions have the same owner
+      *reinterpret_cast<float2*>(cluster.map_shared_rank(s_xpart, own) + (split * kMaxG + g) * dpc +
+                                 (d0 - own * dpc)) = make_float2(acc0, acc1);
+      if ((tid & 63) < a.nsplit) {  // the (max, sum) pair of this split goes to every CTA of the cluster
+        *reinterpret_cast<float2*>(&cluster.map_shared_rank(&s_xml[0][0][0], tid & 63)[(split * kMaxG + g) * 2]) =
+            make_float2(M, Lsum);
       }
     }
   }
