@@ -287,8 +287,12 @@ int calidrop_decode_batched(const calidrop_params* p, int32_t n_layers, const ca
   if (want > w.max_split) want = w.max_split;
   a.nsplit = 1;
   while (a.nsplit * 2 <= want && a.nsplit < 8) a.nsplit *= 2;
-  // few units with a long cache: several clusters per unit, combined through the workspace
+  // Few units with a long cache: several clusters per unit, combined through the workspace.  That
+  // combine costs about 4 us (fences, a ticket, a round trip through L2), as much as a CTA needs
+  // to stream a thousand rows, so a unit is split only while every CTA keeps at least 1024 rows.
   a.nclu = want / a.nsplit;
+  const int rows_single = (n_kv + a.nsplit - 1) / a.nsplit;
+  if (a.nclu > rows_single / 1024) a.nclu = rows_single / 1024;
   if (a.nclu < 1) a.nclu = 1;
   a.rows_per_split = (n_kv + a.nsplit * a.nclu - 1) / (a.nsplit * a.nclu);
   a.scale2 = scale2_of(p);

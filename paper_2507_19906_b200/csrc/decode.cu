@@ -19,10 +19,10 @@
 // The splits are combined inside the cluster through distributed shared memory: every CTA
 // finishes a slice of the 128 output dimensions for all heads of the group, and each CTA pushes
 // its partial of a slice into the shared memory of the slice's owner, so that after one cluster
-// barrier every CTA reduces local data only.  Only when very few units share a long cache does
-// one cluster per unit leave most SMs idle; then a unit gets up to eight clusters, each writes
-// its combined partial, its (max, sum) pair and its best similarity to the workspace, and the
-// CTA that takes the last ticket of the unit's arrival counter merges them and resets the counter.
+// barrier every CTA reduces local data only.  Only when very few units share a very long cache
+// (more than 1024 rows per CTA even with a cluster of eight) does a unit get up to eight clusters;
+// each writes its combined partial, its (max, sum) pair and its best similarity to the workspace, and
+// the CTA that takes the last ticket of the unit's arrival counter merges them and resets the counter.
 //
 // A launch moves only tens of MB, so its latency chain matters as much as its bandwidth:
 //   * the launch carries the programmatic-serialisation attribute and the kernel prefetches its

@@ -37,8 +37,8 @@ SMALL = [
     (1, 7, 1, 700, 64, 7, 160, 64),      # 448 window rows per kv head: two row blocks in the vote pass
     (1, 16, 2, 900, 64, 5, 200, 16),     # G = 8, W = 64: 512 window rows, four 128-row statistic blocks
     (1, 4, 1, 3000, 128, 7, 400, 128),   # W = 128: one query head per calibration row block
-    (1, 8, 1, 4000, 16, 7, 2100, 16),    # one unit, long cache: decode runs eight clusters per unit
-    (2, 8, 2, 2500, 16, 7, 1000, 7),     # four units: three clusters per unit, most CTAs without a C_q row
+    (1, 8, 1, 4000, 16, 7, 2100, 16),    # one unit: one cluster of eight CTAs, 263 rows each
+    (2, 8, 2, 2500, 16, 7, 1000, 7),     # four units: most CTAs without a C_q row
 ]
 
 
@@ -325,8 +325,10 @@ def test_config5_sampled_unit(cuda_lib):
 @pytest.mark.parametrize("B,Hq,Hkv,kv0,steps,n_cal", [
     (1, 4, 2, 0, 6, 3),       # the cache starts empty: the first step attends to its own row alone
     (2, 8, 2, 60, 8, 2),      # the appended row crosses the first 64-row slot boundary
-    (1, 7, 1, 1020, 10, 5),   # ... and a 16-row block boundary deep in a long slice (one unit: eight clusters)
+    (1, 7, 1, 1020, 10, 5),   # ... and a 16-row block boundary deep in a slice
     (3, 8, 8, 250, 4, 1),     # 24 units: clusters of 4, slices of about 64 rows
+    (1, 4, 1, 16500, 3, 2),   # one unit, 16500 rows: two clusters per unit meet through the workspace
+    (1, 8, 2, 40000, 2, 1),   # two units, 40000 rows each: four clusters per unit
 ])
 def test_decode_ignores_cache_rows_beyond_kv_len(cuda_lib, B, Hq, Hkv, kv0, steps, n_cal):
     """The cache rows at and beyond kv_len belong to the caller and may hold anything; here they
