@@ -9,7 +9,7 @@
 //
 // Grid: (split, batch*kv-head, layer); the splits of one (unit, layer) form thread-block
 // clusters of 1, 2, 4 or 8 CTAs.  A CTA has one producer warp and eight stream warps.  The
-// producer moves the CTA's slice of K and V through a ring of three 64-row slots with TMA
+// producer moves the CTA's slice of K and V through a ring of six 64-row slots with TMA
 // (128-byte swizzle, so ldmatrix is conflict-free and no load instruction per 16 bytes is
 // spent on the stream); each slot is consumed by four stream warps, 16 rows each, with their
 // own online softmax.  The products are taken transposed, keys on the 16-row side of the MMA and
@@ -25,12 +25,16 @@
 // the CTA that takes the last ticket of the unit's arrival counter merges them and resets the counter.
 //
 // A launch moves only tens of MB, so its latency chain matters as much as its bandwidth:
-//   * the launch carries the programmatic-serialisation attribute and the kernel prefetches its
-//     K/V slice into L2 before the dependency wait; a CTA takes less than half an SM, so the
-//     CTAs of the next decode call are resident, and prefetching, while this one finishes;
+//   * the launch carries the programmatic-serialisation attribute and the kernel, first thing,
+//     prefetches the head of its K/V slice into L2, ahead of the dependency wait; the ring takes
+//     most of an SM's shared memory, so a launch has one CTA per SM at most;
+//   * everything that does not need the predecessor's results (barrier setup, the address
+//     arithmetic of all later loads) is done ahead of the wait as well;
 //   * the similarity work (which needs only q and C_q) runs while the first slots are in flight,
-//     and the cluster exchanges each CTA's best (similarity, row) pair early, so the chosen O_c
-//     row is already being fetched while the partial outputs are combined.
+//     and the cluster exchanges each CTA's best (similarity, row) pair early; the producer warp,
+//     idle once the last slot is on its way, settles the calibration row meanwhile, and the chosen
+//     O_c elements are fetched while the partial outputs are combined;
+//   * the cache stream carries an evict-first L2 hint, the calibration state an evict-last hint.
 #include <cooperative_groups.h>
 
 #include "common.cuh"
