@@ -237,8 +237,10 @@ int calidrop_decode_batched(const calidrop_params* p, int32_t n_layers,
  *   - The first call on each device looks the array's device address up and caches it.  Make
  *     that first call outside any stream capture.
  *   - All calls on a device share the one array and it keeps whatever the last call left.  The
- *     part that must start at zero (the arrival counters) is cleared on `stream` ahead of the
- *     kernel by every call.  Two calls that may overlap on the GPU (different streams without
+ *     part that must start at zero (the arrival counters and the error word of the bounded
+ *     waits) is cleared on `stream` ahead of the kernel by every call.  The rest of the array is
+ *     used only when a unit is split over several thread-block clusters (one or two units with
+ *     tens of thousands of cached rows); otherwise the splits meet in shared memory.  Two calls that may overlap on the GPU (different streams without
  *     an ordering between them) race on the array; serialise them, or give the overlapping
  *     ones their own workspace through calidrop_decode.
  */
