@@ -371,3 +371,49 @@ def test_decode_ignores_cache_rows_beyond_kv_len(cuda_lib, B, Hq, Hkv, kv0, step
         np.testing.assert_array_equal(to_bits(st.K_kept)[:, :, :kv0 + t + 1], Kk[:, :, :kv0 + t + 1])
         np.testing.assert_array_equal(to_bits(st.V_kept)[:, :, :kv0 + t + 1], Vk[:, :, :kv0 + t + 1])
         np.testing.assert_array_equal(to_bits(st.K_kept)[:, :, kv0 + t + 1:], Kk[:, :, kv0 + t + 1:])
+
+
+def test_batched_layers_with_several_clusters_per_unit(cuda_lib):
+    """Two layers of one unit with 17000 cached rows in one launch: every (layer, unit) is split over
+    two clusters that meet through the workspace, each layer with its own counters and partials.
+    Checked against the oracle, twice on the same workspace (the counters must come back to zero)."""
+    cd = cuda_lib
+    rng = np.random.Generator(np.random.Philox(key=[91, 5]))
+    B, Hq, Hkv, D, kv0, n_cal, NL = 1, 4, 1, 128, 17000, 2, 2
+    cap = kv0 + 2
+    bits = lambda x: wl.f32_to_bf16_bits(np.ascontiguousarray(x, dtype=np.float32))
+    p = cd.make_params(B=B, Hq=Hq, Hkv=Hkv, L=kv0 + 64, window=8, pool=7, budget=kv0, n_cal=n_cal, cap=cap)
+    p.theta1, p.theta2 = 0.7, -1.0
+    ws = torch.zeros((cd.calidrop_decode_workspace_bytes(p, cap) * NL,), dtype=torch.uint8, device="cuda")
+    host, layers = [], []
+    for _ in range(NL):
+        Kk = np.zeros((B, Hkv, cap, D), dtype=np.uint16); Vk = np.zeros_like(Kk)
+        Kk[:, :, :kv0] = bits(rng.standard_normal((B, Hkv, kv0, D)))
+        Vk[:, :, :kv0] = bits(rng.standard_normal((B, Hkv, kv0, D)))
+        Cq = bits(rng.standard_normal((B, Hq, n_cal, D)))
+        Oc = rng.standard_normal((B, Hq, n_cal, D)).astype(np.float32)
+        Lc = (rng.standard_normal((B, Hq, n_cal)) + 9.0).astype(np.float32)
+        dev = dict(K_kept=to_dev(Kk), V_kept=to_dev(Vk), C_q=to_dev(Cq), O_c=torch.from_numpy(Oc).cuda(),
+                   LSE_c=torch.from_numpy(Lc).cuda(),
+                   out=torch.empty((B, Hq, D), dtype=torch.bfloat16, device="cuda"),
+                   lse_out=torch.empty((B, Hq), dtype=torch.float32, device="cuda"),
+                   flags=torch.empty((B, Hq), dtype=torch.uint8, device="cuda"))
+        host.append((Kk, Vk, Cq, Oc, Lc)); layers.append(dev)
+    for t in range(2):
+        step = []
+        for dev, (Kk, Vk, Cq, Oc, Lc) in zip(layers, host):
+            q = bits(wl.bf16_bits_to_f32(Cq[:, :, t % n_cal]) + 0.5 * rng.standard_normal((B, Hq, D)).astype(np.float32))
+            kn, vn = bits(rng.standard_normal((B, Hkv, D))), bits(rng.standard_normal((B, Hkv, D)))
+            dev.update(q=to_dev(q), k_new=to_dev(kn), v_new=to_dev(vn))
+            step.append((q, kn, vn))
+        cd.calidrop_decode_batched(p, cd.make_decode_layers(layers), kv0 + t, ws)
+        torch.cuda.synchronize()
+        off = cd.calidrop_decode_workspace_status_offset(p)
+        assert int(ws[off:off + 4].view(torch.int32).item()) == 0
+        for dev, (Kk, Vk, Cq, Oc, Lc), (q, kn, vn) in zip(layers, host, step):
+            o = oracle.decode(q, kn, vn, Kk, Vk, kv0 + t, Oc, Lc, Cq, theta1=0.7, theta2=-1.0)
+            same = (dev["flags"].cpu().numpy() >> 2) == (o.flags >> 2)
+            assert same.all()
+            assert_close_out(wl.bf16_bits_to_f64(to_bits(dev["out"])), o.out, f"step {t}")
+            assert_close_lse(dev["lse_out"].cpu().numpy(), o.lse, f"step {t} lse")
+            np.testing.assert_array_equal(to_bits(dev["K_kept"]), Kk)
