@@ -111,6 +111,26 @@ int calidrop_compress(const calidrop_params* p,
                       void* workspace, size_t workspace_bytes, void* stream);
 
 /*
+ * Gather and calibrate for a kept list chosen by the CALLER (Algorithm 1, line 3 "Select
+ * KV_compress using eviction strategy", lets any eviction rule stand there; lines 5-8 are the same
+ * for all of them): steps 2 and 3 of calidrop_compress with `kept_idx` as an INPUT, e.g. the
+ * index rule of a sink-plus-recent cache or an accumulated-score rule computed elsewhere.
+ *
+ *   kept_idx in [B, Hkv, n_kept] i32, n_kept = min(budget, L), ascending per (b, kv head), each
+ *            entry in [0, L), no duplicates.  The last `window` prompt rows count as kept whether
+ *            the list names them or not (E = [0, L - window) minus the listed rows), so a list
+ *            that is to be consistent with the gathered cache contains them.
+ *   all other arguments, the workspace size and the errors: as for calidrop_compress.  The row
+ *            LSE of the calibration queries is taken from lse_obs or, if that is NULL, computed by
+ *            the statistics pass of the window scoring.  `pool` of `p` is not used.
+ */
+int calidrop_calibrate(const calidrop_params* p,
+                       const void* Q_obs, const void* K, const void* V, const float* lse_obs,
+                       const int32_t* kept_idx, void* K_kept, void* V_kept,
+                       float* O_c, float* LSE_c, void* C_q,
+                       void* workspace, size_t workspace_bytes, void* stream);
+
+/*
  * Offsets (bytes from the workspace base) of intermediate arrays of the last
  * calidrop_compress call that used this workspace, for diagnostics and tests:
  *   vote   [B, Hkv, L-W] f32, pooled [B, Hkv, L-W] f32, row_lse [B, Hq, W] f32 (natural log;

@@ -23,7 +23,8 @@ STATIC_SCRATCH_BYTES = 4 << 20
 MAX_LAYERS = 32
 
 EXPORTS = [
-    "calidrop_compress_workspace_bytes", "calidrop_compress", "calidrop_compress_workspace_layout",
+    "calidrop_compress_workspace_bytes", "calidrop_compress", "calidrop_calibrate",
+    "calidrop_compress_workspace_layout",
     "calidrop_decode_workspace_bytes", "calidrop_decode_workspace_init",
     "calidrop_decode_workspace_status_offset", "calidrop_decode",
     "calidrop_decode_batched", "calidrop_decode_static", "calidrop_compress_host", "calidrop_decode_host",
@@ -71,6 +72,8 @@ def load():
     vp = C.c_void_p
     lib.calidrop_compress.restype = C.c_int
     lib.calidrop_compress.argtypes = [C.POINTER(Params)] + [vp] * 11 + [C.c_size_t, vp]
+    lib.calidrop_calibrate.restype = C.c_int
+    lib.calidrop_calibrate.argtypes = [C.POINTER(Params)] + [vp] * 11 + [C.c_size_t, vp]
     lib.calidrop_decode_workspace_status_offset.restype = C.c_size_t
     lib.calidrop_decode_workspace_status_offset.argtypes = [C.POINTER(Params)]
     lib.calidrop_decode_workspace_init.restype = C.c_int
@@ -155,6 +158,16 @@ def calidrop_compress(p, Q_obs, K, V, lse_obs, kept_idx, K_kept, V_kept, O_c, LS
                                   _ptr(workspace), workspace.numel() * workspace.element_size(), _stream())
     if check:
         _check(rc, "calidrop_compress")
+    return rc
+
+
+def calidrop_calibrate(p, Q_obs, K, V, lse_obs, kept_idx, K_kept, V_kept, O_c, LSE_c, C_q, workspace,
+                       check=True) -> int:
+    rc = load().calidrop_calibrate(C.byref(p), _ptr(Q_obs), _ptr(K), _ptr(V), _ptr(lse_obs), _ptr(kept_idx),
+                                   _ptr(K_kept), _ptr(V_kept), _ptr(O_c), _ptr(LSE_c), _ptr(C_q),
+                                   _ptr(workspace), workspace.numel() * workspace.element_size(), _stream())
+    if check:
+        _check(rc, "calidrop_calibrate")
     return rc
 
 

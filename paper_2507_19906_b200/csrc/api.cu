@@ -240,6 +240,45 @@ int calidrop_compress(const calidrop_params* p, const void* Q_obs, const void* K
   return CALIDROP_OK;
 }
 
+int calidrop_calibrate(const calidrop_params* p, const void* Q_obs, const void* K, const void* V,
+                       const float* lse_obs, const int32_t* kept_idx, void* K_kept, void* V_kept, float* O_c,
+                       float* LSE_c, void* C_q, void* workspace, size_t workspace_bytes, void* stream) {
+  int rc = check_compress(p);
+  if (rc != CALIDROP_OK) return rc;
+  const void* ptrs[] = {Q_obs, K, V, kept_idx, K_kept, V_kept, O_c, LSE_c, C_q, workspace};
+  for (const void* q : ptrs)
+    if (!q || !aligned16(q)) return CALIDROP_INVALID_ARG;
+  if (lse_obs && !aligned16(lse_obs)) return CALIDROP_INVALID_ARG;
+  if (reinterpret_cast<uintptr_t>(workspace) & 255u) return CALIDROP_INVALID_ARG;
+  const CompressGeom g = make_geom(p);
+  const CompressWs ws = make_ws(g);
+  if (workspace_bytes < ws.total) return CALIDROP_WORKSPACE_TOO_SMALL;
+  if (!device_supported()) return CALIDROP_UNSUPPORTED;
+
+  cudaStream_t st = (cudaStream_t)stream;
+  char* wsp = (char*)workspace;
+  cudaError_t e = cudaMemsetAsync(wsp + ws.status, 0, 4, st);
+  if (e != cudaSuccess) return cuda_fail(e);
+  const bool tc_path = score_tc_supported(g) && !scalar_path_forced();
+  // the calibration probabilities refer to the full-row softmax: its row LSE comes from the caller
+  // or from the statistics pass of the scoring
+  const float* row_lse = lse_obs;
+  if (!g.keep_all && !row_lse) {
+    e = tc_path ? launch_row_stats_tc(g, ws, Q_obs, K, wsp, st) : launch_row_stats(g, ws, Q_obs, K, wsp, st);
+    if (e != cudaSuccess) return cuda_fail(e);
+    row_lse = (const float*)(wsp + ws.row_lse);
+  }
+  e = launch_bitmap_from_indices(g, ws, wsp, kept_idx, st);
+  if (e != cudaSuccess) return cuda_fail(e);
+  e = launch_gather(g, K, V, kept_idx, K_kept, V_kept, st);
+  if (e != cudaSuccess) return cuda_fail(e);
+  e = (tc_path && calib_tc_supported(g))
+          ? launch_calib_tc(g, ws, Q_obs, K, V, row_lse, wsp, O_c, LSE_c, C_q, st)
+          : launch_calib_direct(g, ws, Q_obs, K, V, wsp, O_c, LSE_c, C_q, st);
+  if (e != cudaSuccess) return cuda_fail(e);
+  return CALIDROP_OK;
+}
+
 size_t calidrop_decode_workspace_bytes(const calidrop_params* p, int32_t kv_len_max) {
   if (check_common(p) != CALIDROP_OK || kv_len_max < 1) return 0;
   return make_decode_ws(p).per_layer;

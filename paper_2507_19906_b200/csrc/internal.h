@@ -103,6 +103,8 @@ cudaError_t launch_pool_select(const CompressGeom& g, const CompressWs& ws, char
 bool select_cluster_supported(const CompressGeom& g);
 cudaError_t launch_pool_select_cluster(const CompressGeom& g, const CompressWs& ws, char* wsp, int32_t* kept_idx,
                                        cudaStream_t st);
+cudaError_t launch_bitmap_from_indices(const CompressGeom& g, const CompressWs& ws, char* wsp,
+                                       const int32_t* kept_idx, cudaStream_t st);
 cudaError_t launch_gather(const CompressGeom& g, const void* K, const void* V, const int32_t* kept_idx,
                           void* K_kept, void* V_kept, cudaStream_t st);
 // decode.cu

@@ -160,6 +160,20 @@ __global__ void keep_all_kernel(uint32_t* __restrict__ bitmap, int32_t* __restri
   if (t < bitmap_words) bitmap[(size_t)unit * bitmap_words + t] = 0xffffffffu;
 }
 
+// Kept bitmap of a caller-supplied kept list: the listed rows plus the observation-window rows
+// [n_cand, L), which count as kept whatever the list says.  The bitmap is zeroed beforehand.
+__global__ void bitmap_from_indices_kernel(const int32_t* __restrict__ kept_idx, uint32_t* __restrict__ bitmap,
+                                           int n_kept, int n_cand, int L, int bitmap_words) {
+  const int unit = blockIdx.y;
+  const int32_t* kept = kept_idx + (size_t)unit * n_kept;
+  uint32_t* bm = bitmap + (size_t)unit * bitmap_words;
+  const int n = n_kept + (L - n_cand);
+  for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < n; i += gridDim.x * blockDim.x) {
+    const int t = i < n_kept ? kept[i] : n_cand + (i - n_kept);
+    if (t >= 0 && t < L) atomicOr(&bm[t >> 5], 1u << (t & 31));
+  }
+}
+
 // K_kept[u, i, :] = K[u, kept_idx[u, i], :], same for V; 16 lanes x 16 bytes per row.
 __global__ void __launch_bounds__(256)
 gather_kernel(const uint4* __restrict__ K, const uint4* __restrict__ V,
@@ -189,6 +203,19 @@ cudaError_t launch_pool_select(const CompressGeom& g, const CompressWs& ws, char
         (const float*)(wsp + ws.vote), (float*)(wsp + ws.pooled), (uint32_t*)(wsp + ws.bitmap), kept_idx,
         g.n_cand, g.L, g.pool, g.k_sel, g.n_kept, g.bitmap_words);
   }
+  count_launch(1);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_bitmap_from_indices(const CompressGeom& g, const CompressWs& ws, char* wsp,
+                                       const int32_t* kept_idx, cudaStream_t st) {
+  cudaError_t e = cudaMemsetAsync(wsp + ws.bitmap, 0, (size_t)g.units * g.bitmap_words * 4, st);
+  if (e != cudaSuccess) return e;
+  const int n = g.n_kept + (g.L - g.n_cand);
+  int blocks = (n + 255) / 256;
+  if (blocks > 64) blocks = 64;
+  bitmap_from_indices_kernel<<<dim3(blocks, g.units), 256, 0, st>>>(kept_idx, (uint32_t*)(wsp + ws.bitmap), g.n_kept,
+                                                                    g.n_cand, g.L, g.bitmap_words);
   count_launch(1);
   return cudaGetLastError();
 }

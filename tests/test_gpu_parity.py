@@ -417,3 +417,53 @@ def test_batched_layers_with_several_clusters_per_unit(cuda_lib):
             assert_close_out(wl.bf16_bits_to_f64(to_bits(dev["out"])), o.out, f"step {t}")
             assert_close_lse(dev["lse_out"].cpu().numpy(), o.lse, f"step {t} lse")
             np.testing.assert_array_equal(to_bits(dev["K_kept"]), Kk)
+
+
+# ---------------------------------------------------------------- a kept list chosen by the caller
+def _streaming_indices(B, Hkv, L, budget, n_sink):
+    """Index rule of a sink-plus-recent cache: the first n_sink rows and the most recent ones."""
+    idx = np.concatenate([np.arange(n_sink), np.arange(L - (budget - n_sink), L)]).astype(np.int32)
+    return np.broadcast_to(idx, (B, Hkv, budget)).copy()
+
+
+@pytest.mark.parametrize("B,Hq,Hkv,L,W,budget,n_cal,rule,supply_lse", [
+    (1, 4, 2, 700, 16, 96, 4, "streaming", False),
+    (2, 8, 2, 1500, 32, 256, 32, "random", False),     # two 128-row calibration blocks per kv head
+    (1, 7, 1, 3000, 64, 400, 64, "streaming", True),   # G = 7, row LSE supplied by the caller
+])
+def test_calibrate_with_a_supplied_kept_list(cuda_lib, B, Hq, Hkv, L, W, budget, n_cal, rule, supply_lse):
+    cd = cuda_lib
+    cfg = wl.small_config(B=B, Hq=Hq, Hkv=Hkv, L=L, window=W, pool=7, budget=budget, steps=3,
+                          n_sink=4, n_heavy=max(1, L // 50))
+    Q, K, V = _inputs(cfg)
+    if rule == "streaming":
+        kept = _streaming_indices(B, Hkv, L, budget, 32)
+    else:
+        rng = np.random.Generator(np.random.Philox(key=[5, L]))
+        kept = np.stack([np.stack([np.sort(np.concatenate([
+            rng.choice(L - W, size=budget - W, replace=False), np.arange(L - W, L)])).astype(np.int32)
+            for _ in range(Hkv)]) for _ in range(B)])
+    T = 3
+    p = cd.make_params(B=B, Hq=Hq, Hkv=Hkv, L=L, window=W, pool=7, budget=budget, n_cal=n_cal, cap=budget + T)
+    st = cd.alloc_layer_state(p)
+    ref = oracle.calibrate_given_indices(Q, K, V, kept, n_cal=n_cal, cap=budget + T)
+    lse = None
+    if supply_lse:
+        lse = torch.from_numpy(oracle.compress(Q, K, V, window=W, pool=7, budget=budget, n_cal=n_cal)
+                               .row_lse.astype(np.float32)).cuda()
+    cd.calidrop_calibrate(p, to_dev(Q), to_dev(K), to_dev(V), lse, torch.from_numpy(kept).cuda(), st.K_kept,
+                          st.V_kept, st.O_c, st.LSE_c, st.C_q, st.ws_compress)
+    torch.cuda.synchronize()
+    lay = cd.calidrop_compress_workspace_layout(p)
+    assert int(st.ws_compress[lay.status_offset:lay.status_offset + 4].view(torch.int32).item()) == 0
+    np.testing.assert_array_equal(to_bits(st.K_kept)[:, :, :budget], ref.K_kept[:, :, :budget])
+    np.testing.assert_array_equal(to_bits(st.V_kept)[:, :, :budget], ref.V_kept[:, :, :budget])
+    np.testing.assert_array_equal(to_bits(st.C_q), ref.C_q)
+    assert_close_lse(st.LSE_c.cpu().numpy(), ref.LSE_c, "LSE_c")
+    assert_close_out(st.O_c.cpu().numpy(), ref.O_c, "O_c")
+    # and the decode steps that follow use this state like any other
+    from types import SimpleNamespace
+    g = SimpleNamespace(st=st, p=p, n_kept=budget)
+    q, kn, vn = wl.gen_decode_inputs(cfg, Q, steps=T)
+    res = decode_steps_compare(g, ref, q, kn, vn, steps=T)
+    assert res["total"] == T * B * Hq
