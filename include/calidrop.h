@@ -131,6 +131,42 @@ int calidrop_calibrate(const calidrop_params* p,
                        void* workspace, size_t workspace_bytes, void* stream);
 
 /*
+ * The complement of calidrop_compress's gather: the evicted candidate rows, compacted, for the
+ * caller to offload ("offload them to the CPU", Algorithm 1 line 4) and to hand back to
+ * calidrop_recalibrate when a decode step raises needs_recompute.
+ *
+ *   kept_idx  in  [B, Hkv, n_kept] i32 as written by calidrop_compress (or given to calidrop_calibrate)
+ *   evict_idx out [B, Hkv, n_evict] i32, n_evict = L - budget: the rows of [0, L - window) that
+ *             kept_idx does not list, ascending
+ *   K_evict, V_evict out [B, Hkv, n_evict, D] bf16: bit copies of those rows
+ *   workspace as for calidrop_compress (its kept bitmap is rebuilt from kept_idx)
+ * INVALID_ARG also when budget >= L (nothing is evicted).
+ */
+int calidrop_gather_evicted(const calidrop_params* p, const void* K, const void* V, const int32_t* kept_idx,
+                            int32_t* evict_idx, void* K_evict, void* V_evict,
+                            void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * Recompute one calibration entry with the current query (Algorithm 2, lines 4-6, taken when
+ * rho < theta1; the printed "Q_-1" is read as the current query Q_t, which line 6 stores):
+ * per (b, query head hq of kv head h)
+ *   O_c[b, hq, slot, :] = attention of q[b, hq] over the evicted rows K_evict/V_evict[b, h, 0..n_evict),
+ *   LSE_c[b, hq, slot]  = log of its softmax denominator,
+ *   C_q[b, hq, slot, :] = q[b, hq].
+ * The other calibration rows are left as they are; with n_cal = 1 this is the paper's update.
+ * The caller then repeats the decode step (whose similarity with the new C_q row is 1).
+ *
+ *   q in [B, Hq, D] bf16; K_evict, V_evict in [B, Hkv, n_evict, D] bf16 (e.g. from
+ *   calidrop_gather_evicted, reloaded); n_evict >= 1; slot in [0, n_cal);
+ *   O_c, LSE_c, C_q in/out as written by calidrop_compress;
+ *   workspace: a decode workspace (see calidrop_decode_workspace_bytes / _init).
+ * The rows are streamed by the decode kernel (same split, same bounded waits, same error word).
+ */
+int calidrop_recalibrate(const calidrop_params* p, const void* q, const void* K_evict, const void* V_evict,
+                         int32_t n_evict, int32_t slot, float* O_c, float* LSE_c, void* C_q,
+                         void* workspace, size_t workspace_bytes, void* stream);
+
+/*
  * Offsets (bytes from the workspace base) of intermediate arrays of the last
  * calidrop_compress call that used this workspace, for diagnostics and tests:
  *   vote   [B, Hkv, L-W] f32, pooled [B, Hkv, L-W] f32, row_lse [B, Hq, W] f32 (natural log;

@@ -23,7 +23,8 @@ STATIC_SCRATCH_BYTES = 4 << 20
 MAX_LAYERS = 32
 
 EXPORTS = [
-    "calidrop_compress_workspace_bytes", "calidrop_compress", "calidrop_calibrate",
+    "calidrop_compress_workspace_bytes", "calidrop_compress", "calidrop_calibrate", "calidrop_gather_evicted",
+    "calidrop_recalibrate",
     "calidrop_compress_workspace_layout",
     "calidrop_decode_workspace_bytes", "calidrop_decode_workspace_init",
     "calidrop_decode_workspace_status_offset", "calidrop_decode",
@@ -72,6 +73,11 @@ def load():
     vp = C.c_void_p
     lib.calidrop_compress.restype = C.c_int
     lib.calidrop_compress.argtypes = [C.POINTER(Params)] + [vp] * 11 + [C.c_size_t, vp]
+    lib.calidrop_gather_evicted.restype = C.c_int
+    lib.calidrop_gather_evicted.argtypes = [C.POINTER(Params)] + [vp] * 7 + [C.c_size_t, vp]
+    lib.calidrop_recalibrate.restype = C.c_int
+    lib.calidrop_recalibrate.argtypes = [C.POINTER(Params), vp, vp, vp, C.c_int32, C.c_int32, vp, vp, vp, vp,
+                                         C.c_size_t, vp]
     lib.calidrop_calibrate.restype = C.c_int
     lib.calidrop_calibrate.argtypes = [C.POINTER(Params)] + [vp] * 11 + [C.c_size_t, vp]
     lib.calidrop_decode_workspace_status_offset.restype = C.c_size_t
@@ -168,6 +174,24 @@ def calidrop_calibrate(p, Q_obs, K, V, lse_obs, kept_idx, K_kept, V_kept, O_c, L
                                    _ptr(workspace), workspace.numel() * workspace.element_size(), _stream())
     if check:
         _check(rc, "calidrop_calibrate")
+    return rc
+
+
+def calidrop_gather_evicted(p, K, V, kept_idx, evict_idx, K_evict, V_evict, workspace, check=True) -> int:
+    rc = load().calidrop_gather_evicted(C.byref(p), _ptr(K), _ptr(V), _ptr(kept_idx), _ptr(evict_idx),
+                                        _ptr(K_evict), _ptr(V_evict), _ptr(workspace),
+                                        workspace.numel() * workspace.element_size(), _stream())
+    if check:
+        _check(rc, "calidrop_gather_evicted")
+    return rc
+
+
+def calidrop_recalibrate(p, q, K_evict, V_evict, n_evict, slot, O_c, LSE_c, C_q, workspace, check=True) -> int:
+    rc = load().calidrop_recalibrate(C.byref(p), _ptr(q), _ptr(K_evict), _ptr(V_evict), int(n_evict), int(slot),
+                                     _ptr(O_c), _ptr(LSE_c), _ptr(C_q), _ptr(workspace),
+                                     workspace.numel() * workspace.element_size(), _stream())
+    if check:
+        _check(rc, "calidrop_recalibrate")
     return rc
 
 

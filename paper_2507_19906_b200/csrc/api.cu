@@ -146,6 +146,42 @@ DecodeWs make_decode_ws(const calidrop_params* p) {
   return w;
 }
 
+// Split plan and workspace carving of one decode-kernel launch over `cap_rows`-row caches.
+DecodeCommon plan_decode(const calidrop_params* p, const DecodeWs& w, int n_layers, int kv_len, int n_kv,
+                         bool has_new, int cap_rows, void* workspace) {
+  DecodeCommon a{};
+  a.B = p->B; a.Hq = p->Hq; a.Hkv = p->Hkv; a.G = p->Hq / p->Hkv; a.n_cal = p->n_cal; a.cap = cap_rows;
+  a.kv_len = kv_len; a.n_kv = n_kv; a.has_new = has_new ? 1 : 0;
+  a.units = p->B * p->Hkv; a.n_layers = n_layers;
+  // the splits of a unit form one thread-block cluster: 1, 2, 4 or 8 CTAs
+  int want = decode_nsplit(a.units * n_layers, n_kv);
+  if (want > w.max_split) want = w.max_split;
+  a.nsplit = 1;
+  while (a.nsplit * 2 <= want && a.nsplit < 8) a.nsplit *= 2;
+  // Few units with a long cache: several clusters per unit, combined through the workspace.  That
+  // combine costs about 4 us (fences, a ticket, a round trip through L2), as much as a CTA needs
+  // to stream a thousand rows, so a unit is split only while every CTA keeps at least 1024 rows.
+  a.nclu = want / a.nsplit;
+  const int rows_single = (n_kv + a.nsplit - 1) / a.nsplit;
+  if (a.nclu > rows_single / 1024) a.nclu = rows_single / 1024;
+  if (a.nclu < 1) a.nclu = 1;
+  a.rows_per_split = (n_kv + a.nsplit * a.nclu - 1) / (a.nsplit * a.nclu);
+  a.scale2 = scale2_of(p);
+  a.theta1 = p->theta1; a.theta2 = p->theta2; a.always_apply = p->theta2 <= -1.0f;
+  // The workspace is laid out array by array with the layer index outermost inside each
+  // array, so it is carved for n_layers at once.
+  char* base = (char*)workspace;
+  const size_t nl = (size_t)n_layers;
+  size_t off = 0;
+  a.counters = (unsigned*)(base + off); off += align_up((size_t)a.units * 4 * kDecodeMaxLayers, 256);
+  a.status = (unsigned*)(base + off);   off += 256;
+  a.part_ml = (float*)(base + off);     off += align_up((size_t)a.units * a.nclu * kMaxG * 2 * 4 * nl, 256);
+  a.part_best = (unsigned long long*)(base + off); off += align_up((size_t)a.units * a.nclu * kMaxG * 8 * nl, 256);
+  a.part_o = (float*)(base + off);
+  a.recal_slot = 0;
+  return a;
+}
+
 // Built-in scratch of calidrop_decode_static.  In host code this name is only a handle for
 // cudaGetSymbolAddress; the kernel must be given the device address that call returns.
 static __device__ __align__(256) unsigned char g_static_decode_scratch[CALIDROP_STATIC_SCRATCH_BYTES];
@@ -279,6 +315,54 @@ int calidrop_calibrate(const calidrop_params* p, const void* Q_obs, const void* 
   return CALIDROP_OK;
 }
 
+int calidrop_gather_evicted(const calidrop_params* p, const void* K, const void* V, const int32_t* kept_idx,
+                            int32_t* evict_idx, void* K_evict, void* V_evict, void* workspace,
+                            size_t workspace_bytes, void* stream) {
+  int rc = check_compress(p);
+  if (rc != CALIDROP_OK) return rc;
+  const void* ptrs[] = {K, V, kept_idx, evict_idx, K_evict, V_evict, workspace};
+  for (const void* q : ptrs)
+    if (!q || !aligned16(q)) return CALIDROP_INVALID_ARG;
+  if (reinterpret_cast<uintptr_t>(workspace) & 255u) return CALIDROP_INVALID_ARG;
+  const CompressGeom g = make_geom(p);
+  if (g.keep_all) return CALIDROP_INVALID_ARG;  // nothing is evicted
+  const CompressWs ws = make_ws(g);
+  if (workspace_bytes < ws.total) return CALIDROP_WORKSPACE_TOO_SMALL;
+  if (!device_supported()) return CALIDROP_UNSUPPORTED;
+  cudaStream_t st = (cudaStream_t)stream;
+  char* wsp = (char*)workspace;
+  cudaError_t e = launch_bitmap_from_indices(g, ws, wsp, kept_idx, st);
+  if (e != cudaSuccess) return cuda_fail(e);
+  e = launch_evicted_indices(g, ws, wsp, evict_idx, st);
+  if (e != cudaSuccess) return cuda_fail(e);
+  const int n_evict = g.L - g.n_kept;
+  e = launch_gather_rows(g, K, V, evict_idx, n_evict, n_evict, K_evict, V_evict, st);
+  return e == cudaSuccess ? CALIDROP_OK : cuda_fail(e);
+}
+
+int calidrop_recalibrate(const calidrop_params* p, const void* q, const void* K_evict, const void* V_evict,
+                         int32_t n_evict, int32_t slot, float* O_c, float* LSE_c, void* C_q, void* workspace,
+                         size_t workspace_bytes, void* stream) {
+  int rc = check_common(p);
+  if (rc != CALIDROP_OK) return rc;
+  const void* req[] = {q, K_evict, V_evict, O_c, LSE_c, C_q, workspace};
+  for (const void* r : req)
+    if (!r || !aligned16(r)) return CALIDROP_INVALID_ARG;
+  if (reinterpret_cast<uintptr_t>(workspace) & 255u) return CALIDROP_INVALID_ARG;
+  if (n_evict < 1 || slot < 0 || slot >= p->n_cal) return CALIDROP_INVALID_ARG;
+  const DecodeWs w = make_decode_ws(p);
+  if (workspace_bytes < w.per_layer) return CALIDROP_WORKSPACE_TOO_SMALL;
+  if (!device_supported()) return CALIDROP_UNSUPPORTED;
+  DecodeArgsT<1> args{};
+  args.c = plan_decode(p, w, 1, n_evict, n_evict, false, n_evict, workspace);
+  args.c.recal_slot = slot;
+  args.layer[0] = DecodeLayerPtrs{q, nullptr, nullptr, const_cast<void*>(K_evict), const_cast<void*>(V_evict), O_c,
+                                  LSE_c, C_q, nullptr, nullptr, nullptr};
+  if (!make_decode_maps(args.c, args.layer[0], &args.maps[0])) return CALIDROP_CUDA_ERROR;
+  cudaError_t e = launch_recalibrate(args, (cudaStream_t)stream);
+  return e == cudaSuccess ? CALIDROP_OK : cuda_fail(e);
+}
+
 size_t calidrop_decode_workspace_bytes(const calidrop_params* p, int32_t kv_len_max) {
   if (check_common(p) != CALIDROP_OK || kv_len_max < 1) return 0;
   return make_decode_ws(p).per_layer;
@@ -317,35 +401,7 @@ int calidrop_decode_batched(const calidrop_params* p, int32_t n_layers, const ca
   if (workspace_bytes < w.per_layer * (size_t)n_layers) return CALIDROP_WORKSPACE_TOO_SMALL;
   if (!device_supported()) return CALIDROP_UNSUPPORTED;
 
-  DecodeCommon a{};
-  a.B = p->B; a.Hq = p->Hq; a.Hkv = p->Hkv; a.G = p->Hq / p->Hkv; a.n_cal = p->n_cal; a.cap = p->cap;
-  a.kv_len = kv_len; a.n_kv = n_kv; a.has_new = has_new ? 1 : 0;
-  a.units = p->B * p->Hkv; a.n_layers = n_layers;
-  // the splits of a unit form one thread-block cluster: 1, 2, 4 or 8 CTAs
-  int want = decode_nsplit(a.units * n_layers, n_kv);
-  if (want > w.max_split) want = w.max_split;
-  a.nsplit = 1;
-  while (a.nsplit * 2 <= want && a.nsplit < 8) a.nsplit *= 2;
-  // Few units with a long cache: several clusters per unit, combined through the workspace.  That
-  // combine costs about 4 us (fences, a ticket, a round trip through L2), as much as a CTA needs
-  // to stream a thousand rows, so a unit is split only while every CTA keeps at least 1024 rows.
-  a.nclu = want / a.nsplit;
-  const int rows_single = (n_kv + a.nsplit - 1) / a.nsplit;
-  if (a.nclu > rows_single / 1024) a.nclu = rows_single / 1024;
-  if (a.nclu < 1) a.nclu = 1;
-  a.rows_per_split = (n_kv + a.nsplit * a.nclu - 1) / (a.nsplit * a.nclu);
-  a.scale2 = scale2_of(p);
-  a.theta1 = p->theta1; a.theta2 = p->theta2; a.always_apply = p->theta2 <= -1.0f;
-  // The workspace is laid out array by array with the layer index outermost inside each
-  // array, so it is carved for n_layers at once.
-  char* base = (char*)workspace;
-  const size_t nl = (size_t)n_layers;
-  size_t off = 0;
-  a.counters = (unsigned*)(base + off); off += align_up((size_t)a.units * 4 * kDecodeMaxLayers, 256);
-  a.status = (unsigned*)(base + off);   off += 256;
-  a.part_ml = (float*)(base + off);     off += align_up((size_t)a.units * a.nclu * kMaxG * 2 * 4 * nl, 256);
-  a.part_best = (unsigned long long*)(base + off); off += align_up((size_t)a.units * a.nclu * kMaxG * 8 * nl, 256);
-  a.part_o = (float*)(base + off);
+  DecodeCommon a = plan_decode(p, w, n_layers, kv_len, n_kv, has_new, p->cap, workspace);
   cudaError_t e;
   if (n_layers == 1) {
     DecodeArgsT<1> args{};

@@ -216,7 +216,21 @@ __device__ __forceinline__ void merge_store(const DecodeCommon& a, const DecodeL
   }
 }
 
-template <int NL>
+// Algorithm 2, lines 4-6, for the launches that recompute a calibration entry: the attention of the
+// current query over the (reloaded) evicted KV is the new O_c row, its log-denominator the new LSE_c,
+// and the query itself the new C_q row (the reading of line 4-5's "Q_-1" as the current query).
+__device__ __forceinline__ void recal_store(const DecodeCommon& a, const DecodeLayerPtrs& P, int hq, int d, float acc,
+                                            float M, float Lsum) {
+  const size_t row = (size_t)hq * a.n_cal + a.recal_slot;
+  const_cast<float*>(P.O_c)[row * kD + d] = acc / Lsum;
+  reinterpret_cast<__nv_bfloat16*>(const_cast<void*>(P.C_q))[row * kD + d] =
+      reinterpret_cast<const __nv_bfloat16*>(P.q)[(size_t)hq * kD + d];
+  if (d == 0) const_cast<float*>(P.LSE_c)[row] = (M + log2f(Lsum)) * kLn2;
+}
+
+// RECAL = false: the decode step.  RECAL = true: the same stream over the evicted KV, without the
+// similarity and the gate, ending in recal_store.
+template <int NL, bool RECAL>
 __global__ void __launch_bounds__(kThreads, 1) decode_kernel(const __grid_constant__ DecodeArgsT<NL> args) {
   extern __shared__ unsigned char smem_raw[];
   __shared__ __align__(8) unsigned long long s_full[kSlots][2], s_empty[kSlots][2];
@@ -282,7 +296,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_kernel(const __grid_consta
   // calibration rows of this CTA: the contiguous range [c_begin, c_begin + n_c)
   const int c_per = (a.n_cal + n_gs - 1) / n_gs;
   const int c_begin = min(a.n_cal, gs * c_per);
-  const int n_c = min(a.n_cal, c_begin + c_per) - c_begin;
+  const int n_c = RECAL ? 0 : min(a.n_cal, c_begin + c_per) - c_begin;
   if (tid == 0) {
     for (int s = 0; s < kSlots; ++s)
       for (int p = 0; p < 2; ++p) {
@@ -325,7 +339,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_kernel(const __grid_consta
   const int dpc = kD / a.nsplit, lg_dpc = 31 - __clz(dpc);  // nsplit is a power of two
   const int n_items = a.G * dpc;
   const bool single = a.nclu == 1;
-  const bool early = single && n_items <= kThreads;  // one output element per thread at most
+  const bool early = !RECAL && single && n_items <= kThreads;  // one output element per thread at most
   const int eg = min(tid >> lg_dpc, a.G - 1), ed = split * dpc + (tid & (dpc - 1));
   const float* oc_base = P.O_c + (size_t)(hq0 + eg) * a.n_cal * kD + ed;
   const float* lsec_base = P.LSE_c + (size_t)(hq0 + eg) * a.n_cal;
@@ -547,7 +561,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_kernel(const __grid_consta
   __syncthreads();  // all warps are done with the ring: reuse it for the combine
   // the common case has one output element per thread at most: its O_c element and LSE_c are
   // loaded now and arrive while the partials are combined
-  if (!single || n_items > kThreads) {
+  if (!RECAL && (!single || n_items > kThreads)) {
     if (tid < a.G && single) {
       const size_t crow = (size_t)(hq0 + tid) * a.n_cal + (unsigned)(s_bestall[tid] & 0xffffffffull);
       const float* orow = P.O_c + crow * kD;
@@ -635,13 +649,17 @@ __global__ void __launch_bounds__(kThreads, 1) decode_kernel(const __grid_consta
       acc = fmaf(xs[s], sc, acc);
     }
     if (single) {
-      float lse_c = lse_c_early, oc = oc_early;
-      if (!early) {
-        const size_t crow = (size_t)hq * a.n_cal + (unsigned)(best & 0xffffffffull);
-        lse_c = __ldg(P.LSE_c + crow);
-        oc = __ldg(P.O_c + crow * kD + d);
+      if constexpr (RECAL) {
+        recal_store(a, P, hq, d, acc, M, Lsum);
+      } else {
+        float lse_c = lse_c_early, oc = oc_early;
+        if (!early) {
+          const size_t crow = (size_t)hq * a.n_cal + (unsigned)(best & 0xffffffffull);
+          lse_c = __ldg(P.LSE_c + crow);
+          oc = __ldg(P.O_c + crow * kD + d);
+        }
+        merge_store(a, P, hq, d, acc, M, Lsum, best, lse_c, oc);
       }
-      merge_store(a, P, hq, d, acc, M, Lsum, best, lse_c, oc);
     } else {
       // this cluster's partial goes to the workspace; (M, Lsum, best) are the same in all its CTAs
       const size_t pc = ((size_t)lu * a.nclu + clu) * kMaxG + g;
@@ -680,8 +698,8 @@ __global__ void __launch_bounds__(kThreads, 1) decode_kernel(const __grid_consta
         }
         const int hq = hq0 + g;
         const size_t crow = (size_t)hq * a.n_cal + (unsigned)(best & 0xffffffffull);
-        const float lse_c = __ldg(P.LSE_c + crow);
-        const float oc = __ldg(P.O_c + crow * kD + d);
+        const float lse_c = RECAL ? 0.f : __ldg(P.LSE_c + crow);
+        const float oc = RECAL ? 0.f : __ldg(P.O_c + crow * kD + d);
         float M = -INFINITY;
 #pragma unroll
         for (int c = 0; c < 8; ++c) M = fmaxf(M, ms[c]);
@@ -692,7 +710,8 @@ __global__ void __launch_bounds__(kThreads, 1) decode_kernel(const __grid_consta
           Lsum = fmaf(ls[c], sc, Lsum);
           acc = fmaf(os[c], sc, acc);
         }
-        merge_store(a, P, hq, d, acc, M, Lsum, best, lse_c, oc);
+        if constexpr (RECAL) recal_store(a, P, hq, d, acc, M, Lsum);
+        else merge_store(a, P, hq, d, acc, M, Lsum, best, lse_c, oc);
       }
       if (tid == 0) a.counters[lu] = 0u;  // ready for the next launch on this workspace
     }
@@ -715,14 +734,14 @@ bool make_decode_maps(const DecodeCommon& c, const DecodeLayerPtrs& L, DecodeLay
 
 namespace {
 
-template <int NL>
+template <int NL, bool RECAL>
 cudaError_t launch_decode_t(const DecodeArgsT<NL>& a, cudaStream_t st) {
   static bool attr_set[64] = {};
   int dev = 0;
   cudaError_t e = cudaGetDevice(&dev);
   if (e != cudaSuccess) return e;
   if (dev < 0 || dev >= 64 || !attr_set[dev]) {
-    e = cudaFuncSetAttribute(decode_kernel<NL>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+    e = cudaFuncSetAttribute(decode_kernel<NL, RECAL>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
     if (e != cudaSuccess) return e;
     if (dev >= 0 && dev < 64) attr_set[dev] = true;
   }
@@ -740,7 +759,7 @@ cudaError_t launch_decode_t(const DecodeArgsT<NL>& a, cudaStream_t st) {
   attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 2;
-  e = cudaLaunchKernelEx(&cfg, decode_kernel<NL>, a);
+  e = cudaLaunchKernelEx(&cfg, decode_kernel<NL, RECAL>, a);
   if (e != cudaSuccess) return e;
   count_launch(1);
   return cudaGetLastError();
@@ -748,9 +767,10 @@ cudaError_t launch_decode_t(const DecodeArgsT<NL>& a, cudaStream_t st) {
 
 }  // namespace
 
-cudaError_t launch_decode(const DecodeArgsT<1>& a, cudaStream_t st) { return launch_decode_t<1>(a, st); }
+cudaError_t launch_decode(const DecodeArgsT<1>& a, cudaStream_t st) { return launch_decode_t<1, false>(a, st); }
 cudaError_t launch_decode(const DecodeArgsT<kDecodeMaxLayers>& a, cudaStream_t st) {
-  return launch_decode_t<kDecodeMaxLayers>(a, st);
+  return launch_decode_t<kDecodeMaxLayers, false>(a, st);
 }
+cudaError_t launch_recalibrate(const DecodeArgsT<1>& a, cudaStream_t st) { return launch_decode_t<1, true>(a, st); }
 
 }  // namespace calidrop

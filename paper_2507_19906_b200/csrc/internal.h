@@ -64,6 +64,7 @@ struct DecodeCommon {
   unsigned long long* part_best;  // [layer][unit][nclu][8] best (similarity, row) keys
   unsigned* counters;             // [layer][unit]
   unsigned* status;               // error word of the workspace: nonzero after a wait ran out
+  int recal_slot;                 // launch_recalibrate only: the calibration row that is rewritten
 };
 
 // Kernel argument block for NL layers (1 for the single-layer entry points, 32 for the batched one:
@@ -105,6 +106,8 @@ cudaError_t launch_pool_select_cluster(const CompressGeom& g, const CompressWs& 
                                        cudaStream_t st);
 cudaError_t launch_bitmap_from_indices(const CompressGeom& g, const CompressWs& ws, char* wsp,
                                        const int32_t* kept_idx, cudaStream_t st);
+cudaError_t launch_gather_rows(const CompressGeom& g, const void* K, const void* V, const int32_t* idx, int n_rows,
+                               int out_rows, void* K_out, void* V_out, cudaStream_t st);
 cudaError_t launch_gather(const CompressGeom& g, const void* K, const void* V, const int32_t* kept_idx,
                           void* K_kept, void* V_kept, cudaStream_t st);
 // decode.cu
@@ -112,6 +115,11 @@ cudaError_t launch_gather(const CompressGeom& g, const void* K, const void* V, c
 bool make_decode_maps(const DecodeCommon& c, const DecodeLayerPtrs& L, DecodeLayerMaps* out);
 cudaError_t launch_decode(const DecodeArgsT<1>& a, cudaStream_t st);
 cudaError_t launch_decode(const DecodeArgsT<kDecodeMaxLayers>& a, cudaStream_t st);
+// The same stream over the evicted KV (K, V of the layer = the compacted evicted rows), rewriting
+// row recal_slot of O_c, LSE_c, C_q (Algorithm 2, lines 4-6).
+cudaError_t launch_recalibrate(const DecodeArgsT<1>& a, cudaStream_t st);
+cudaError_t launch_evicted_indices(const CompressGeom& g, const CompressWs& ws, char* wsp, int32_t* evict_idx,
+                                   cudaStream_t st);
 
 void count_launch(int n = 1);
 

@@ -207,6 +207,65 @@ cudaError_t launch_pool_select(const CompressGeom& g, const CompressWs& ws, char
   return cudaGetLastError();
 }
 
+// Ascending list of the evicted candidates of a unit: the zero bits of its kept bitmap below n_cand.
+// One CTA per unit; thread i owns a contiguous run of bitmap words, so a block-wide exclusive scan of
+// the per-thread counts gives every thread the position of its first index.
+__global__ void __launch_bounds__(kSelThreads)
+evicted_indices_kernel(const uint32_t* __restrict__ bitmap, int32_t* __restrict__ evict_idx, int n_cand, int n_evict,
+                       int bitmap_words) {
+  __shared__ unsigned warp_sum[kSelThreads / 32];
+  const int unit = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const uint32_t* bm = bitmap + (size_t)unit * bitmap_words;
+  int32_t* out = evict_idx + (size_t)unit * n_evict;
+  const int n_words = (n_cand + 31) >> 5;
+  const int wpt = (n_words + kSelThreads - 1) / kSelThreads;
+  const int w0 = tid * wpt, w1 = min(n_words, w0 + wpt);
+  auto zeros_of = [&](int w) {
+    uint32_t z = ~bm[w];
+    const int rem = n_cand - (w << 5);
+    if (rem < 32) z &= (1u << rem) - 1u;
+    return z;
+  };
+  unsigned cnt = 0;
+  for (int w = w0; w < w1; ++w) cnt += __popc(zeros_of(w));
+  unsigned incl = cnt;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const unsigned n = __shfl_up_sync(0xffffffffu, incl, o);
+    if (lane >= o) incl += n;
+  }
+  if (lane == 31) warp_sum[warp] = incl;
+  __syncthreads();
+  if (warp == 0) {
+    unsigned v = lane < kSelThreads / 32 ? warp_sum[lane] : 0u, iv = v;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const unsigned n = __shfl_up_sync(0xffffffffu, iv, o);
+      if (lane >= o) iv += n;
+    }
+    if (lane < kSelThreads / 32) warp_sum[lane] = iv - v;
+  }
+  __syncthreads();
+  unsigned pos = warp_sum[warp] + incl - cnt;
+  for (int w = w0; w < w1; ++w) {
+    uint32_t z = zeros_of(w);
+    while (z) {
+      const int b = __ffs(z) - 1;
+      z &= z - 1;
+      if (pos < (unsigned)n_evict) out[pos] = (w << 5) + b;
+      ++pos;
+    }
+  }
+}
+
+cudaError_t launch_evicted_indices(const CompressGeom& g, const CompressWs& ws, char* wsp, int32_t* evict_idx,
+                                   cudaStream_t st) {
+  evicted_indices_kernel<<<g.units, kSelThreads, 0, st>>>((const uint32_t*)(wsp + ws.bitmap), evict_idx, g.n_cand,
+                                                          g.L - g.n_kept, g.bitmap_words);
+  count_launch(1);
+  return cudaGetLastError();
+}
+
 cudaError_t launch_bitmap_from_indices(const CompressGeom& g, const CompressWs& ws, char* wsp,
                                        const int32_t* kept_idx, cudaStream_t st) {
   cudaError_t e = cudaMemsetAsync(wsp + ws.bitmap, 0, (size_t)g.units * g.bitmap_words * 4, st);
@@ -220,13 +279,18 @@ cudaError_t launch_bitmap_from_indices(const CompressGeom& g, const CompressWs& 
   return cudaGetLastError();
 }
 
-cudaError_t launch_gather(const CompressGeom& g, const void* K, const void* V, const int32_t* kept_idx,
-                          void* K_kept, void* V_kept, cudaStream_t st) {
-  dim3 grid((g.n_kept + 15) / 16, g.units);
-  gather_kernel<<<grid, 256, 0, st>>>((const uint4*)K, (const uint4*)V, kept_idx, (uint4*)K_kept,
-                                      (uint4*)V_kept, g.L, g.n_kept, g.cap);
+cudaError_t launch_gather_rows(const CompressGeom& g, const void* K, const void* V, const int32_t* idx, int n_rows,
+                               int out_rows, void* K_out, void* V_out, cudaStream_t st) {
+  dim3 grid((n_rows + 15) / 16, g.units);
+  gather_kernel<<<grid, 256, 0, st>>>((const uint4*)K, (const uint4*)V, idx, (uint4*)K_out, (uint4*)V_out, g.L,
+                                      n_rows, out_rows);
   count_launch(1);
   return cudaGetLastError();
+}
+
+cudaError_t launch_gather(const CompressGeom& g, const void* K, const void* V, const int32_t* kept_idx,
+                          void* K_kept, void* V_kept, cudaStream_t st) {
+  return launch_gather_rows(g, K, V, kept_idx, g.n_kept, g.cap, K_kept, V_kept, st);
 }
 
 }  // namespace calidrop

@@ -467,3 +467,64 @@ def test_calibrate_with_a_supplied_kept_list(cuda_lib, B, Hq, Hkv, L, W, budget,
     q, kn, vn = wl.gen_decode_inputs(cfg, Q, steps=T)
     res = decode_steps_compare(g, ref, q, kn, vn, steps=T)
     assert res["total"] == T * B * Hq
+
+
+# ---------------------------------------------------------------- the recompute branch (Algorithm 2, lines 3-8)
+@pytest.mark.parametrize("B,Hq,Hkv,L,W,budget,n_cal,slot", [
+    (1, 4, 2, 600, 16, 80, 1, 0),          # the paper's single calibration query
+    (2, 8, 2, 1500, 32, 256, 4, 2),        # G = 4, one of four rows rewritten
+    (1, 7, 1, 20000, 64, 2048, 64, 63),    # one unit, 17952 evicted rows: two clusters per unit
+])
+def test_gather_evicted_and_recalibrate(cuda_lib, B, Hq, Hkv, L, W, budget, n_cal, slot):
+    cd = cuda_lib
+    cfg = wl.small_config(B=B, Hq=Hq, Hkv=Hkv, L=L, window=W, pool=7, budget=budget, steps=2,
+                          n_sink=4, n_heavy=max(1, L // 50))
+    Q, K, V = _inputs(cfg)
+    g = gpu_compress(Q, K, V, window=W, pool=7, budget=budget, n_cal=n_cal, cap=budget + 2, keep_inputs=True)
+    n_e = L - budget
+    ev_idx = torch.empty((B, Hkv, n_e), dtype=torch.int32, device="cuda")
+    K_e = torch.empty((B, Hkv, n_e, 128), dtype=torch.bfloat16, device="cuda")
+    V_e = torch.empty_like(K_e)
+    cd.calidrop_gather_evicted(g.p, g.dK, g.dV, g.st.kept_idx, ev_idx, K_e, V_e, g.st.ws_compress)
+    torch.cuda.synchronize()
+    ev = ev_idx.cpu().numpy()
+    for b in range(B):
+        for h in range(Hkv):
+            want = np.setdiff1d(np.arange(L - W), g.kept_idx[b, h])     # ascending complement among candidates
+            np.testing.assert_array_equal(ev[b, h], want)
+            np.testing.assert_array_equal(to_bits(K_e)[b, h], K[b, h][want])
+            np.testing.assert_array_equal(to_bits(V_e)[b, h], V[b, h][want])
+    # a query far from every calibration query, as in the branch's condition
+    rng = np.random.Generator(np.random.Philox(key=[11, L]))
+    q = wl.f32_to_bf16_bits(rng.standard_normal((B, Hq, 128)).astype(np.float32))
+    O_before, L_before, C_before = g.st.O_c.clone(), g.st.LSE_c.clone(), g.st.C_q.clone()
+    cd.calidrop_recalibrate(g.p, to_dev(q), K_e, V_e, n_e, slot, g.st.O_c, g.st.LSE_c, g.st.C_q, g.st.ws_decode)
+    torch.cuda.synchronize()
+    off = cd.calidrop_decode_workspace_status_offset(g.p)
+    assert int(g.st.ws_decode[off:off + 4].view(torch.int32).item()) == 0
+    G = Hq // Hkv
+    for b in range(B):
+        for hq in range(Hq):
+            h = hq // G
+            o, l = oracle.full_attention(q[b, hq][None], K[b, h][ev[b, h]], V[b, h][ev[b, h]])
+            assert_close_out(g.st.O_c[b, hq, slot].cpu().numpy(), o[0], "recomputed O_c")
+            assert abs(float(g.st.LSE_c[b, hq, slot]) - l[0]) < 1e-3
+    np.testing.assert_array_equal(to_bits(g.st.C_q)[:, :, slot], q)
+    keep = [c for c in range(n_cal) if c != slot]                      # the other rows are untouched
+    assert torch.equal(g.st.O_c[:, :, keep], O_before[:, :, keep])
+    assert torch.equal(g.st.LSE_c[:, :, keep], L_before[:, :, keep])
+    assert torch.equal(g.st.C_q[:, :, keep], C_before[:, :, keep])
+    # the repeated decode step now finds rho = 1 with the new row and merges: the result is the
+    # attention of q over the kept and the evicted rows together, i.e. over the whole prompt
+    out = torch.empty((B, Hq, 128), dtype=torch.bfloat16, device="cuda")
+    flags = torch.empty((B, Hq), dtype=torch.uint8, device="cuda")
+    cd.calidrop_decode(g.p, to_dev(q), None, None, g.st.K_kept, g.st.V_kept, budget, g.st.O_c, g.st.LSE_c, g.st.C_q,
+                       out, None, flags, g.st.ws_decode)
+    torch.cuda.synchronize()
+    f = flags.cpu().numpy()
+    assert np.all(f & 1 == 1) and np.all(f & 2 == 0)
+    got = wl.bf16_bits_to_f64(to_bits(out))
+    for b in range(B):
+        for hq in range(Hq):
+            o, _ = oracle.full_attention(q[b, hq][None], K[b, hq // G], V[b, hq // G])
+            assert_close_out(got[b, hq], o[0], "decode after the recompute vs attention over the whole prompt")
