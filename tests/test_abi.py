@@ -67,3 +67,16 @@ def test_null_arguments_are_rejected_before_any_cuda_call(lib):
     rc = lib.calidrop_decode(ctypes.byref(p), None, None, None, None, None, 1, None, None, None, None, None,
                              None, None, 0, None)
     assert rc == cd.INVALID_ARG
+    rc = lib.calidrop_calibrate(ctypes.byref(p), None, None, None, None, None, None, None, None, None, None,
+                                None, 0, None)
+    assert rc == cd.INVALID_ARG
+    rc = lib.calidrop_gather_evicted(ctypes.byref(p), None, None, None, None, None, None, None, 0, None)
+    assert rc == cd.INVALID_ARG
+    buf = (ctypes.c_char * 4096)()
+    a = ctypes.addressof(buf)
+    a = (a + 255) & ~255                                   # an aligned host address: never dereferenced
+    ptr = ctypes.c_void_p(a)
+    # slot outside [0, n_cal) and an empty evicted set are refused before any CUDA call
+    assert lib.calidrop_recalibrate(ctypes.byref(p), ptr, ptr, ptr, 10, 1, ptr, ptr, ptr, ptr, 1 << 20, None) == cd.INVALID_ARG
+    assert lib.calidrop_recalibrate(ctypes.byref(p), ptr, ptr, ptr, 0, 0, ptr, ptr, ptr, ptr, 1 << 20, None) == cd.INVALID_ARG
+    assert lib.calidrop_recalibrate(ctypes.byref(p), None, ptr, ptr, 10, 0, ptr, ptr, ptr, ptr, 1 << 20, None) == cd.INVALID_ARG
