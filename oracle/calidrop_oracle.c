@@ -8,7 +8,7 @@
  *
  * Inputs are bf16 bit patterns (uint16), widened exactly to double.
  *
- * What follows the paper, and what is this build's reading where the paper is silent:
+ * What follows the paper, and what is this implementation's reading where the paper is silent:
  *   - Eq. 1-2 (attention decomposition): oracle_decode's merge.
  *   - Algorithm 1 lines 3-8 (select with an eviction strategy, calibrate with the last
  *     query over the evicted KV): oracle_compress / oracle_calibrate_given_indices.

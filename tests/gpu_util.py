@@ -10,7 +10,7 @@ import oracle
 from paper_2507_19906_b200 import binding as cd
 from paper_2507_19906_b200 import workload as wl
 
-OUT_MAX_ABS, OUT_MEAN_ABS, LSE_ABS = 2e-2, 2e-3, 1e-3   # tolerances fixed by the benchmark spec
+OUT_MAX_ABS, OUT_MEAN_ABS, LSE_ABS = 2e-2, 2e-3, 1e-3   # bf16 outputs and O_c: max-abs, mean-abs; log-sum-exps: abs
 SWAP_REL = 1e-5                                         # allowed near-tie swaps in the kept set
 
 

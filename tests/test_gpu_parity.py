@@ -1,6 +1,6 @@
 """GPU parity: the CUDA path through the C-ABI against the fp64 oracle, element by element.
 
-Tolerances are the ones the task fixes: kept-index sets bit-exact except near-tie swaps
+Tolerances: kept-index sets bit-exact except near-tie swaps
 (oracle pooled votes within 1e-5 relative); K_kept/V_kept/C_q bit-exact; O_c and decode
 outputs within max-abs 2e-2 and mean-abs 2e-3; LSE_c and the output LSE within 1e-3.
 """
