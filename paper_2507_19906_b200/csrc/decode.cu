@@ -51,11 +51,11 @@ constexpr int kStreamWarps = 8;
 constexpr int kThreads = (kStreamWarps + 1) * 32;  // the last warp is the producer
 constexpr int kBlkRows = 16;                        // rows of one warp's MMA block
 constexpr int kSlotRows = 64;                       // rows per ring slot: four blocks
-constexpr int kSlots = 6;
+constexpr int kSlotsWide = 6;    // ring of a launch with one CTA per SM at most: 192 KB
+constexpr int kSlotsNarrow = 3;  // ring of a launch with more CTAs than SMs: 96 KB, two CTAs per SM
 constexpr int kPlaneBytes = kSlotRows * 128;        // 64 rows x 64 columns of bf16 (one TMA box)
 constexpr int kSlotBytes = 4 * kPlaneBytes;         // K low / K high / V low / V high column halves
-constexpr int kRingBytes = kSlots * kSlotBytes;     // 192 KB -> one CTA per SM
-constexpr int kSmemBytes = kRingBytes + 1024;       // + slack for the 1024-byte alignment
+constexpr int smem_bytes(int slots) { return slots * kSlotBytes + 1024; }  // + slack for the 1024-byte alignment
 constexpr int kWoStride = kD + 4;  // row stride of the per-warp partial outputs: heads land in distinct banks
 constexpr long long kWaitLimitCycles = 2000000000ll;  // about a second: a wait this long has failed
 
@@ -229,9 +229,12 @@ __device__ __forceinline__ void recal_store(const DecodeCommon& a, const DecodeL
 }
 
 // RECAL = false: the decode step.  RECAL = true: the same stream over the evicted KV, without the
-// similarity and the gate, ending in recal_store.
-template <int NL, bool RECAL>
-__global__ void __launch_bounds__(kThreads, 1) decode_kernel(const __grid_constant__ DecodeArgsT<NL> args) {
+// similarity and the gate, ending in recal_store.  kSlots: ring depth (six slots and one CTA per
+// SM, or three slots and two CTAs per SM for launches of many short, independent slices, where the
+// fixed chain of one CTA is what a second resident CTA can overlap).
+template <int NL, bool RECAL, int kSlots>
+__global__ void __launch_bounds__(kThreads, kSlots > 3 ? 1 : 2)
+decode_kernel(const __grid_constant__ DecodeArgsT<NL> args) {
   extern __shared__ unsigned char smem_raw[];
   __shared__ __align__(8) unsigned long long s_full[kSlots][2], s_empty[kSlots][2];
   __shared__ unsigned long long s_best[kMaxG];     // best (similarity, row) of this CTA's calibration rows
@@ -734,14 +737,15 @@ bool make_decode_maps(const DecodeCommon& c, const DecodeLayerPtrs& L, DecodeLay
 
 namespace {
 
-template <int NL, bool RECAL>
-cudaError_t launch_decode_t(const DecodeArgsT<NL>& a, cudaStream_t st) {
+template <int NL, bool RECAL, int kSlots>
+cudaError_t launch_decode_s(const DecodeArgsT<NL>& a, cudaStream_t st) {
+  constexpr int kSmemBytes = smem_bytes(kSlots);
   static bool attr_set[64] = {};
   int dev = 0;
   cudaError_t e = cudaGetDevice(&dev);
   if (e != cudaSuccess) return e;
   if (dev < 0 || dev >= 64 || !attr_set[dev]) {
-    e = cudaFuncSetAttribute(decode_kernel<NL, RECAL>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+    e = cudaFuncSetAttribute(decode_kernel<NL, RECAL, kSlots>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
     if (e != cudaSuccess) return e;
     if (dev >= 0 && dev < 64) attr_set[dev] = true;
   }
@@ -759,10 +763,21 @@ cudaError_t launch_decode_t(const DecodeArgsT<NL>& a, cudaStream_t st) {
   attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 2;
-  e = cudaLaunchKernelEx(&cfg, decode_kernel<NL, RECAL>, a);
+  e = cudaLaunchKernelEx(&cfg, decode_kernel<NL, RECAL, kSlots>, a);
   if (e != cudaSuccess) return e;
   count_launch(1);
   return cudaGetLastError();
+}
+
+// More CTAs than SMs and short slices (a stack of small caches in one launch): the narrow ring, so
+// that two CTAs share an SM and one's fixed chain overlaps the other's stream.  Long slices keep the
+// wide ring, which they need to stream at full rate (measured: 32 layers of 129-384 rows 115 -> 95 us
+// with the narrow ring, 8 caches of 2049 rows 53 -> 57 us).
+template <int NL, bool RECAL>
+cudaError_t launch_decode_t(const DecodeArgsT<NL>& a, cudaStream_t st) {
+  const long long ctas = (long long)a.c.nsplit * a.c.nclu * a.c.units * a.c.n_layers;
+  const bool narrow = ctas > kDecodeTargetCtas && a.c.rows_per_split <= 8 * kSlotRows;
+  return narrow ? launch_decode_s<NL, RECAL, kSlotsNarrow>(a, st) : launch_decode_s<NL, RECAL, kSlotsWide>(a, st);
 }
 
 }  // namespace
