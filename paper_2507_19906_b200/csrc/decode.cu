@@ -71,7 +71,7 @@ __device__ __forceinline__ uint32_t movmatrix_trans(uint32_t x) {
   return y;
 }
 
-// ---- mbarrier / TMA helpers (no cluster multicast anywhere: every copy lands in this CTA)
+// ---- mbarrier / TMA helpers (every copy lands in the shared memory of the CTA that issued it)
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
   asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
 }
