@@ -528,3 +528,35 @@ def test_gather_evicted_and_recalibrate(cuda_lib, B, Hq, Hkv, L, W, budget, n_ca
         for hq in range(Hq):
             o, _ = oracle.full_attention(q[b, hq][None], K[b, hq // G], V[b, hq // G])
             assert_close_out(got[b, hq], o[0], "decode after the recompute vs attention over the whole prompt")
+
+
+# ---------------------------------------------------------------- seeded random shapes
+def _random_shapes(n, seed):
+    rng = np.random.Generator(np.random.Philox(key=[seed, 1]))
+    out = []
+    for _ in range(n):
+        Hkv = int(rng.integers(1, 5))
+        G = int(rng.integers(1, 9))
+        B = int(rng.integers(1, 4))
+        W = int(rng.choice([1, 2, 4, 8, 16, 32, 64]))
+        if G * W > 512:
+            W = 512 // G
+        L = int(rng.integers(W + 40, 2600))
+        budget = int(rng.integers(W + 1, min(L, W + 700)))
+        pool = int(rng.choice([1, 3, 5, 7]))
+        n_cal = int(rng.integers(1, W + 1))
+        out.append((B, Hkv * G, Hkv, L, W, pool, budget, n_cal))
+    return out
+
+
+@pytest.mark.parametrize("B,Hq,Hkv,L,W,pool,budget,n_cal", _random_shapes(16, 2507))
+def test_compress_and_decode_random_shapes(cuda_lib, B, Hq, Hkv, L, W, pool, budget, n_cal):
+    cfg = wl.small_config(B=B, Hq=Hq, Hkv=Hkv, L=L, window=W, pool=pool, budget=budget, steps=3,
+                          n_sink=2, n_heavy=max(1, L // 50))
+    Q, K, V = _inputs(cfg)
+    T = 3
+    g = gpu_compress(Q, K, V, window=W, pool=pool, budget=budget, n_cal=n_cal, cap=budget + T)
+    ref, _ = compare_compress(g, Q, K, V, window=W, pool=pool, budget=budget, n_cal=n_cal)
+    q, kn, vn = wl.gen_decode_inputs(cfg, Q, steps=T)
+    st = decode_steps_compare(g, ref, q, kn, vn, steps=T)
+    assert st["total"] == T * B * Hq
