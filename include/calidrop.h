@@ -11,6 +11,12 @@
  *                      new query over the retained cache, cosine similarity with the stored
  *                      calibration queries, threshold gate, and the merge of Eq. 1-2.
  *
+ * Around them: calidrop_calibrate (the second half of calidrop_compress for a kept list chosen by
+ * another eviction rule), calidrop_gather_evicted and calidrop_recalibrate (Algorithm 1 line 4 and
+ * Algorithm 2 lines 3-8: the evicted rows compacted for offloading, and the recompute of a
+ * calibration entry from them), calidrop_decode_batched (several layers in one launch) and
+ * calidrop_decode_static (no caller workspace).
+ *
  * Conventions
  *   - Unless a comment says HOST, every tensor pointer is a DEVICE pointer to a contiguous,
  *     16-byte aligned buffer on the current device.  "bf16" buffers hold bfloat16 values.
