@@ -153,6 +153,19 @@ __device__ __forceinline__ float ldg_keep(const float* ptr, uint64_t pol) {
   return v;
 }
 
+// Shared-memory address of `local` in CTA `rank` of the cluster, and an 8-byte store to such an
+// address that reports its bytes to an mbarrier of the same CTA when it lands.
+__device__ __forceinline__ uint32_t cluster_addr(uint32_t local, int rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(local), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ void push_f32x2(uint32_t remote, float x, float y, uint32_t remote_bar) {
+  asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.v2.f32 [%0], {%1, %2}, [%3];" ::"r"(remote),
+               "f"(x), "f"(y), "r"(remote_bar)
+               : "memory");
+}
+
 struct RhoLoad {
   uint4 q0, q1, c0, c1;
 };
@@ -241,6 +254,7 @@ decode_kernel(const __grid_constant__ DecodeArgsT<NL> args) {
   __shared__ unsigned long long s_bestall[kMaxG];  // ... of the whole cluster
   __shared__ __align__(16) float s_xpart[kMaxG * kD];  // [source split][head][dim of this CTA's slice]
   __shared__ __align__(16) float s_xml[8][kMaxG][2];   // [source split][head] (max, sum)
+  __shared__ __align__(8) unsigned long long s_push;  // counts the bytes pushed to this CTA by the cluster
   __shared__ int s_abort;
   __shared__ unsigned s_ticket;
 
@@ -310,6 +324,11 @@ decode_kernel(const __grid_constant__ DecodeArgsT<NL> args) {
     s_abort = 0;
   }
   if (warp == kStreamWarps && lane == 0) {
+    // every CTA of the cluster (this one included) pushes its partial of this CTA's slice and its
+    // (max, sum) pairs here: G * dpc * 4 + G * 8 bytes each
+    mbar_init(smem_u32(&s_push), 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    mbar_expect_tx(smem_u32(&s_push), (uint32_t)(a.nsplit * a.G * (kD / a.nsplit * 4 + 8)));
     asm volatile("prefetch.tensormap [%0];" ::"l"(&TM.k64) : "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(&TM.v64) : "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(&TM.k16) : "memory");
@@ -617,16 +636,18 @@ decode_kernel(const __grid_constant__ DecodeArgsT<NL> args) {
         acc1 = fmaf(wv.y, sc, acc1);
       }
       const int own = d0 >> lg_dpc;  // dpc is even: both dimensions have the same owner
-      *reinterpret_cast<float2*>(cluster.map_shared_rank(s_xpart, own) + (split * kMaxG + g) * dpc +
-                                 (d0 - own * dpc)) = make_float2(acc0, acc1);
+      push_f32x2(cluster_addr(smem_u32(s_xpart + (split * kMaxG + g) * dpc + (d0 - own * dpc)), own), acc0, acc1,
+                 cluster_addr(smem_u32(&s_push), own));
       if ((tid & 63) < a.nsplit) {  // the (max, sum) pair of this split goes to every CTA of the cluster
-        *reinterpret_cast<float2*>(&cluster.map_shared_rank(&s_xml[0][0][0], tid & 63)[(split * kMaxG + g) * 2]) =
-            make_float2(M, Lsum);
+        push_f32x2(cluster_addr(smem_u32(&s_xml[split][g][0]), tid & 63), M, Lsum,
+                   cluster_addr(smem_u32(&s_push), tid & 63));
       }
     }
   }
-  cluster_arrive();  // (B) this CTA's pushes are done
-  cluster_wait();    //     and everything pushed to this CTA has arrived
+  // (B) everything pushed to this CTA has arrived when its byte count is complete.  No cluster
+  // barrier: a CTA waits for its own data only, and it cannot leave before the others have read its
+  // s_best, because their pushes, which it waits for, come after those reads.
+  mbar_wait(smem_u32(&s_push), 0, abort_flag, a.status, 0x300u);
 
   // ---- (6) finish: reduce the splits for this CTA's output slice (local data only from here on,
   // so no CTA has to wait for another before it leaves)
