@@ -37,7 +37,7 @@ UNIT = "GB/s"
 FALLBACK_HBM_GBS, FALLBACK_BF16_TFLOPS = 6650.0, 1590.0
 # dram__bytes_read.sum + dram__bytes_write.sum per decode launch at config 3 from the committed ncu
 # capture (profiles/decode_kernel_config3.md); reported only for that workload.
-DECODE_DRAM_TRAFFIC_PER_LAUNCH = 35871232
+DECODE_DRAM_TRAFFIC_PER_LAUNCH = 35872128
 
 
 def load_peaks():
