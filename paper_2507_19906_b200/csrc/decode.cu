@@ -18,8 +18,9 @@
 //   O^T[128 dims x 8 heads] += V_blk^T[128 x 16 keys] . P^T[16 x 8]     (8 MMAs)
 // The splits are combined inside the cluster through distributed shared memory: every CTA
 // finishes a slice of the 128 output dimensions for all heads of the group, and each CTA pushes
-// its partial of a slice into the shared memory of the slice's owner, so that after one cluster
-// barrier every CTA reduces local data only.  Only when very few units share a very long cache
+// its partial of a slice into the shared memory of the slice's owner with asynchronous stores that
+// report their bytes to an mbarrier there, so that every CTA waits for its own data only and then
+// reduces local data.  Only when very few units share a very long cache
 // (more than 1024 rows per CTA even with a cluster of eight) does a unit get up to eight clusters;
 // each writes its combined partial, its (max, sum) pair and its best similarity to the workspace, and
 // the CTA that takes the last ticket of the unit's arrival counter merges them and resets the counter.
