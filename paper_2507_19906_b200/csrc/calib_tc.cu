@@ -299,7 +299,7 @@ calib_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
         const int kb = tbase + 32 * q;
         word[q] = 0xffffffffu;
         if (kb < a.n_cand) {
-          word[q] = __ldg(bm + (kb >> 5));
+          word[q] = bm_all ? __ldg(bm + (kb >> 5)) : 0u;   // no bitmap: every key below n_cand counts
           if (kb + 32 > a.n_cand) word[q] |= 0xffffffffu << (a.n_cand - kb);
         }
       }
@@ -396,14 +396,14 @@ calib_reduce_kernel(const __nv_bfloat16* __restrict__ Q_obs, const float* __rest
 bool calib_tc_supported(const CompressGeom& g) { return !g.keep_all && g.n_cal <= 128 && g.n_cand >= 1; }
 
 // Row blocks per unit and the tile partition; `parts` = partial (O, l) slots the workspace holds.
-void calib_tc_plan(const CompressGeom& g, int* gpb, int* n_cblocks, int* tiles_per_cta, int* max_slots,
+void calib_tc_plan(const CompressGeom& g, int n_keys, int* gpb, int* n_cblocks, int* tiles_per_cta, int* max_slots,
                    size_t* parts) {
   int per = 128 / g.n_cal;
   if (per < 1) per = 1;
   if (per > g.G) per = g.G;
   *gpb = per;
   *n_cblocks = (g.G + per - 1) / per;
-  const int n_tiles = (g.n_cand + kTileKeys - 1) / kTileKeys;
+  const int n_tiles = (n_keys + kTileKeys - 1) / kTileKeys;
   // the (kv unit, tile) space is shared out over groups of n_cblocks CTAs
   const int total = g.units * n_tiles;
   int groups = kSms / *n_cblocks;
@@ -414,22 +414,25 @@ void calib_tc_plan(const CompressGeom& g, int* gpb, int* n_cblocks, int* tiles_p
   *parts = (size_t)g.units * *n_cblocks * *max_slots;
 }
 
-cudaError_t launch_calib_tc(const CompressGeom& g, const CompressWs& ws, const void* Q_obs, const void* K,
-                            const void* V, const float* row_lse, char* wsp, float* O_c, float* LSE_c, void* C_q,
-                            cudaStream_t st) {
+// The masked sums of one key source: rows [0, n_keys) of every unit of K / V (a unit's rows are
+// `unit_rows` apart), minus the keys whose bit is set in `bitmap` (none when it is null), into the
+// partial arrays o_part / l_part.
+cudaError_t launch_calib_tc_parts(const CompressGeom& g, const void* Q_obs, const void* K, const void* V,
+                                  int n_keys, size_t unit_rows, const uint32_t* bitmap, const float* row_lse,
+                                  float* o_part, float* l_part, unsigned* status, cudaStream_t st) {
   CalibArgs a{};
-  a.Hq = g.Hq; a.G = g.G; a.W = g.W; a.L = g.L; a.n_cand = g.n_cand; a.n_cal = g.n_cal;
+  a.Hq = g.Hq; a.G = g.G; a.W = g.W; a.L = g.L; a.n_cand = n_keys; a.n_cal = g.n_cal;
   size_t parts;
-  calib_tc_plan(g, &a.gpb, &a.n_cblocks, &a.tiles_per_cta, &a.max_slots, &parts);
-  a.n_tiles = (g.n_cand + kTileKeys - 1) / kTileKeys;
+  calib_tc_plan(g, n_keys, &a.gpb, &a.n_cblocks, &a.tiles_per_cta, &a.max_slots, &parts);
+  a.n_tiles = (n_keys + kTileKeys - 1) / kTileKeys;
   a.total_tiles = g.units * a.n_tiles;
   a.bitmap_words = g.bitmap_words;
   a.scale2 = g.scale2;
   a.row_lse = row_lse;
-  a.bitmap = (const uint32_t*)(wsp + ws.bitmap);
-  a.o_part = (float*)(wsp + ws.calib_o);
-  a.l_part = (float*)(wsp + ws.calib_l);
-  a.status = (unsigned*)(wsp + ws.status);
+  a.bitmap = bitmap;
+  a.o_part = o_part;
+  a.l_part = l_part;
+  a.status = status;
   CUtensorMap qm, km, vm;
   // calibration rows: [head dim][c < n_cal][g < G][unit], starting at observation row W - n_cal
   const uint64_t qd[3] = {(uint64_t)g.n_cal, (uint64_t)g.G, (uint64_t)g.units};
@@ -437,7 +440,8 @@ cudaError_t launch_calib_tc(const CompressGeom& g, const CompressWs& ws, const v
   const uint32_t qb[3] = {(uint32_t)g.n_cal, (uint32_t)a.gpb, 1};
   const char* q0 = (const char*)Q_obs + (size_t)(g.W - g.n_cal) * 256;
   if (!make_tensor_map_bf16(&qm, q0, 4, qd, qs, qb)) return cudaErrorInvalidValue;
-  const uint64_t kd[2] = {(uint64_t)g.L, (uint64_t)g.units}, ks[2] = {256, (uint64_t)g.L * 256};
+  // rows at or beyond n_keys are never used (their probabilities are masked), so the maps end there
+  const uint64_t kd[2] = {(uint64_t)n_keys, (uint64_t)g.units}, ks[2] = {256, (uint64_t)unit_rows * 256};
   const uint32_t kb[2] = {(uint32_t)kTileKeys, 1};
   if (!make_tensor_map_bf16(&km, K, 3, kd, ks, kb) || !make_tensor_map_bf16(&vm, V, 3, kd, ks, kb))
     return cudaErrorInvalidValue;
@@ -452,11 +456,27 @@ cudaError_t launch_calib_tc(const CompressGeom& g, const CompressWs& ws, const v
   }
   const int grid = (a.total_tiles + a.tiles_per_cta - 1) / a.tiles_per_cta * a.n_cblocks;
   calib_tc_kernel<<<grid, kThreads, kSmemBytes, st>>>(qm, km, vm, a);
+  count_launch(1);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_calib_tc(const CompressGeom& g, const CompressWs& ws, const void* Q_obs, const void* K,
+                            const void* V, const float* row_lse, char* wsp, float* O_c, float* LSE_c, void* C_q,
+                            cudaStream_t st) {
+  float* o_part = (float*)(wsp + ws.calib_o);
+  float* l_part = (float*)(wsp + ws.calib_l);
+  cudaError_t e = launch_calib_tc_parts(g, Q_obs, K, V, g.n_cand, (size_t)g.L, (const uint32_t*)(wsp + ws.bitmap),
+                                        row_lse, o_part, l_part, (unsigned*)(wsp + ws.status), st);
+  if (e != cudaSuccess) return e;
+  int gpb, n_cblocks, tiles_per_cta, max_slots;
+  size_t parts;
+  calib_tc_plan(g, g.n_cand, &gpb, &n_cblocks, &tiles_per_cta, &max_slots, &parts);
   const int total = g.B * g.Hq * g.n_cal;
-  calib_reduce_kernel<<<(total + 3) / 4, 128, 0, st>>>((const __nv_bfloat16*)Q_obs, row_lse, a.o_part, a.l_part, O_c,
+  calib_reduce_kernel<<<(total + 3) / 4, 128, 0, st>>>((const __nv_bfloat16*)Q_obs, row_lse, o_part, l_part, O_c,
                                                       LSE_c, (__nv_bfloat16*)C_q, g.B, g.Hq, g.G, g.W, g.n_cal,
-                                                      a.gpb, a.n_cblocks, a.n_tiles, a.tiles_per_cta, a.max_slots);
-  count_launch(2);
+                                                      gpb, n_cblocks, (g.n_cand + kTileKeys - 1) / kTileKeys,
+                                                      tiles_per_cta, max_slots);
+  count_launch(1);
   return cudaGetLastError();
 }
 
