@@ -20,6 +20,8 @@
 // Warp roles: two softmax warpgroups (group g owns S buffer g and P buffer g, i.e. the tiles with
 // local index i % 2 == g), one TMA producer warp, one warp that allocates TMEM and issues MMAs.
 // Tensor memory: S buffers at columns 0 and 128, O at 256, P buffers (64 columns each) at 384, 448.
+#include <type_traits>
+
 #include "internal.h"
 #include "tc_common.cuh"
 
@@ -53,7 +55,20 @@ struct CalibArgs {
   float* o_part;           // [virtual unit][slot][128][128]
   float* l_part;           // [virtual unit][slot][group][128]
   unsigned* status;
+  // Work-list mode (null = every unit): the kernel runs over the units listed in work_list only,
+  // n_work of them (read on the device, so the grid is fixed while the work is not), shared out
+  // evenly over the CTA groups; partials are then indexed [CTA group][segment < seg_max][row block].
+  const int* work_list;
+  const int* n_work;
+  int units, seg_max;
 };
+
+// Tiles per CTA group when n_units units are shared out over `groups` groups.
+__host__ __device__ inline int tiles_per_group(int n_units, int n_tiles, int groups) {
+  const long long total = (long long)n_units * n_tiles;
+  const long long t = (total + groups - 1) / groups;
+  return t < 1 ? 1 : (int)t;
+}
 
 __global__ void __launch_bounds__(kThreads, 1)
 calib_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__ CUtensorMap k_map,
@@ -68,10 +83,17 @@ calib_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
   // range at the same pace, one calibration row block each, so that a K/V tile fetched for one
   // of them is still in L2 when the others ask for it and crosses the HBM interface once.
   const int cta = blockIdx.x / a.n_cblocks, cb = blockIdx.x % a.n_cblocks;
-  const int g_begin = cta * a.tiles_per_cta;
-  const int g_end = min(a.total_tiles, g_begin + a.tiles_per_cta);
+  const bool listed = a.work_list != nullptr;
+  const int n_units = listed ? *a.n_work : a.units;
+  if (n_units <= 0) return;   // nothing listed: uniform over the grid, before anything is set up
+  const int total_tiles = n_units * a.n_tiles;
+  const int tiles_per_cta = listed ? tiles_per_group(n_units, a.n_tiles, gridDim.x / a.n_cblocks) : a.tiles_per_cta;
+  const int g_begin = cta * tiles_per_cta;
+  const int g_end = min(total_tiles, g_begin + tiles_per_cta);
   const int nt = g_end - g_begin;
   const int Hkv = a.Hq / a.G;
+  // position in the (listed) unit space -> the unit itself
+  auto unit_of = [&](int pos) { return listed ? a.work_list[pos] : pos; };
 
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   const uint32_t q_base = smem_base;
@@ -137,7 +159,7 @@ calib_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
           const int g0 = (vu - unit * a.n_cblocks) * a.gpb;
           mbar_arrive_expect_tx(q_full, 2u * (uint32_t)(a.gpb * a.n_cal) * kLineBytes);
           for (int half = 0; half < 2; ++half)
-            tma_load_4d(q_base + half * (kTileBytes / 2), &q_map, q_full, half * kHalfCols, 0, g0, unit);
+            tma_load_4d(q_base + half * (kTileBytes / 2), &q_map, q_full, half * kHalfCols, 0, g0, unit_of(unit));
           ++seg;
         }
         const int s = i % kStages;
@@ -146,12 +168,12 @@ calib_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
         mbar_arrive_expect_tx(full_k(s), kTileBytes);
         for (int half = 0; half < 2; ++half)
           tma_load_3d(k_base + s * kTileBytes + half * (kTileBytes / 2), &k_map, full_k(s), half * kHalfCols,
-                      tile * kTileKeys, unit);
+                      tile * kTileKeys, unit_of(unit));
         if (!mbar_wait(&ctl, empty_v(s), ph, 22u | ((unsigned)i << 8))) break;
         mbar_arrive_expect_tx(full_v(s), kTileBytes);
         for (int half = 0; half < 2; ++half)
           tma_load_3d(v_base + s * kTileBytes + half * (kTileBytes / 2), &v_map, full_v(s), half * kHalfCols,
-                      tile * kTileKeys, unit);
+                      tile * kTileKeys, unit_of(unit));
       }
     }
   } else if (warp == kMmaWarp) {
@@ -166,20 +188,41 @@ calib_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
       const uint32_t tmem_o = tmem_base + kColO;
       int seg = 0;
       bool ok = true;
-      // k-step kk of S(i) and of P.V(i)
-      auto s_step = [&](int i, int kk) {
-        const int s = i % kStages;
-        umma_ss(tmem_base + (uint32_t)((i & 1) * 128), kmajor_desc(q_base, kTileBytes / 2, kk),
-                kmajor_desc(k_base + s * kTileBytes, kTileBytes / 2, kk), idesc, kk > 0 ? 1u : 0u);
+      // Descriptors are built once per buffer and a k-step adds a constant to the address field: the
+      // issuing thread's own instructions between two MMAs are what limits the issue rate.
+      const uint64_t dq = smem_desc_sw128(q_base, 16u, 1024u);
+      const uint64_t dk0 = smem_desc_sw128(k_base, 16u, 1024u);
+      // V tile with the keys as K, i.e. MN-major: blocks of 64 head-dim elements are half a tile
+      // apart, groups of 8 keys 1024 bytes apart
+      const uint64_t dv0 = smem_desc_sw128(v_base, kTileBytes / 2, 1024u);
+      const uint32_t tmem_p = tmem_base + kColP;
+      // S(i): eight k-steps
+      auto s_steps = [&](int i) {
+        const uint32_t d = tmem_base + (uint32_t)((i & 1) * 128);
+        const uint64_t kd = desc_advance(dk0, (uint32_t)(i % kStages) * kTileBytes);
+        umma_ss_imm<0>(d, dq, kd, idesc);
+#pragma unroll
+        for (int kk = 1; kk < kD / 16; ++kk)
+          umma_ss_imm<1>(d, desc_advance(dq, kmajor_step_bytes(kTileBytes / 2, kk)),
+                         desc_advance(kd, kmajor_step_bytes(kTileBytes / 2, kk)), idesc);
       };
-      auto pv_step = [&](int i, int kk, bool first) {
-        // A: P, 16 keys = 8 columns per step.  B: V tile with the keys as K, i.e. MN-major: blocks
-        // of 64 head-dim elements are half a tile apart, groups of 8 keys 1024 bytes apart.
-        const int s = i % kStages;
-        const uint64_t vd = smem_desc_sw128(v_base + s * kTileBytes + (uint32_t)kk * 16u * kLineBytes,
-                                            kTileBytes / 2, 1024u);
-        umma_ts(tmem_o, tmem_base + kColP + (uint32_t)((i & 1) * 64 + kk * 8), vd, idesc_o,
-                (!first || kk > 0) ? 1u : 0u);
+      // P.V(i) (A: P in tensor memory, 16 keys = 8 columns per step), with or without S(i + 2) interleaved
+      auto batch = [&](int i, auto first_tag, auto with_s_tag) {
+        constexpr bool kFirst = decltype(first_tag)::value, kWithS = decltype(with_s_tag)::value;
+        const uint64_t vd = desc_advance(dv0, (uint32_t)(i % kStages) * kTileBytes);
+        const uint32_t pa = tmem_p + (uint32_t)((i & 1) * 64);
+        const uint32_t d = tmem_base + (uint32_t)((i & 1) * 128);
+        const uint64_t kd = desc_advance(dk0, (uint32_t)((i + 2) % kStages) * kTileBytes);
+#pragma unroll
+        for (int kk = 0; kk < kTileKeys / 16; ++kk) {
+          if (kFirst && kk == 0) umma_ts_imm<0>(tmem_o, pa, vd, idesc_o);
+          else umma_ts_imm<1>(tmem_o, pa + (uint32_t)(kk * 8), desc_advance(vd, (uint32_t)kk * 16u * kLineBytes), idesc_o);
+          if (kWithS) {
+            if (kk == 0) umma_ss_imm<0>(d, dq, kd, idesc);
+            else umma_ss_imm<1>(d, desc_advance(dq, kmajor_step_bytes(kTileBytes / 2, kk)),
+                                desc_advance(kd, kmajor_step_bytes(kTileBytes / 2, kk)), idesc);
+          }
+        }
       };
       auto wait_k = [&](int i) { return mbar_wait(&ctl, full_k(i % kStages), (i / kStages) & 1, 24u | ((unsigned)i << 8)); };
       auto s_done = [&](int i) { umma_commit(s_full(i & 1)); umma_commit(empty_k(i % kStages)); };
@@ -198,11 +241,8 @@ calib_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
           ok = wait_k(i) && (!two || wait_k(i + 1));
           if (!ok) break;
           tc_fence_after_sync();
-#pragma unroll
-          for (int kk = 0; kk < kD / 16; ++kk) {
-            s_step(i, kk);
-            if (two) s_step(i + 1, kk);
-          }
+          s_steps(i);
+          if (two) s_steps(i + 1);
           s_done(i);
           if (two) s_done(i + 1);
         }
@@ -212,10 +252,12 @@ calib_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
         if (!mbar_wait(&ctl, full_v(i % kStages), (i / kStages) & 1, 27u | ((unsigned)i << 8))) break;
         if (with_s && !wait_k(i + 2)) break;
         tc_fence_after_sync();
-#pragma unroll
-        for (int kk = 0; kk < kTileKeys / 16; ++kk) {
-          pv_step(i, kk, first);
-          if (with_s) s_step(i + 2, kk);
+        if (with_s) {
+          if (first) batch(i, std::true_type{}, std::true_type{});
+          else batch(i, std::false_type{}, std::true_type{});
+        } else {
+          if (first) batch(i, std::true_type{}, std::false_type{});
+          else batch(i, std::false_type{}, std::false_type{});
         }
         if (with_s) s_done(i + 2);
         umma_commit(empty_v(i % kStages));
@@ -242,8 +284,9 @@ calib_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
       w = __all_sync(0xffffffffu, w);
       if (!w) return false;
       tc_fence_after_sync();
-      const int slot = cta - ((vu / a.n_cblocks) * a.n_tiles) / a.tiles_per_cta;
-      const size_t part = (size_t)vu * a.max_slots + slot;
+      const int slot = cta - ((vu / a.n_cblocks) * a.n_tiles) / tiles_per_cta;
+      const size_t part = listed ? ((size_t)cta * a.seg_max + (seg - 1)) * a.n_cblocks + cb
+                                 : (size_t)vu * a.max_slots + slot;
       float* orow = a.o_part + (part * 128 + r) * kD;
 #pragma unroll 1
       for (int c0 = grp * 64; c0 < grp * 64 + 64; c0 += 32) {
@@ -262,7 +305,8 @@ calib_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
     };
     // This thread's row of the virtual unit: is there one, and its -lse2.
     auto load_q = [&](int vu) {
-      const int unit = vu / a.n_cblocks, cb = vu - unit * a.n_cblocks;
+      const int pos = vu / a.n_cblocks, cb = vu - pos * a.n_cblocks;
+      const int unit = unit_of(pos);
       const int hq0 = (unit / Hkv) * a.Hq + (unit % Hkv) * a.G;
       const int g0 = cb * a.gpb;
       const int rows = min(a.gpb, a.G - g0) * a.n_cal;
@@ -291,7 +335,7 @@ calib_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
       if ((i & 1) != grp) continue;
       // kept-key bits of the tile's 128 keys (bit set = the key does not contribute), fetched
       // before the wait so that the loads are off the critical path
-      const uint32_t* bm = bm_all + (size_t)unit * a.bitmap_words;
+      const uint32_t* bm = bm_all + (size_t)unit_of(unit) * a.bitmap_words;
       const int tbase = tile * kTileKeys;
       uint32_t word[4];
 #pragma unroll
@@ -359,7 +403,8 @@ calib_reduce_kernel(const __nv_bfloat16* __restrict__ Q_obs, const float* __rest
                     const float* __restrict__ o_part, const float* __restrict__ l_part,
                     float* __restrict__ O_c, float* __restrict__ LSE_c, __nv_bfloat16* __restrict__ C_q, int B,
                     int Hq, int G, int W, int n_cal, int gpb, int n_cblocks, int n_tiles, int tiles_per_cta,
-                    int max_slots) {
+                    int max_slots, const int* __restrict__ unit_pos, const int* __restrict__ n_work, int groups,
+                    int seg_max) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int row = blockIdx.x * 4 + warp;  // (b, hq, c)
   if (row >= B * Hq * n_cal) return;
@@ -367,15 +412,24 @@ calib_reduce_kernel(const __nv_bfloat16* __restrict__ Q_obs, const float* __rest
   const int b = bhq / Hq, hq = bhq % Hq;
   const int Hkv = Hq / G, h = hq / G, g = hq % G;
   const int unit = b * Hkv + h, cb = g / gpb, r = (g % gpb) * n_cal + c;
-  const int vu = unit * n_cblocks + cb;
-  const int first = (unit * n_tiles) / tiles_per_cta, last = ((unit + 1) * n_tiles - 1) / tiles_per_cta;
-  const size_t part0 = (size_t)vu * max_slots;
+  // Work-list mode (unit_pos given): only the rows of listed units are rewritten; the partials
+  // are those of the CTA groups whose share of the listed tile space overlaps the unit.
+  const bool listed = unit_pos != nullptr;
+  int pos = unit;
+  if (listed) {
+    pos = unit_pos[unit];
+    if (pos < 0) return;
+    tiles_per_cta = tiles_per_group(*n_work, n_tiles, groups);
+  }
+  const int first = (pos * n_tiles) / tiles_per_cta, last = ((pos + 1) * n_tiles - 1) / tiles_per_cta;
   float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
   float l = 0.f;
   for (int s = 0; s <= last - first; ++s) {
-    const float4 v = *reinterpret_cast<const float4*>(o_part + ((part0 + s) * 128 + r) * kD + 4 * lane);
+    const size_t part = listed ? ((size_t)(first + s) * seg_max + (pos - ((first + s) * tiles_per_cta) / n_tiles)) * n_cblocks + cb
+                               : (size_t)(unit * n_cblocks + cb) * max_slots + s;
+    const float4 v = *reinterpret_cast<const float4*>(o_part + (part * 128 + r) * kD + 4 * lane);
     acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
-    for (int grp = 0; grp < kGroups; ++grp) l += l_part[((part0 + s) * kGroups + grp) * 128 + r];
+    for (int grp = 0; grp < kGroups; ++grp) l += l_part[(part * kGroups + grp) * 128 + r];
   }
   const int qrow = W - n_cal + c;
   float4 out = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -414,13 +468,30 @@ void calib_tc_plan(const CompressGeom& g, int n_keys, int* gpb, int* n_cblocks, 
   *parts = (size_t)g.units * *n_cblocks * *max_slots;
 }
 
+// Work-list mode: the grid is `groups` CTA groups whatever the number of listed units; a group's share
+// then spans at most seg_max units, and `parts` partial slots cover every (group, segment, row block).
+void calib_tc_list_plan(const CompressGeom& g, int n_keys, int* groups, int* seg_max, size_t* parts) {
+  int gpb, n_cblocks, tpc, max_slots;
+  size_t p;
+  calib_tc_plan(g, n_keys, &gpb, &n_cblocks, &tpc, &max_slots, &p);
+  int gr = kSms / n_cblocks;
+  if (gr < 1) gr = 1;
+  const int n_tiles = (n_keys + kTileKeys - 1) / kTileKeys;
+  const int tpc_max = tiles_per_group(g.units, n_tiles, gr);   // the share grows with the number of listed units
+  *groups = gr;
+  *seg_max = (tpc_max + n_tiles - 1) / n_tiles + 1;
+  *parts = (size_t)gr * *seg_max * n_cblocks;
+}
+
 // The masked sums of one key source: rows [0, n_keys) of every unit of K / V (a unit's rows are
 // `unit_rows` apart), minus the keys whose bit is set in `bitmap` (none when it is null), into the
 // partial arrays o_part / l_part.
 cudaError_t launch_calib_tc_parts(const CompressGeom& g, const void* Q_obs, const void* K, const void* V,
                                   int n_keys, size_t unit_rows, const uint32_t* bitmap, const float* row_lse,
-                                  float* o_part, float* l_part, unsigned* status, cudaStream_t st) {
+                                  float* o_part, float* l_part, unsigned* status, const int* work_list,
+                                  const int* n_work, cudaStream_t st) {
   CalibArgs a{};
+  a.work_list = work_list; a.n_work = n_work; a.units = g.units;
   a.Hq = g.Hq; a.G = g.G; a.W = g.W; a.L = g.L; a.n_cand = n_keys; a.n_cal = g.n_cal;
   size_t parts;
   calib_tc_plan(g, n_keys, &a.gpb, &a.n_cblocks, &a.tiles_per_cta, &a.max_slots, &parts);
@@ -454,7 +525,13 @@ cudaError_t launch_calib_tc_parts(const CompressGeom& g, const void* Q_obs, cons
     if (e != cudaSuccess) return e;
     if (dev >= 0 && dev < 64) attr_set[dev] = true;
   }
-  const int grid = (a.total_tiles + a.tiles_per_cta - 1) / a.tiles_per_cta * a.n_cblocks;
+  int grid = (a.total_tiles + a.tiles_per_cta - 1) / a.tiles_per_cta * a.n_cblocks;
+  if (work_list) {
+    // listed units only: a fixed grid of whole CTA groups, the shares are worked out on the device
+    int groups;
+    calib_tc_list_plan(g, n_keys, &groups, &a.seg_max, &parts);
+    grid = groups * a.n_cblocks;
+  }
   calib_tc_kernel<<<grid, kThreads, kSmemBytes, st>>>(qm, km, vm, a);
   count_launch(1);
   return cudaGetLastError();
@@ -466,7 +543,7 @@ cudaError_t launch_calib_tc(const CompressGeom& g, const CompressWs& ws, const v
   float* o_part = (float*)(wsp + ws.calib_o);
   float* l_part = (float*)(wsp + ws.calib_l);
   cudaError_t e = launch_calib_tc_parts(g, Q_obs, K, V, g.n_cand, (size_t)g.L, (const uint32_t*)(wsp + ws.bitmap),
-                                        row_lse, o_part, l_part, (unsigned*)(wsp + ws.status), st);
+                                        row_lse, o_part, l_part, (unsigned*)(wsp + ws.status), nullptr, nullptr, st);
   if (e != cudaSuccess) return e;
   int gpb, n_cblocks, tiles_per_cta, max_slots;
   size_t parts;
@@ -475,7 +552,32 @@ cudaError_t launch_calib_tc(const CompressGeom& g, const CompressWs& ws, const v
   calib_reduce_kernel<<<(total + 3) / 4, 128, 0, st>>>((const __nv_bfloat16*)Q_obs, row_lse, o_part, l_part, O_c,
                                                       LSE_c, (__nv_bfloat16*)C_q, g.B, g.Hq, g.G, g.W, g.n_cal,
                                                       gpb, n_cblocks, (g.n_cand + kTileKeys - 1) / kTileKeys,
-                                                      tiles_per_cta, max_slots);
+                                                      tiles_per_cta, max_slots, nullptr, nullptr, 0, 0);
+  count_launch(1);
+  return cudaGetLastError();
+}
+
+// The masked calibration pass over the units listed on the device (work_list, *n_work; unit_pos is
+// the inverse map, -1 for the others): only their rows of O_c / LSE_c / C_q are rewritten.  With
+// nothing listed both launches return at once.
+cudaError_t launch_calib_tc_listed(const CompressGeom& g, const CompressWs& ws, const void* Q_obs, const void* K,
+                                   const void* V, const float* row_lse, char* wsp, const int* work_list,
+                                   const int* unit_pos, const int* n_work, float* O_c, float* LSE_c, void* C_q,
+                                   cudaStream_t st) {
+  float* o_part = (float*)(wsp + ws.calib_o);
+  float* l_part = (float*)(wsp + ws.calib_l);
+  cudaError_t e = launch_calib_tc_parts(g, Q_obs, K, V, g.n_cand, (size_t)g.L, (const uint32_t*)(wsp + ws.bitmap),
+                                        row_lse, o_part, l_part, (unsigned*)(wsp + ws.status), work_list, n_work, st);
+  if (e != cudaSuccess) return e;
+  int gpb, n_cblocks, tiles_per_cta, max_slots, groups, seg_max;
+  size_t parts;
+  calib_tc_plan(g, g.n_cand, &gpb, &n_cblocks, &tiles_per_cta, &max_slots, &parts);
+  calib_tc_list_plan(g, g.n_cand, &groups, &seg_max, &parts);
+  const int total = g.B * g.Hq * g.n_cal;
+  calib_reduce_kernel<<<(total + 3) / 4, 128, 0, st>>>((const __nv_bfloat16*)Q_obs, row_lse, o_part, l_part, O_c,
+                                                      LSE_c, (__nv_bfloat16*)C_q, g.B, g.Hq, g.G, g.W, g.n_cal,
+                                                      gpb, n_cblocks, (g.n_cand + kTileKeys - 1) / kTileKeys,
+                                                      tiles_per_cta, max_slots, unit_pos, n_work, groups, seg_max);
   count_launch(1);
   return cudaGetLastError();
 }

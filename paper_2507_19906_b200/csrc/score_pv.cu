@@ -9,10 +9,13 @@
 //     sum over evicted = sum over ALL candidates - sum over the selected candidates.
 // This kernel forms the first sum (O_all = P V and the row sums l_all over every candidate key)
 // while it computes the votes, i.e. K is streamed once for both results and V once; the second sum
-// runs afterwards over the few selected rows, which by then lie compacted in K_kept / V_kept
-// (calib_tc_kernel on those), and calib_combine_kernel subtracts.  The same bf16-rounded
-// probabilities enter both sums, so their rounding cancels in the difference; what remains is the
-// fp32 accumulation error of the two sums, relative to the evicted share of the softmax mass.
+// runs afterwards over the few selected rows, which by then lie compacted in K_kept / V_kept (this
+// same kernel on those, without the votes), and calib_combine_kernel subtracts.  Because both sums
+// come from the same instruction sequence, a selected key has bit-identical logits and hence the
+// same bf16-rounded probability in both, so its terms cancel exactly; what remains is the fp32
+// accumulation error of the two sums, relative to the evicted share of the softmax mass.  (With
+// the second sum taken by calib_tc_kernel, whose MMA has the operands the other way round, single
+// probabilities differed by one bf16 step, which showed in O_c at 4e-2 when the key was a heavy one.)
 //
 // Work is the linear space of (kv unit, 128-key tile) pairs, cut into equal contiguous ranges; the
 // CTAs of the row blocks of a unit (a row block = whole query heads, at most 128 window rows) walk
@@ -49,10 +52,10 @@ constexpr int kTmemCols = 512;
 constexpr uint32_t kColO = 256;
 constexpr int kStages = 2;                 // K ring and V ring alike
 constexpr int kTileBytes = kKvTileBytes;   // 32 KB
-constexpr int kNumBars = 24;
+constexpr int kNumBars = 20;
 // dynamic shared memory: Q block, two P^T buffers, K ring, V ring (1024-byte aligned), then the
-// barriers, the -lse2 table, the vote exchange, the control block and the TMEM slot
-constexpr int kMiscBytes = kNumBars * 8 + 128 * 4 + 2 * 128 * 4 + 32;
+// barriers, the -lse2 table, the control block and the TMEM slot
+constexpr int kMiscBytes = kNumBars * 8 + 128 * 4 + 32;
 constexpr int kSmemBytes = (3 + 2 * kStages) * kTileBytes + 1024 + kMiscBytes;
 static_assert(kSmemBytes <= 232448, "shared memory of score_pv_kernel exceeds one SM");
 constexpr int kSms = 148;
@@ -66,7 +69,7 @@ struct PvArgs {
   int total_tiles, tiles_per_cta, max_slots;
   float scale2;
   const float* row_lse;   // [B, Hq, W] natural log
-  float* vote;            // [n_cblocks][units][n_cand]: the partial vote of every row block
+  float* vote;            // [n_cblocks][2][units][n_cand]: the partial votes of the halves of every row block
   size_t vote_stride;     // units * n_cand
   float* o_part;          // [virtual unit][slot][128 rows][128]
   float* l_part;          // [virtual unit][slot][8 warps][64 rows]
@@ -80,7 +83,9 @@ __device__ __forceinline__ void tma_prefetch_l2_3d(const CUtensorMap* map, int c
 }
 
 __device__ __forceinline__ void st_shared_v4(uint32_t addr, uint32_t x, uint32_t y, uint32_t z, uint32_t w) {
-  asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(x), "r"(y), "r"(z), "r"(w) : "memory");
+  // (no memory clobber: the compiler may move its own loads across it; the proxy fence that
+  // follows the last store is volatile too and stays behind every one of them)
+  asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(x), "r"(y), "r"(z), "r"(w));
 }
 
 __global__ void __launch_bounds__(kThreads, 1)
@@ -104,8 +109,7 @@ score_pv_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
   unsigned char* const misc = smem_al + (3 + 2 * kStages) * kTileBytes;
   unsigned long long* const bars = reinterpret_cast<unsigned long long*>(misc);
   float* const nlse2_s = reinterpret_cast<float*>(misc + kNumBars * 8);       // [128]
-  float* const vx = nlse2_s + 128;                                             // [2][128]
-  Ctl* const ctl = reinterpret_cast<Ctl*>(vx + 256);
+  Ctl* const ctl = reinterpret_cast<Ctl*>(nlse2_s + 128);
   uint32_t* const tmem_slot = reinterpret_cast<uint32_t*>(ctl + 1);
 
   const uint32_t bar0 = smem_u32(bars);
@@ -118,8 +122,6 @@ score_pv_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
   auto s_full = [&](int b) { return bar(14 + b); };
   auto p_full = [&](int b) { return bar(16 + b); };
   auto p_empty = [&](int b) { return bar(18 + b); };
-  auto vx_full = [&](int b) { return bar(20 + b); };
-  auto vx_empty = [&](int b) { return bar(22 + b); };
 
   if (tid == 0) {
     ctl->abort = 0;
@@ -135,7 +137,6 @@ score_pv_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
     }
     for (int b = 0; b < 2; ++b) {
       mbar_init(s_full(b), 1); mbar_init(p_full(b), kGroups * 128); mbar_init(p_empty(b), 1);
-      mbar_init(vx_full(b), 128); mbar_init(vx_empty(b), 128);
     }
     fence_mbar_init();
   }
@@ -234,18 +235,40 @@ score_pv_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
       const uint32_t tmem_o = tmem_base + kColO;
       int seg = 0;
       bool ok = true;
-      auto s_step = [&](int i, int kk) {
-        const int s = i % kStages;
-        umma_ss(tmem_base + (uint32_t)((i & 1) * 128), kmajor_desc(k_base + s * kTileBytes, kTileBytes / 2, kk),
-                kmajor_desc(q_base, kTileBytes / 2, kk), idesc_s, kk > 0 ? 1u : 0u);
+      // Descriptors of every operand buffer, built once; a k-step adds a constant to the address field.
+      const uint64_t dq = smem_desc_sw128(q_base, 16u, 1024u);
+      static_assert(kStages == 2, "the ring slots are picked by the parity of the tile index");
+      const uint64_t dk0 = smem_desc_sw128(k_base, 16u, 1024u), dk1 = desc_advance(dk0, kTileBytes);
+      const uint64_t dv0 = smem_desc_sw128(v_base, kTileBytes / 2, 1024u), dv1 = desc_advance(dv0, kTileBytes);
+      const uint64_t dp0 = smem_desc_sw128(p_base, kTileBytes / 2, 1024u), dp1 = desc_advance(dp0, kTileBytes);
+      // S(i): eight k-steps, K-major operands
+      auto s_steps = [&](int i) {
+        const uint32_t d = tmem_base + (uint32_t)((i & 1) * 128);
+        const uint64_t kd = (i & 1) ? dk1 : dk0;
+        umma_ss_imm<0>(d, kd, dq, idesc_s);
+#pragma unroll
+        for (int kk = 1; kk < kD / 16; ++kk)
+          umma_ss_imm<1>(d, desc_advance(kd, kmajor_step_bytes(kTileBytes / 2, kk)),
+                         desc_advance(dq, kmajor_step_bytes(kTileBytes / 2, kk)), idesc_s);
       };
-      auto pv_step = [&](int i, int kk, bool first) {
-        // 16 keys per step.  Both operands have the keys as K and 64-element blocks along M / N half a
-        // tile apart, groups of 8 keys 1024 bytes apart.
-        const uint32_t koff = (uint32_t)kk * 16u * kLineBytes;
-        const uint64_t vd = smem_desc_sw128(v_base + (i % kStages) * kTileBytes + koff, kTileBytes / 2, 1024u);
-        const uint64_t pd = smem_desc_sw128(p_base + (i & 1) * kTileBytes + koff, kTileBytes / 2, 1024u);
-        umma_ss(tmem_o, vd, pd, idesc_o, (!first || kk > 0) ? 1u : 0u);
+      // P.V(i) with or without S(i2) interleaved: 16 keys per step; both P.V operands have the keys
+      // as K (MN-major), 64-element blocks along M / N half a tile apart, groups of 8 keys 1024 bytes apart
+      auto batch = [&](int i, auto first_tag, auto with_s_tag) {
+        constexpr bool kFirst = decltype(first_tag)::value, kWithS = decltype(with_s_tag)::value;
+        const uint64_t vd = (i & 1) ? dv1 : dv0, pd = (i & 1) ? dp1 : dp0;
+        const uint32_t d = tmem_base + (uint32_t)((i & 1) * 128);   // S(i+2) reuses the buffer of S(i)
+        const uint64_t kd = (i & 1) ? dk1 : dk0;                    // and K(i+2) the ring slot of K(i)
+#pragma unroll
+        for (int kk = 0; kk < kTileKeys / 16; ++kk) {
+          const uint32_t koff = (uint32_t)kk * 16u * kLineBytes;
+          if (kFirst && kk == 0) umma_ss_imm<0>(tmem_o, vd, pd, idesc_o);
+          else umma_ss_imm<1>(tmem_o, desc_advance(vd, koff), desc_advance(pd, koff), idesc_o);
+          if (kWithS) {
+            if (kk == 0) umma_ss_imm<0>(d, kd, dq, idesc_s);
+            else umma_ss_imm<1>(d, desc_advance(kd, kmajor_step_bytes(kTileBytes / 2, kk)),
+                                desc_advance(dq, kmajor_step_bytes(kTileBytes / 2, kk)), idesc_s);
+          }
+        }
       };
       auto wait_k = [&](int i) { return mbar_wait(ctl, full_k(i % kStages), (i / kStages) & 1, 44u | ((unsigned)i << 8)); };
       auto s_done = [&](int i) { umma_commit(s_full(i & 1)); umma_commit(empty_k(i % kStages)); };
@@ -264,11 +287,8 @@ score_pv_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
           ok = wait_k(i) && (!two || wait_k(i + 1));
           if (!ok) break;
           tc_fence_after_sync();
-#pragma unroll
-          for (int kk = 0; kk < kD / 16; ++kk) {
-            s_step(i, kk);
-            if (two) s_step(i + 1, kk);
-          }
+          s_steps(i);
+          if (two) s_steps(i + 1);
           s_done(i);
           if (two) s_done(i + 1);
         }
@@ -278,10 +298,12 @@ score_pv_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
         if (!mbar_wait(ctl, full_v(i % kStages), (i / kStages) & 1, 47u | ((unsigned)i << 8))) break;
         if (with_s && !wait_k(i + 2)) break;
         tc_fence_after_sync();
-#pragma unroll
-        for (int kk = 0; kk < kTileKeys / 16; ++kk) {
-          pv_step(i, kk, first);
-          if (with_s) s_step(i + 2, kk);
+        if (with_s) {
+          if (first) batch(i, std::true_type{}, std::true_type{});
+          else batch(i, std::false_type{}, std::true_type{});
+        } else {
+          if (first) batch(i, std::true_type{}, std::false_type{});
+          else batch(i, std::false_type{}, std::false_type{});
         }
         if (with_s) s_done(i + 2);
         umma_commit(empty_v(i % kStages));
@@ -364,65 +386,66 @@ score_pv_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
         ++seg;
       }
       const int buf = i & 1;
-      const bool key_ok = tile * kTileKeys + ct < a.n_cand;
+      const int key = tile * kTileKeys + ct;
+      const bool key_ok = key < a.n_cand;
+      const bool tile_full = (tile + 1) * kTileKeys <= a.n_cand;   // no key of the tile needs masking
       ok = mbar_wait(ctl, s_full(buf), (i >> 1) & 1, 48u | ((unsigned)i << 8));
       if (ok) ok = mbar_wait(ctl, p_empty(buf), ((i >> 1) & 1) ^ 1, 49u | ((unsigned)i << 8));
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       tc_fence_after_sync();
       const uint32_t p_addr = p_base + (uint32_t)(buf * kTileBytes) + p_line;
-      const float* nl = nlse2_s + grp * 64;
+      const float4* nl = reinterpret_cast<const float4*>(nlse2_s + grp * 64);
       float acc0 = 0.f, acc1 = 0.f, acc2 = 0.f, acc3 = 0.f;
       // probabilities of 32 row columns: votes, row sums, bf16 pairs into this key's line of P^T
-      auto soft32 = [&](const uint32_t (&sv)[32], auto c0_tag) {
+      auto soft32 = [&](const uint32_t (&sv)[32], auto c0_tag, auto masked_tag) {
         constexpr int c0 = decltype(c0_tag)::value;
+        constexpr bool masked = decltype(masked_tag)::value;
+        float pr[32];
+#pragma unroll
+        for (int e = 0; e < 32; e += 4) {
+          const float4 n4 = nl[(c0 + e) >> 2];
+          pr[e + 0] = ex2_approx(fmaf(__uint_as_float(sv[e + 0]), a.scale2, n4.x));
+          pr[e + 1] = ex2_approx(fmaf(__uint_as_float(sv[e + 1]), a.scale2, n4.y));
+          pr[e + 2] = ex2_approx(fmaf(__uint_as_float(sv[e + 2]), a.scale2, n4.z));
+          pr[e + 3] = ex2_approx(fmaf(__uint_as_float(sv[e + 3]), a.scale2, n4.w));
+        }
+        if (masked) {
+#pragma unroll
+          for (int e = 0; e < 32; ++e) pr[e] = key_ok ? pr[e] : 0.f;
+        }
+#pragma unroll
+        for (int e = 0; e < 32; e += 4) {
+          acc0 += pr[e + 0]; acc1 += pr[e + 1]; acc2 += pr[e + 2]; acc3 += pr[e + 3];
+          lrow[c0 + e + 0] += pr[e + 0]; lrow[c0 + e + 1] += pr[e + 1];
+          lrow[c0 + e + 2] += pr[e + 2]; lrow[c0 + e + 3] += pr[e + 3];
+        }
 #pragma unroll
         for (int e = 0; e < 32; e += 8) {
-          const float4 n0 = *reinterpret_cast<const float4*>(nl + c0 + e);
-          const float4 n1 = *reinterpret_cast<const float4*>(nl + c0 + e + 4);
-          float p0 = ex2_approx(fmaf(__uint_as_float(sv[e + 0]), a.scale2, n0.x));
-          float p1 = ex2_approx(fmaf(__uint_as_float(sv[e + 1]), a.scale2, n0.y));
-          float p2 = ex2_approx(fmaf(__uint_as_float(sv[e + 2]), a.scale2, n0.z));
-          float p3 = ex2_approx(fmaf(__uint_as_float(sv[e + 3]), a.scale2, n0.w));
-          float p4 = ex2_approx(fmaf(__uint_as_float(sv[e + 4]), a.scale2, n1.x));
-          float p5 = ex2_approx(fmaf(__uint_as_float(sv[e + 5]), a.scale2, n1.y));
-          float p6 = ex2_approx(fmaf(__uint_as_float(sv[e + 6]), a.scale2, n1.z));
-          float p7 = ex2_approx(fmaf(__uint_as_float(sv[e + 7]), a.scale2, n1.w));
-          if (!key_ok) p0 = p1 = p2 = p3 = p4 = p5 = p6 = p7 = 0.f;
-          acc0 += p0 + p4; acc1 += p1 + p5; acc2 += p2 + p6; acc3 += p3 + p7;
-          lrow[c0 + e + 0] += p0; lrow[c0 + e + 1] += p1; lrow[c0 + e + 2] += p2; lrow[c0 + e + 3] += p3;
-          lrow[c0 + e + 4] += p4; lrow[c0 + e + 5] += p5; lrow[c0 + e + 6] += p6; lrow[c0 + e + 7] += p7;
           const uint32_t chunk = (uint32_t)((c0 + e) >> 3);
-          st_shared_v4(p_addr + ((chunk ^ p_xor) << 4), pack_bf16(p0, p1), pack_bf16(p2, p3), pack_bf16(p4, p5),
-                       pack_bf16(p6, p7));
+          st_shared_v4(p_addr + ((chunk ^ p_xor) << 4), pack_bf16(pr[e + 0], pr[e + 1]), pack_bf16(pr[e + 2], pr[e + 3]),
+                       pack_bf16(pr[e + 4], pr[e + 5]), pack_bf16(pr[e + 6], pr[e + 7]));
         }
       };
       uint32_t ra[32], rb[32];
       tmem_ld32_issue(s_addr + (uint32_t)(buf * 128), ra);
       tmem_ld_wait(ra);
       tmem_ld32_issue(s_addr + (uint32_t)(buf * 128 + 32), rb);
-      soft32(ra, std::integral_constant<int, 0>{});
-      tmem_ld_wait(rb);
-      soft32(rb, std::integral_constant<int, 32>{});
+      if (tile_full) {
+        soft32(ra, std::integral_constant<int, 0>{}, std::false_type{});
+        tmem_ld_wait(rb);
+        soft32(rb, std::integral_constant<int, 32>{}, std::false_type{});
+      } else {
+        soft32(ra, std::integral_constant<int, 0>{}, std::true_type{});
+        tmem_ld_wait(rb);
+        soft32(rb, std::integral_constant<int, 32>{}, std::true_type{});
+      }
       fence_proxy_async_smem();   // the P^T stores must be visible to the MMA's shared-memory reads
       tc_fence_before_sync();
       mbar_arrive(p_full(buf));
-      // the two halves of the key's vote meet in shared memory; group 0 stores the sum
-      const float part = (acc0 + acc1) + (acc2 + acc3);
-      if (grp == 1) {
-        ok = mbar_wait(ctl, vx_empty(buf), ((i >> 1) & 1) ^ 1, 52u | ((unsigned)i << 8));
-        ok = __all_sync(0xffffffffu, ok);
-        if (!ok) break;
-        vx[buf * 128 + ct] = part;
-        mbar_arrive(vx_full(buf));
-      } else {
-        ok = mbar_wait(ctl, vx_full(buf), (i >> 1) & 1, 53u | ((unsigned)i << 8));
-        ok = __all_sync(0xffffffffu, ok);
-        if (!ok) break;
-        const float v = part + vx[buf * 128 + ct];
-        mbar_arrive(vx_empty(buf));
-        if (key_ok) a.vote[(size_t)cb * a.vote_stride + (size_t)unit * a.n_cand + tile * kTileKeys + ct] = v;
-      }
+      // each group stores the partial vote of its half of the rows; sum_vote_parts_kernel adds them
+      if (key_ok && a.vote)
+        a.vote[(size_t)(cb * kGroups + grp) * a.vote_stride + (size_t)unit * a.n_cand + key] = (acc0 + acc1) + (acc2 + acc3);
     }
     if (ok && cur_unit >= 0) store_partial(cur_unit);
   }
@@ -436,7 +459,7 @@ score_pv_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
   if (warp == kMmaWarp) tmem_dealloc(tmem_base, kTmemCols);
 }
 
-// vote[i] = sum of the row blocks' partial votes, in block order.
+// vote[i] = sum of the partial votes (two per row block), in order.
 __global__ void sum_vote_parts_kernel(float* __restrict__ vote, size_t n, int parts) {
   const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= n) return;
@@ -445,58 +468,94 @@ __global__ void sum_vote_parts_kernel(float* __restrict__ vote, size_t n, int pa
   vote[i] = s;
 }
 
+// The subtraction loses accuracy when the evicted keys carry little of a row's softmax mass: the
+// fp32 accumulation error of the sum over all candidates (about 1e-5 of it, measured) is divided by
+// that share.  Rows below this share have their unit listed for the masked pass over the evicted
+// keys themselves (calib_tc_kernel in work-list mode), which rewrites the unit's rows.
+constexpr float kMinEvictedShare = 1.0f / 64.0f;
+
 // One warp per (batch, query head, window row): the sums over all candidates (score_pv_kernel)
-// minus the sums over the selected ones (calib_tc_kernel on the compacted rows), each added up over
+// minus the sums over the selected ones (the same kernel on the compacted rows), each added up over
 // its CTAs' partials in a fixed order; then O_c = O / l, LSE_c = lse + log l, C_q = the query.
+// redo = {block counter, n_work, unit_flag[units], unit_pos[units], work_list[units]}, zeroed by the
+// caller: rows that need the masked pass flag their unit, and the block that finishes last turns
+// the flags into the ascending list of those units.
 __global__ void __launch_bounds__(128)
 calib_combine_kernel(const __nv_bfloat16* __restrict__ Q_obs, const float* __restrict__ row_lse,
                      const float* __restrict__ o_all, const float* __restrict__ l_all, int n_tiles_all,
                      int tpc_all, int slots_all, const float* __restrict__ o_sel, const float* __restrict__ l_sel,
                      int n_tiles_sel, int tpc_sel, int slots_sel, float* __restrict__ O_c,
                      float* __restrict__ LSE_c, __nv_bfloat16* __restrict__ C_q, int B, int Hq, int G, int W, int gpb,
-                     int n_cblocks) {
+                     int n_cblocks, int* __restrict__ redo) {
+  __shared__ bool is_last;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int row = blockIdx.x * 4 + warp;  // (b, hq, c), n_cal = W
-  if (row >= B * Hq * W) return;
-  const int c = row % W, bhq = row / W;
-  const int b = bhq / Hq, hq = bhq % Hq;
-  const int Hkv = Hq / G, h = hq / G, g = hq % G;
-  const int unit = b * Hkv + h, cb = g / gpb, r = (g % gpb) * W + c;
-  const int vu = unit * n_cblocks + cb;
-  float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-  float l = 0.f;
-  {
-    const int first = (unit * n_tiles_all) / tpc_all, last = ((unit + 1) * n_tiles_all - 1) / tpc_all;
-    const size_t part0 = (size_t)vu * slots_all;
-    for (int s = 0; s <= last - first; ++s) {
-      const float4 v = *reinterpret_cast<const float4*>(o_all + ((part0 + s) * 128 + r) * kD + 4 * lane);
-      acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
-      for (int w = 0; w < 4; ++w) l += l_all[((part0 + s) * 8 + (r >> 6) * 4 + w) * 64 + (r & 63)];
+  const int units = B * (Hq / G);
+  int* const unit_flag = redo + 2;
+  if (row < B * Hq * W) {
+    const int c = row % W, bhq = row / W;
+    const int b = bhq / Hq, hq = bhq % Hq;
+    const int Hkv = Hq / G, h = hq / G, g = hq % G;
+    const int unit = b * Hkv + h, cb = g / gpb, r = (g % gpb) * W + c;
+    const int vu = unit * n_cblocks + cb;
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    float l = 0.f;
+    {
+      const int first = (unit * n_tiles_all) / tpc_all, last = ((unit + 1) * n_tiles_all - 1) / tpc_all;
+      const size_t part0 = (size_t)vu * slots_all;
+      for (int s = 0; s <= last - first; ++s) {
+        const float4 v = *reinterpret_cast<const float4*>(o_all + ((part0 + s) * 128 + r) * kD + 4 * lane);
+        acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
+        for (int w = 0; w < 4; ++w) l += l_all[((part0 + s) * 8 + (r >> 6) * 4 + w) * 64 + (r & 63)];
+      }
     }
-  }
-  float4 sel = make_float4(0.f, 0.f, 0.f, 0.f);
-  float ls = 0.f;
-  {
-    const int first = (unit * n_tiles_sel) / tpc_sel, last = ((unit + 1) * n_tiles_sel - 1) / tpc_sel;
-    const size_t part0 = (size_t)vu * slots_sel;
-    for (int s = 0; s <= last - first; ++s) {
-      const float4 v = *reinterpret_cast<const float4*>(o_sel + ((part0 + s) * 128 + r) * kD + 4 * lane);
-      sel.x += v.x; sel.y += v.y; sel.z += v.z; sel.w += v.w;
-      for (int grp = 0; grp < 2; ++grp) ls += l_sel[((part0 + s) * 2 + grp) * 128 + r];
+    float4 sel = make_float4(0.f, 0.f, 0.f, 0.f);
+    float ls = 0.f;
+    {
+      const int first = (unit * n_tiles_sel) / tpc_sel, last = ((unit + 1) * n_tiles_sel - 1) / tpc_sel;
+      const size_t part0 = (size_t)vu * slots_sel;
+      for (int s = 0; s <= last - first; ++s) {
+        const float4 v = *reinterpret_cast<const float4*>(o_sel + ((part0 + s) * 128 + r) * kD + 4 * lane);
+        sel.x += v.x; sel.y += v.y; sel.z += v.z; sel.w += v.w;
+        for (int w = 0; w < 4; ++w) ls += l_sel[((part0 + s) * 8 + (r >> 6) * 4 + w) * 64 + (r & 63)];
+      }
     }
+    const float l_cand = l;
+    l -= ls;
+    if (lane == 0 && !(l >= kMinEvictedShare * l_cand)) atomicOr(&unit_flag[unit], 1);
+    float4 out = make_float4(0.f, 0.f, 0.f, 0.f);
+    float lse = -INFINITY;
+    if (l > 0.f) {
+      const float inv = 1.f / l;
+      out = make_float4((acc.x - sel.x) * inv, (acc.y - sel.y) * inv, (acc.z - sel.z) * inv, (acc.w - sel.w) * inv);
+      lse = row_lse[(size_t)bhq * W + c] + logf(l);
+    }
+    reinterpret_cast<float4*>(O_c + (size_t)row * kD)[lane] = out;
+    if (lane == 0) LSE_c[row] = lse;
+    reinterpret_cast<uint2*>(C_q + (size_t)row * kD)[lane] =
+        reinterpret_cast<const uint2*>(Q_obs + (size_t)row * kD)[lane];
   }
-  l -= ls;
-  float4 out = make_float4(0.f, 0.f, 0.f, 0.f);
-  float lse = -INFINITY;
-  if (l > 0.f) {
-    const float inv = 1.f / l;
-    out = make_float4((acc.x - sel.x) * inv, (acc.y - sel.y) * inv, (acc.z - sel.z) * inv, (acc.w - sel.w) * inv);
-    lse = row_lse[(size_t)bhq * W + c] + logf(l);
+  // the last block to finish lists the flagged units (no block waits for another)
+  __threadfence();
+  __syncthreads();
+  if (threadIdx.x == 0) is_last = atomicAdd(reinterpret_cast<unsigned*>(redo), 1u) == gridDim.x - 1;
+  __syncthreads();
+  if (is_last && warp == 0) {
+    __threadfence();
+    int* const unit_pos = unit_flag + units;
+    int* const work_list = unit_pos + units;
+    int count = 0;
+    for (int base = 0; base < units; base += 32) {
+      const int u = base + lane;
+      const bool f = u < units && __ldcg(unit_flag + u) != 0;
+      const unsigned ball = __ballot_sync(0xffffffffu, f);
+      const int pos = count + __popc(ball & ((1u << lane) - 1u));
+      if (u < units) unit_pos[u] = f ? pos : -1;
+      if (f) work_list[pos] = u;
+      count += __popc(ball);
+    }
+    if (lane == 0) redo[1] = count;
   }
-  reinterpret_cast<float4*>(O_c + (size_t)row * kD)[lane] = out;
-  if (lane == 0) LSE_c[row] = lse;
-  reinterpret_cast<uint2*>(C_q + (size_t)row * kD)[lane] =
-      reinterpret_cast<const uint2*>(Q_obs + (size_t)row * kD)[lane];
 }
 
 }  // namespace
@@ -508,28 +567,33 @@ bool score_pv_supported(const CompressGeom& g) {
   return !g.keep_all && g.n_cal == g.W && g.W <= 128 && g.k_sel >= 1 && g.n_cand - g.k_sel > g.k_sel;
 }
 
-cudaError_t launch_score_pv(const CompressGeom& g, const CompressWs& ws, const void* Q_obs, const void* K,
-                            const void* V, const float* row_lse, char* wsp, cudaStream_t st) {
+// One pass of score_pv_kernel over rows [0, n_keys) of every unit of K / V (a unit's rows are
+// `unit_rows` apart): the partial (O, l) sums into o_part / l_part and, when `vote` is not null, the
+// votes of those keys.
+static cudaError_t launch_pv_pass(const CompressGeom& g, const void* Q_obs, const void* K, const void* V, int n_keys,
+                                  size_t unit_rows, const float* row_lse, float* vote, float* o_part, float* l_part,
+                                  unsigned* status, cudaStream_t st) {
   PvArgs a{};
-  a.Hq = g.Hq; a.G = g.G; a.W = g.W; a.L = g.L; a.n_cand = g.n_cand;
+  a.Hq = g.Hq; a.G = g.G; a.W = g.W; a.L = g.L; a.n_cand = n_keys;
   size_t parts;
-  calib_tc_plan(g, g.n_cand, &a.gpb, &a.n_cblocks, &a.tiles_per_cta, &a.max_slots, &parts);
-  a.n_tiles = (g.n_cand + kTileKeys - 1) / kTileKeys;
+  calib_tc_plan(g, n_keys, &a.gpb, &a.n_cblocks, &a.tiles_per_cta, &a.max_slots, &parts);
+  a.n_tiles = (n_keys + kTileKeys - 1) / kTileKeys;
   a.total_tiles = g.units * a.n_tiles;
   a.scale2 = g.scale2;
   a.row_lse = row_lse;
-  a.vote = (float*)(wsp + ws.vote);
-  a.vote_stride = (size_t)g.units * g.n_cand;
-  a.o_part = (float*)(wsp + ws.calib_o);
-  a.l_part = (float*)(wsp + ws.pv_l);
-  a.status = (unsigned*)(wsp + ws.status);
+  a.vote = vote;
+  a.vote_stride = (size_t)g.units * n_keys;
+  a.o_part = o_part;
+  a.l_part = l_part;
+  a.status = status;
   CUtensorMap qm, km, vm;
   // window rows: [head dim][j < W][g < G][unit]
   const uint64_t qd[3] = {(uint64_t)g.W, (uint64_t)g.G, (uint64_t)g.units};
   const uint64_t qs[3] = {256, (uint64_t)g.W * 256, (uint64_t)g.G * g.W * 256};
   const uint32_t qb[3] = {(uint32_t)g.W, (uint32_t)a.gpb, 1};
   if (!make_tensor_map_bf16(&qm, Q_obs, 4, qd, qs, qb)) return cudaErrorInvalidValue;
-  const uint64_t kd[2] = {(uint64_t)g.L, (uint64_t)g.units}, ks[2] = {256, (uint64_t)g.L * 256};
+  // rows at or beyond n_keys are never used (their probabilities are masked), so the maps end there
+  const uint64_t kd[2] = {(uint64_t)n_keys, (uint64_t)g.units}, ks[2] = {256, (uint64_t)unit_rows * 256};
   const uint32_t kb[2] = {(uint32_t)kTileKeys, 1};
   if (!make_tensor_map_bf16(&km, K, 3, kd, ks, kb) || !make_tensor_map_bf16(&vm, V, 3, kd, ks, kb))
     return cudaErrorInvalidValue;
@@ -545,12 +609,28 @@ cudaError_t launch_score_pv(const CompressGeom& g, const CompressWs& ws, const v
   const int grid = (a.total_tiles + a.tiles_per_cta - 1) / a.tiles_per_cta * a.n_cblocks;
   score_pv_kernel<<<grid, kThreads, kSmemBytes, st>>>(qm, km, vm, a);
   count_launch(1);
-  if (a.n_cblocks > 1) {
+  if (vote) {
     const size_t n = a.vote_stride;
-    sum_vote_parts_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(a.vote, n, a.n_cblocks);
+    sum_vote_parts_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(vote, n, a.n_cblocks * kGroups);
     count_launch(1);
   }
   return cudaGetLastError();
+}
+
+// Votes of every candidate key (into ws.vote) and the sums over all candidates.
+cudaError_t launch_score_pv(const CompressGeom& g, const CompressWs& ws, const void* Q_obs, const void* K,
+                            const void* V, const float* row_lse, char* wsp, cudaStream_t st) {
+  return launch_pv_pass(g, Q_obs, K, V, g.n_cand, (size_t)g.L, row_lse, (float*)(wsp + ws.vote),
+                        (float*)(wsp + ws.calib_o), (float*)(wsp + ws.pv_l), (unsigned*)(wsp + ws.status), st);
+}
+
+// The sums over the selected rows, rows [0, k_sel) of every unit of the kept cache: the same kernel,
+// hence the same logits and the same bf16 probabilities as in the pass over all candidates.
+cudaError_t launch_score_pv_selected(const CompressGeom& g, const CompressWs& ws, const void* Q_obs,
+                                     const void* K_kept, const void* V_kept, const float* row_lse, char* wsp,
+                                     cudaStream_t st) {
+  return launch_pv_pass(g, Q_obs, K_kept, V_kept, g.k_sel, (size_t)g.cap, row_lse, nullptr, (float*)(wsp + ws.sel_o),
+                        (float*)(wsp + ws.sel_l), (unsigned*)(wsp + ws.status), st);
 }
 
 cudaError_t launch_calib_combine(const CompressGeom& g, const CompressWs& ws, const void* Q_obs,
@@ -565,7 +645,7 @@ cudaError_t launch_calib_combine(const CompressGeom& g, const CompressWs& ws, co
       (const __nv_bfloat16*)Q_obs, row_lse, (const float*)(wsp + ws.calib_o), (const float*)(wsp + ws.pv_l),
       (g.n_cand + kTileKeys - 1) / kTileKeys, tpc_all, slots_all, (const float*)(wsp + ws.sel_o),
       (const float*)(wsp + ws.sel_l), (g.k_sel + kTileKeys - 1) / kTileKeys, tpc_sel, slots_sel, O_c, LSE_c,
-      (__nv_bfloat16*)C_q, g.B, g.Hq, g.G, g.W, gpb, n_cblocks);
+      (__nv_bfloat16*)C_q, g.B, g.Hq, g.G, g.W, gpb, n_cblocks, (int*)(wsp + ws.redo));
   count_launch(1);
   return cudaGetLastError();
 }

@@ -174,6 +174,10 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
     // ------------------------------------------------------------ MMA issuer
     if (lane == 0) {
       const uint32_t idesc = umma_idesc(128, kVotes ? a.block_rows : 256, false, false);
+      // Descriptors are built once per buffer; a k-step adds a constant to the address field (the
+      // issuing thread's own instructions between two MMAs are what limits the issue rate).
+      const uint64_t dq0 = smem_desc_sw128(q_base, 16u, 1024u);
+      const uint64_t dk0 = smem_desc_sw128(k_base, 16u, 1024u);
       int cur_vu = -1, seg = 0, j = 0, vu = vu_begin, tile = tile_begin;
       for (int i = 0; i < nt; ++i, ++tile) {
         if (tile == a.n_tiles) { tile = 0; ++vu; }
@@ -185,6 +189,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
         const int s = i % a.stages;
         if (!mbar_wait(&ctl, full_k(s), (i / a.stages) & 1, (kVotes ? 33u : 13u) | ((unsigned)i << 8))) break;
         bool ok = true;
+        const uint64_t kd = desc_advance(dk0, (uint32_t)s * STAGE_BYTES);
         for (int blk = 0; blk < a.n_blocks; ++blk, ++j) {
           const int buf = j & 1;
           if (!mbar_wait(&ctl, t_empty(buf), ((j >> 1) & 1) ^ 1, (kVotes ? 34u : 14u) | ((unsigned)j << 8))) {
@@ -193,13 +198,16 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
           }
           tc_fence_after_sync();
           const uint32_t d = tmem_base + (uint32_t)(buf * kBufCols);
-          const uint32_t kt = k_base + (uint32_t)s * STAGE_BYTES, qt = q_base + (uint32_t)blk * q_blk_bytes;
+          const uint64_t qd = desc_advance(dq0, (uint32_t)blk * q_blk_bytes);
+          // the second halves (k-steps 4..7) start half a tile further on
+          const uint64_t kd2 = desc_advance(kd, STAGE_BYTES / 2), qd2 = desc_advance(qd, q_half_bytes);
+          umma_ss_imm<0>(d, kVotes ? kd : qd, kVotes ? qd : kd, idesc);
 #pragma unroll
-          for (int kk = 0; kk < kD / 16; ++kk) {
-            const uint64_t kd = kmajor_desc(kt, STAGE_BYTES / 2, kk);
-            const uint64_t qd = kmajor_desc(qt, q_half_bytes, kk);
-            umma_ss(d, kVotes ? kd : qd, kVotes ? qd : kd, idesc, kk > 0 ? 1u : 0u);
-          }
+          for (int kk = 1; kk < 4; ++kk)
+            umma_ss_imm<1>(d, desc_advance(kVotes ? kd : qd, kk * 32u), desc_advance(kVotes ? qd : kd, kk * 32u), idesc);
+#pragma unroll
+          for (int kk = 0; kk < 4; ++kk)
+            umma_ss_imm<1>(d, desc_advance(kVotes ? kd2 : qd2, kk * 32u), desc_advance(kVotes ? qd2 : kd2, kk * 32u), idesc);
           umma_commit(t_full(buf));
         }
         if (!ok) break;

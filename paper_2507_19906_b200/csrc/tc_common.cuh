@@ -236,6 +236,44 @@ __device__ __forceinline__ void umma_commit(uint32_t bar) {
                : "memory");
 }
 
+// ---- lean issue: the MMA-issuing thread is ONE thread, whose dependent scalar instructions cost
+// several cycles each, so every instruction between two MMAs counts (measured: an issue loop that
+// rebuilds its descriptors from addresses runs at 100-150 cycles per 128x128x16 MMA whatever the
+// operands; with the descriptors prepared and the accumulate flag an immediate the same MMAs run
+// at 64 cycles, the tensor pipe's own rate, even as one dependent chain).  So descriptors are built
+// once per buffer and advanced by adding a compile-time byte offset to their address field.
+__device__ __forceinline__ uint64_t desc_advance(uint64_t desc, uint32_t bytes) {
+  uint2 v = *reinterpret_cast<uint2*>(&desc);
+  v.x += bytes >> 4;   // the address field holds bytes / 16 in the low bits; tiles never wrap it
+  return *reinterpret_cast<uint64_t*>(&v);
+}
+// Byte offset of MMA k-step kk inside a K-major tile whose 64-element halves are half_bytes apart.
+__host__ __device__ constexpr uint32_t kmajor_step_bytes(uint32_t half_bytes, int kk) {
+  return (uint32_t)(kk >> 2) * half_bytes + (uint32_t)(kk & 3) * 32u;
+}
+template <int ACC>
+__device__ __forceinline__ void umma_ss_imm(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc) {
+  asm volatile(
+      "{\n"
+      ".reg .pred p;\n"
+      "setp.ne.b32 p, %4, 0;\n"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n"
+      "}\n"
+      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "n"(ACC)
+      : "memory");
+}
+template <int ACC>
+__device__ __forceinline__ void umma_ts_imm(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc) {
+  asm volatile(
+      "{\n"
+      ".reg .pred p;\n"
+      "setp.ne.b32 p, %4, 0;\n"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n"
+      "}\n"
+      ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "n"(ACC)
+      : "memory");
+}
+
 constexpr int kHalfCols = 64;          // head-dim elements per shared-memory half tile
 constexpr int kLineBytes = 128;        // one half-tile line
 constexpr int kTileKeys = 128;         // keys per streamed K/V tile
