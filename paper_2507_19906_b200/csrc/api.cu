@@ -72,17 +72,8 @@ CompressWs make_ws(const CompressGeom& g) {
   CompressWs w{};
   size_t off = 0;
   const size_t n_cand = (size_t)(g.L > g.W ? g.L - g.W : 0);
-  // The vote array leads a run of per-row-block partial votes (one block's worth each, contiguous):
-  // the two-block vote pass uses vote and vote2, the one-pass kernel two per row block.
-  size_t vote_parts = g.G * g.W > 256 ? 2 : 1;
-  if (score_tc_supported(g) && score_pv_supported(g)) {
-    int gpb, n_cblocks, tpc, max_slots;
-    size_t parts;
-    calib_tc_plan(g, g.n_cand, &gpb, &n_cblocks, &tpc, &max_slots, &parts);
-    if ((size_t)n_cblocks * 2 > vote_parts) vote_parts = (size_t)n_cblocks * 2;  // one per half block
-  }
-  w.vote = off;    off += (size_t)g.units * n_cand * 4;
-  w.vote2 = off;   off = align_up(off + (vote_parts - 1) * (size_t)g.units * n_cand * 4, 256);
+  w.vote = off;    off = align_up(off + (size_t)g.units * n_cand * 4, 256);
+  w.vote2 = off;   off = align_up(off + (g.G * g.W > 256 ? (size_t)g.units * n_cand * 4 : 0), 256);
   w.pooled = off;  off = align_up(off + (size_t)g.units * n_cand * 4, 256);
   w.row_lse = off; off = align_up(off + (size_t)g.B * g.Hq * g.W * 4, 256);
   w.bitmap = off;  off = align_up(off + (size_t)g.units * g.bitmap_words * 4, 256);
@@ -90,29 +81,13 @@ CompressWs make_ws(const CompressGeom& g) {
   w.stat_slots = w.n_tiles > 320 ? w.n_tiles : 320;
   w.stat_part = off; off = align_up(off + (size_t)g.B * g.Hq * g.W * w.stat_slots * 8, 256);
   w.status = off;    off = align_up(off + 4, 256);
-  // (directly behind the status word, so that one memset clears both)
-  w.redo = off;      off = align_up(off + (size_t)(2 + 3 * g.units) * 4, 256);
   w.calib_o = w.calib_l = off;
   if (score_tc_supported(g) && calib_tc_supported(g)) {
     int gpb, n_cblocks, tpc, max_slots;
     size_t parts;
-    calib_tc_plan(g, g.n_cand, &gpb, &n_cblocks, &tpc, &max_slots, &parts);
-    if (score_pv_supported(g)) {   // the masked pass over listed units indexes its partials by CTA group
-      int groups, seg_max;
-      size_t list_parts;
-      calib_tc_list_plan(g, g.n_cand, &groups, &seg_max, &list_parts);
-      if (list_parts > parts) parts = list_parts;
-    }
+    calib_tc_plan(g, &gpb, &n_cblocks, &tpc, &max_slots, &parts);
     w.calib_o = off; off = align_up(off + parts * 128 * kD * 4, 256);
     w.calib_l = off; off = align_up(off + parts * 2 * 128 * 4, 256);
-    calib_tc_plan(g, g.n_cand, &gpb, &n_cblocks, &tpc, &max_slots, &parts);
-    w.pv_l = w.sel_o = w.sel_l = off;
-    if (score_pv_supported(g)) {
-      w.pv_l = off;  off = align_up(off + parts * 8 * 64 * 4, 256);
-      calib_tc_plan(g, g.k_sel, &gpb, &n_cblocks, &tpc, &max_slots, &parts);
-      w.sel_o = off; off = align_up(off + parts * 128 * kD * 4, 256);
-      w.sel_l = off; off = align_up(off + parts * 8 * 64 * 4, 256);
-    }
   }
   w.total = off;
   return w;
@@ -274,14 +249,11 @@ int calidrop_compress(const calidrop_params* p, const void* Q_obs, const void* K
 
   cudaStream_t st = (cudaStream_t)stream;
   char* wsp = (char*)workspace;
-  cudaError_t e = cudaMemsetAsync(wsp + ws.status, 0, ws.calib_o - ws.status, st);   // error word and the redo list
+  cudaError_t e = cudaMemsetAsync(wsp + ws.status, 0, 4, st);
   if (e != cudaSuccess) return cuda_fail(e);
   // The contractions run on the tensor cores whenever the tiles cover the shape; the scalar
   // kernels remain for the rest (more than 512 window rows per kv head, budget >= L).
   const bool tc_path = score_tc_supported(g) && !scalar_path_forced();
-  // One pass for the votes and the calibration sums when every window row calibrates; otherwise
-  // the votes alone, and the calibration as a masked pass after the selection.
-  const bool one_pass = tc_path && calib_tc_supported(g) && score_pv_supported(g);
   const float* row_lse = lse_obs;
   if (!g.keep_all) {
     if (!row_lse) {
@@ -289,9 +261,7 @@ int calidrop_compress(const calidrop_params* p, const void* Q_obs, const void* K
       if (e != cudaSuccess) return cuda_fail(e);
       row_lse = (const float*)(wsp + ws.row_lse);
     }
-    e = one_pass ? launch_score_pv(g, ws, Q_obs, K, V, row_lse, wsp, st)
-        : tc_path ? launch_votes_tc(g, ws, Q_obs, K, row_lse, wsp, st)
-                  : launch_votes(g, ws, Q_obs, K, row_lse, wsp, st);
+    e = tc_path ? launch_votes_tc(g, ws, Q_obs, K, row_lse, wsp, st) : launch_votes(g, ws, Q_obs, K, row_lse, wsp, st);
     if (e != cudaSuccess) return cuda_fail(e);
   }
   e = (select_cluster_supported(g) && !scalar_path_forced()) ? launch_pool_select_cluster(g, ws, wsp, kept_idx, st)
@@ -299,22 +269,9 @@ int calidrop_compress(const calidrop_params* p, const void* Q_obs, const void* K
   if (e != cudaSuccess) return cuda_fail(e);
   e = launch_gather(g, K, V, kept_idx, K_kept, V_kept, st);
   if (e != cudaSuccess) return cuda_fail(e);
-  if (one_pass) {
-    // the sums over the selected rows, which are rows [0, k_sel) of every unit of the kept cache
-    e = launch_score_pv_selected(g, ws, Q_obs, K_kept, V_kept, row_lse, wsp, st);
-    if (e != cudaSuccess) return cuda_fail(e);
-    e = launch_calib_combine(g, ws, Q_obs, row_lse, wsp, O_c, LSE_c, C_q, st);
-    if (e != cudaSuccess) return cuda_fail(e);
-    // rows whose evicted keys carry too little mass for the subtraction: their units, listed on the
-    // device by the combine, get the masked pass over the evicted keys themselves
-    const int* redo = (const int*)(wsp + ws.redo);
-    e = launch_calib_tc_listed(g, ws, Q_obs, K, V, row_lse, wsp, redo + 2 + 2 * g.units, redo + 2 + g.units, redo + 1,
-                               O_c, LSE_c, C_q, st);
-  } else {
-    e = (tc_path && calib_tc_supported(g))
-            ? launch_calib_tc(g, ws, Q_obs, K, V, row_lse, wsp, O_c, LSE_c, C_q, st)
-            : launch_calib_direct(g, ws, Q_obs, K, V, wsp, O_c, LSE_c, C_q, st);
-  }
+  e = (tc_path && calib_tc_supported(g))
+          ? launch_calib_tc(g, ws, Q_obs, K, V, row_lse, wsp, O_c, LSE_c, C_q, st)
+          : launch_calib_direct(g, ws, Q_obs, K, V, wsp, O_c, LSE_c, C_q, st);
   if (e != cudaSuccess) return cuda_fail(e);
   return CALIDROP_OK;
 }

@@ -32,9 +32,11 @@ namespace {
 using namespace tc;
 
 constexpr int kGroups = 2;
-constexpr int kProducerWarp = kGroups * 4;
-constexpr int kMmaWarp = kGroups * 4 + 1;
-constexpr int kThreads = kGroups * 128 + 64;
+constexpr int kProducerWarp = kGroups * 4;       // TMA: Q_c blocks and K tiles
+constexpr int kMmaWarp = kGroups * 4 + 1;        // allocates TMEM, issues the S MMAs
+constexpr int kPvWarp = kGroups * 4 + 2;         // issues the P.V MMAs
+constexpr int kVProducerWarp = kGroups * 4 + 3;  // TMA: V tiles
+constexpr int kThreads = kGroups * 128 + 128;
 constexpr int kTmemCols = 512;
 constexpr uint32_t kColO = 256, kColP = 384;
 constexpr int kStages = 3;                 // K ring and V ring alike
@@ -55,26 +57,13 @@ struct CalibArgs {
   float* o_part;           // [virtual unit][slot][128][128]
   float* l_part;           // [virtual unit][slot][group][128]
   unsigned* status;
-  // Work-list mode (null = every unit): the kernel runs over the units listed in work_list only,
-  // n_work of them (read on the device, so the grid is fixed while the work is not), shared out
-  // evenly over the CTA groups; partials are then indexed [CTA group][segment < seg_max][row block].
-  const int* work_list;
-  const int* n_work;
-  int units, seg_max;
 };
-
-// Tiles per CTA group when n_units units are shared out over `groups` groups.
-__host__ __device__ inline int tiles_per_group(int n_units, int n_tiles, int groups) {
-  const long long total = (long long)n_units * n_tiles;
-  const long long t = (total + groups - 1) / groups;
-  return t < 1 ? 1 : (int)t;
-}
 
 __global__ void __launch_bounds__(kThreads, 1)
 calib_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__ CUtensorMap k_map,
                 const __grid_constant__ CUtensorMap v_map, const CalibArgs a) {
   extern __shared__ unsigned char smem_raw[];
-  __shared__ __align__(8) unsigned long long bars[20];
+  __shared__ __align__(8) unsigned long long bars[24];
   __shared__ uint32_t tmem_slot;
   __shared__ Ctl ctl;
 
@@ -83,17 +72,10 @@ calib_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
   // range at the same pace, one calibration row block each, so that a K/V tile fetched for one
   // of them is still in L2 when the others ask for it and crosses the HBM interface once.
   const int cta = blockIdx.x / a.n_cblocks, cb = blockIdx.x % a.n_cblocks;
-  const bool listed = a.work_list != nullptr;
-  const int n_units = listed ? *a.n_work : a.units;
-  if (n_units <= 0) return;   // nothing listed: uniform over the grid, before anything is set up
-  const int total_tiles = n_units * a.n_tiles;
-  const int tiles_per_cta = listed ? tiles_per_group(n_units, a.n_tiles, gridDim.x / a.n_cblocks) : a.tiles_per_cta;
-  const int g_begin = cta * tiles_per_cta;
-  const int g_end = min(total_tiles, g_begin + tiles_per_cta);
+  const int g_begin = cta * a.tiles_per_cta;
+  const int g_end = min(a.total_tiles, g_begin + a.tiles_per_cta);
   const int nt = g_end - g_begin;
   const int Hkv = a.Hq / a.G;
-  // position in the (listed) unit space -> the unit itself
-  auto unit_of = [&](int pos) { return listed ? a.work_list[pos] : pos; };
 
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   const uint32_t q_base = smem_base;
@@ -109,6 +91,8 @@ calib_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
   auto empty_v = [&](int s) { return bar0 + 8u * (11 + s); };
   auto s_full = [&](int b) { return bar0 + 8u * (14 + b); };
   auto p_full = [&](int b) { return bar0 + 8u * (16 + b); };
+  auto s_free = [&](int b) { return bar0 + 8u * (20 + b); };    // S buffer b has been read into registers
+  auto p_empty = [&](int b) { return bar0 + 8u * (22 + b); };   // the P.V that read P buffer b has completed
 
   if (tid == 0) {
     ctl.abort = 0;
@@ -121,7 +105,10 @@ calib_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
       mbar_init(full_k(s), 1); mbar_init(empty_k(s), 1);
       mbar_init(full_v(s), 1); mbar_init(empty_v(s), 1);
     }
-    for (int b = 0; b < 2; ++b) { mbar_init(s_full(b), 1); mbar_init(p_full(b), 128); }
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(s_full(b), 1); mbar_init(p_full(b), 128);
+      mbar_init(s_free(b), 128); mbar_init(p_empty(b), 1);
+    }
     fence_mbar_init();
   }
   if (warp == kMmaWarp) {
@@ -145,11 +132,12 @@ calib_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
   auto seg_last = [&](int i, int tile) { return i == nt - 1 || tile == a.n_tiles - 1; };
 
   if (warp == kProducerWarp) {
-    // ------------------------------------------------------------ TMA producer
+    // ------------------------------------------------------------ TMA producer of Q_c and K
+    // (K and V have a producer each: a K slot frees when its S is done, a V slot only when its P.V
+    // is, and one thread serving both in turn would hold every K load back behind a V slot)
     if (lane == 0) {
       tma_prefetch_desc(&q_map);
       tma_prefetch_desc(&k_map);
-      tma_prefetch_desc(&v_map);
       int seg = 0, vu = vu_begin, tile = tile_begin, unit = unit_begin;
       for (int i = 0; i < nt; ++i, ++tile) {
         if (tile == a.n_tiles) { tile = 0; ++unit; vu += a.n_cblocks; }
@@ -159,112 +147,123 @@ calib_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
           const int g0 = (vu - unit * a.n_cblocks) * a.gpb;
           mbar_arrive_expect_tx(q_full, 2u * (uint32_t)(a.gpb * a.n_cal) * kLineBytes);
           for (int half = 0; half < 2; ++half)
-            tma_load_4d(q_base + half * (kTileBytes / 2), &q_map, q_full, half * kHalfCols, 0, g0, unit_of(unit));
+            tma_load_4d(q_base + half * (kTileBytes / 2), &q_map, q_full, half * kHalfCols, 0, g0, unit);
           ++seg;
         }
         const int s = i % kStages;
-        const uint32_t ph = ((i / kStages) & 1) ^ 1;
-        if (!mbar_wait(&ctl, empty_k(s), ph, 21u | ((unsigned)i << 8))) break;
+        if (!mbar_wait(&ctl, empty_k(s), ((i / kStages) & 1) ^ 1, 21u | ((unsigned)i << 8))) break;
         mbar_arrive_expect_tx(full_k(s), kTileBytes);
         for (int half = 0; half < 2; ++half)
           tma_load_3d(k_base + s * kTileBytes + half * (kTileBytes / 2), &k_map, full_k(s), half * kHalfCols,
-                      tile * kTileKeys, unit_of(unit));
-        if (!mbar_wait(&ctl, empty_v(s), ph, 22u | ((unsigned)i << 8))) break;
+                      tile * kTileKeys, unit);
+      }
+    }
+  } else if (warp == kVProducerWarp) {
+    // ------------------------------------------------------------ TMA producer of V
+    if (lane == 0) {
+      tma_prefetch_desc(&v_map);
+      int tile = tile_begin, unit = unit_begin;
+      for (int i = 0; i < nt; ++i, ++tile) {
+        if (tile == a.n_tiles) { tile = 0; ++unit; }
+        const int s = i % kStages;
+        if (!mbar_wait(&ctl, empty_v(s), ((i / kStages) & 1) ^ 1, 22u | ((unsigned)i << 8))) break;
         mbar_arrive_expect_tx(full_v(s), kTileBytes);
         for (int half = 0; half < 2; ++half)
           tma_load_3d(v_base + s * kTileBytes + half * (kTileBytes / 2), &v_map, full_v(s), half * kHalfCols,
-                      tile * kTileKeys, unit_of(unit));
+                      tile * kTileKeys, unit);
       }
     }
   } else if (warp == kMmaWarp) {
-    // ------------------------------------------------------------ MMA issuer
-    // At the start of a virtual unit S(i) and S(i+1) are issued (k-steps interleaved); from then on
-    // P.V(i) is issued together with S(i+2), again interleaved, as soon as P(i) is complete (which
-    // also means S(i) has been read out of its buffer).  S never runs ahead across a change of
-    // virtual unit: its Q_c block is only loaded once the current unit's MMAs are done.
+    // ------------------------------------------------------------ issuer of the S MMAs
+    // The MMAs have two issuing threads, one for S = Q_c K^T and one for O += P V.  One thread for
+    // both was the bottleneck of this kernel: besides its sixteen MMAs a tile it has three waits and
+    // five commits to go through, each of them some hundred cycles of dependent scalar instructions
+    // for a single thread (measured: 2900 cycles a tile against 1024 of tensor-pipe time, the softmax
+    // groups waiting for S half of the time).  The two chains touch different accumulators; what
+    // orders them is the barriers, not the issue order.
+    // S(t) goes into buffer t % 2 as soon as S(t-2) has been read out of it (s_free), which is well
+    // before P(t-2) is complete.  S never runs ahead across a change of virtual unit: its Q_c block
+    // is only loaded once the current unit's S MMAs are done.
     if (lane == 0) {
       const uint32_t idesc = umma_idesc(128, 128, false, false);     // S: A = Q_c, B = K tile, K-major
-      const uint32_t idesc_o = umma_idesc(128, 128, false, true);    // O: A = P (TMEM), B = V tile, MN-major
-      const uint32_t tmem_o = tmem_base + kColO;
-      int seg = 0;
-      bool ok = true;
       // Descriptors are built once per buffer and a k-step adds a constant to the address field: the
       // issuing thread's own instructions between two MMAs are what limits the issue rate.
       const uint64_t dq = smem_desc_sw128(q_base, 16u, 1024u);
       const uint64_t dk0 = smem_desc_sw128(k_base, 16u, 1024u);
-      // V tile with the keys as K, i.e. MN-major: blocks of 64 head-dim elements are half a tile
-      // apart, groups of 8 keys 1024 bytes apart
-      const uint64_t dv0 = smem_desc_sw128(v_base, kTileBytes / 2, 1024u);
-      const uint32_t tmem_p = tmem_base + kColP;
-      // S(i): eight k-steps
-      auto s_steps = [&](int i) {
-        const uint32_t d = tmem_base + (uint32_t)((i & 1) * 128);
-        const uint64_t kd = desc_advance(dk0, (uint32_t)(i % kStages) * kTileBytes);
+      int seg = 0;
+      bool ok = true;
+      // S(t): wait for its buffer and its K tile, eight k-steps, then tell the softmax group and
+      // the producer
+      auto issue_s = [&](int t) -> bool {
+        if (t >= 2 && !mbar_wait(&ctl, s_free(t & 1), ((t - 2) >> 1) & 1, 29u | ((unsigned)t << 8))) return false;
+        if (!mbar_wait(&ctl, full_k(t % kStages), (t / kStages) & 1, 24u | ((unsigned)t << 8))) return false;
+        tc_fence_after_sync();
+        const uint32_t d = tmem_base + (uint32_t)((t & 1) * 128);
+        const uint64_t kd = desc_advance(dk0, (uint32_t)(t % kStages) * kTileBytes);
         umma_ss_imm<0>(d, dq, kd, idesc);
 #pragma unroll
         for (int kk = 1; kk < kD / 16; ++kk)
           umma_ss_imm<1>(d, desc_advance(dq, kmajor_step_bytes(kTileBytes / 2, kk)),
                          desc_advance(kd, kmajor_step_bytes(kTileBytes / 2, kk)), idesc);
+        umma_commit(s_full(t & 1));
+        umma_commit(empty_k(t % kStages));
+        return true;
       };
-      // P.V(i) (A: P in tensor memory, 16 keys = 8 columns per step), with or without S(i + 2) interleaved
-      auto batch = [&](int i, auto first_tag, auto with_s_tag) {
-        constexpr bool kFirst = decltype(first_tag)::value, kWithS = decltype(with_s_tag)::value;
-        const uint64_t vd = desc_advance(dv0, (uint32_t)(i % kStages) * kTileBytes);
-        const uint32_t pa = tmem_p + (uint32_t)((i & 1) * 64);
-        const uint32_t d = tmem_base + (uint32_t)((i & 1) * 128);
-        const uint64_t kd = desc_advance(dk0, (uint32_t)((i + 2) % kStages) * kTileBytes);
-#pragma unroll
-        for (int kk = 0; kk < kTileKeys / 16; ++kk) {
-          if (kFirst && kk == 0) umma_ts_imm<0>(tmem_o, pa, vd, idesc_o);
-          else umma_ts_imm<1>(tmem_o, pa + (uint32_t)(kk * 8), desc_advance(vd, (uint32_t)kk * 16u * kLineBytes), idesc_o);
-          if (kWithS) {
-            if (kk == 0) umma_ss_imm<0>(d, dq, kd, idesc);
-            else umma_ss_imm<1>(d, desc_advance(dq, kmajor_step_bytes(kTileBytes / 2, kk)),
-                                desc_advance(kd, kmajor_step_bytes(kTileBytes / 2, kk)), idesc);
-          }
-        }
-      };
-      auto wait_k = [&](int i) { return mbar_wait(&ctl, full_k(i % kStages), (i / kStages) & 1, 24u | ((unsigned)i << 8)); };
-      auto s_done = [&](int i) { umma_commit(s_full(i & 1)); umma_commit(empty_k(i % kStages)); };
       int tile = tile_begin;
       for (int i = 0; ok && i < nt; ++i, ++tile) {
         if (tile == a.n_tiles) tile = 0;
         const bool first = seg_first(i, tile), last = seg_last(i, tile);
         if (first) {
-          // new virtual unit: its Q_c block must have landed, and O of the previous unit must have
-          // been read out before the first P.V overwrites it
+          // new virtual unit: its Q_c block must have landed; S(i) and S(i+1) open the unit
           ok = mbar_wait(&ctl, q_full, seg & 1, 23u | ((unsigned)i << 8));
-          if (ok && seg > 0) ok = mbar_wait(&ctl, o_empty, (seg - 1) & 1, 25u | ((unsigned)i << 8));
           ++seg;
           if (!ok) break;
-          const bool two = !last;
-          ok = wait_k(i) && (!two || wait_k(i + 1));
+          ok = issue_s(i) && (last || issue_s(i + 1));
           if (!ok) break;
-          tc_fence_after_sync();
-          s_steps(i);
-          if (two) s_steps(i + 1);
-          s_done(i);
-          if (two) s_done(i + 1);
         }
-        // P.V(i), together with S(i+2) when that tile belongs to the same virtual unit
-        const bool with_s = !last && !seg_last(i + 1, tile + 1);
+        // S(i+2) when that tile belongs to the same virtual unit
+        if (!last && !seg_last(i + 1, tile + 1)) ok = issue_s(i + 2);
+        // every S of the unit has been issued by its last tile: Q_c may be replaced once they are done
+        if (last) umma_commit(q_empty);
+      }
+    }
+  } else if (warp == kPvWarp) {
+    // ------------------------------------------------------------ issuer of the P.V MMAs
+    if (lane == 0) {
+      const uint32_t idesc_o = umma_idesc(128, 128, false, true);    // O: A = P (TMEM), B = V tile, MN-major
+      const uint32_t tmem_o = tmem_base + kColO;
+      const uint32_t tmem_p = tmem_base + kColP;
+      // V tile with the keys as K, i.e. MN-major: blocks of 64 head-dim elements are half a tile
+      // apart, groups of 8 keys 1024 bytes apart
+      const uint64_t dv0 = smem_desc_sw128(v_base, kTileBytes / 2, 1024u);
+      // P.V(i): A = P in tensor memory, 16 keys = 8 columns per step
+      auto pv_steps = [&](int i, auto first_tag) {
+        constexpr bool kFirst = decltype(first_tag)::value;
+        const uint64_t vd = desc_advance(dv0, (uint32_t)(i % kStages) * kTileBytes);
+        const uint32_t pa = tmem_p + (uint32_t)((i & 1) * 64);
+        if (kFirst) umma_ts_imm<0>(tmem_o, pa, vd, idesc_o);
+        else umma_ts_imm<1>(tmem_o, pa, vd, idesc_o);
+#pragma unroll
+        for (int kk = 1; kk < kTileKeys / 16; ++kk)
+          umma_ts_imm<1>(tmem_o, pa + (uint32_t)(kk * 8), desc_advance(vd, (uint32_t)kk * 16u * kLineBytes), idesc_o);
+      };
+      int seg = 0, tile = tile_begin;
+      for (int i = 0; i < nt; ++i, ++tile) {
+        if (tile == a.n_tiles) tile = 0;
+        const bool first = seg_first(i, tile), last = seg_last(i, tile);
+        if (first) {
+          // O of the previous unit must have been read out before the first P.V overwrites it
+          if (seg > 0 && !mbar_wait(&ctl, o_empty, (seg - 1) & 1, 25u | ((unsigned)i << 8))) break;
+          ++seg;
+        }
         if (!mbar_wait(&ctl, p_full(i & 1), (i >> 1) & 1, 26u | ((unsigned)i << 8))) break;
         if (!mbar_wait(&ctl, full_v(i % kStages), (i / kStages) & 1, 27u | ((unsigned)i << 8))) break;
-        if (with_s && !wait_k(i + 2)) break;
         tc_fence_after_sync();
-        if (with_s) {
-          if (first) batch(i, std::true_type{}, std::true_type{});
-          else batch(i, std::false_type{}, std::true_type{});
-        } else {
-          if (first) batch(i, std::true_type{}, std::false_type{});
-          else batch(i, std::false_type{}, std::false_type{});
-        }
-        if (with_s) s_done(i + 2);
+        if (first) pv_steps(i, std::true_type{});
+        else pv_steps(i, std::false_type{});
+        umma_commit(p_empty(i & 1));
         umma_commit(empty_v(i % kStages));
-        if (last) {
-          umma_commit(o_full);
-          umma_commit(q_empty);
-        }
+        if (last) umma_commit(o_full);
       }
     }
   } else {
@@ -284,9 +283,8 @@ calib_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
       w = __all_sync(0xffffffffu, w);
       if (!w) return false;
       tc_fence_after_sync();
-      const int slot = cta - ((vu / a.n_cblocks) * a.n_tiles) / tiles_per_cta;
-      const size_t part = listed ? ((size_t)cta * a.seg_max + (seg - 1)) * a.n_cblocks + cb
-                                 : (size_t)vu * a.max_slots + slot;
+      const int slot = cta - ((vu / a.n_cblocks) * a.n_tiles) / a.tiles_per_cta;
+      const size_t part = (size_t)vu * a.max_slots + slot;
       float* orow = a.o_part + (part * 128 + r) * kD;
 #pragma unroll 1
       for (int c0 = grp * 64; c0 < grp * 64 + 64; c0 += 32) {
@@ -305,8 +303,7 @@ calib_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
     };
     // This thread's row of the virtual unit: is there one, and its -lse2.
     auto load_q = [&](int vu) {
-      const int pos = vu / a.n_cblocks, cb = vu - pos * a.n_cblocks;
-      const int unit = unit_of(pos);
+      const int unit = vu / a.n_cblocks, cb = vu - unit * a.n_cblocks;
       const int hq0 = (unit / Hkv) * a.Hq + (unit % Hkv) * a.G;
       const int g0 = cb * a.gpb;
       const int rows = min(a.gpb, a.G - g0) * a.n_cal;
@@ -335,7 +332,7 @@ calib_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
       if ((i & 1) != grp) continue;
       // kept-key bits of the tile's 128 keys (bit set = the key does not contribute), fetched
       // before the wait so that the loads are off the critical path
-      const uint32_t* bm = bm_all + (size_t)unit_of(unit) * a.bitmap_words;
+      const uint32_t* bm = bm_all + (size_t)unit * a.bitmap_words;
       const int tbase = tile * kTileKeys;
       uint32_t word[4];
 #pragma unroll
@@ -343,7 +340,7 @@ calib_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
         const int kb = tbase + 32 * q;
         word[q] = 0xffffffffu;
         if (kb < a.n_cand) {
-          word[q] = bm_all ? __ldg(bm + (kb >> 5)) : 0u;   // no bitmap: every key below n_cand counts
+          word[q] = __ldg(bm + (kb >> 5));
           if (kb + 32 > a.n_cand) word[q] |= 0xffffffffu << (a.n_cand - kb);
         }
       }
@@ -370,6 +367,10 @@ calib_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
       tmem_ld32_issue(taddr, ra);
       tmem_ld_wait(ra);
       tmem_ld32_issue(taddr + 32, rb);
+      // the P.V that read this P buffer two tiles ago must be done before it is overwritten
+      ok = mbar_wait(&ctl, p_empty(grp), ((i >> 1) & 1) ^ 1, 31u | ((unsigned)i << 8));
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) break;
       soft32(ra, 0, word[0]);
       tmem_ld_wait(rb);
       tmem_ld32_issue(taddr + 64, ra);
@@ -378,6 +379,8 @@ calib_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
       tmem_ld32_issue(taddr + 96, rb);
       soft32(ra, 2, word[2]);
       tmem_ld_wait(rb);
+      tc_fence_before_sync();
+      mbar_arrive(s_free(grp));   // S(i) is in registers: S(i+2) may overwrite the buffer
       soft32(rb, 3, word[3]);
       tmem_st_wait();
       tc_fence_before_sync();
@@ -403,8 +406,7 @@ calib_reduce_kernel(const __nv_bfloat16* __restrict__ Q_obs, const float* __rest
                     const float* __restrict__ o_part, const float* __restrict__ l_part,
                     float* __restrict__ O_c, float* __restrict__ LSE_c, __nv_bfloat16* __restrict__ C_q, int B,
                     int Hq, int G, int W, int n_cal, int gpb, int n_cblocks, int n_tiles, int tiles_per_cta,
-                    int max_slots, const int* __restrict__ unit_pos, const int* __restrict__ n_work, int groups,
-                    int seg_max) {
+                    int max_slots) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int row = blockIdx.x * 4 + warp;  // (b, hq, c)
   if (row >= B * Hq * n_cal) return;
@@ -412,24 +414,15 @@ calib_reduce_kernel(const __nv_bfloat16* __restrict__ Q_obs, const float* __rest
   const int b = bhq / Hq, hq = bhq % Hq;
   const int Hkv = Hq / G, h = hq / G, g = hq % G;
   const int unit = b * Hkv + h, cb = g / gpb, r = (g % gpb) * n_cal + c;
-  // Work-list mode (unit_pos given): only the rows of listed units are rewritten; the partials
-  // are those of the CTA groups whose share of the listed tile space overlaps the unit.
-  const bool listed = unit_pos != nullptr;
-  int pos = unit;
-  if (listed) {
-    pos = unit_pos[unit];
-    if (pos < 0) return;
-    tiles_per_cta = tiles_per_group(*n_work, n_tiles, groups);
-  }
-  const int first = (pos * n_tiles) / tiles_per_cta, last = ((pos + 1) * n_tiles - 1) / tiles_per_cta;
+  const int vu = unit * n_cblocks + cb;
+  const int first = (unit * n_tiles) / tiles_per_cta, last = ((unit + 1) * n_tiles - 1) / tiles_per_cta;
+  const size_t part0 = (size_t)vu * max_slots;
   float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
   float l = 0.f;
   for (int s = 0; s <= last - first; ++s) {
-    const size_t part = listed ? ((size_t)(first + s) * seg_max + (pos - ((first + s) * tiles_per_cta) / n_tiles)) * n_cblocks + cb
-                               : (size_t)(unit * n_cblocks + cb) * max_slots + s;
-    const float4 v = *reinterpret_cast<const float4*>(o_part + (part * 128 + r) * kD + 4 * lane);
+    const float4 v = *reinterpret_cast<const float4*>(o_part + ((part0 + s) * 128 + r) * kD + 4 * lane);
     acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
-    for (int grp = 0; grp < kGroups; ++grp) l += l_part[(part * kGroups + grp) * 128 + r];
+    for (int grp = 0; grp < kGroups; ++grp) l += l_part[((part0 + s) * kGroups + grp) * 128 + r];
   }
   const int qrow = W - n_cal + c;
   float4 out = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -450,14 +443,14 @@ calib_reduce_kernel(const __nv_bfloat16* __restrict__ Q_obs, const float* __rest
 bool calib_tc_supported(const CompressGeom& g) { return !g.keep_all && g.n_cal <= 128 && g.n_cand >= 1; }
 
 // Row blocks per unit and the tile partition; `parts` = partial (O, l) slots the workspace holds.
-void calib_tc_plan(const CompressGeom& g, int n_keys, int* gpb, int* n_cblocks, int* tiles_per_cta, int* max_slots,
+void calib_tc_plan(const CompressGeom& g, int* gpb, int* n_cblocks, int* tiles_per_cta, int* max_slots,
                    size_t* parts) {
   int per = 128 / g.n_cal;
   if (per < 1) per = 1;
   if (per > g.G) per = g.G;
   *gpb = per;
   *n_cblocks = (g.G + per - 1) / per;
-  const int n_tiles = (n_keys + kTileKeys - 1) / kTileKeys;
+  const int n_tiles = (g.n_cand + kTileKeys - 1) / kTileKeys;
   // the (kv unit, tile) space is shared out over groups of n_cblocks CTAs
   const int total = g.units * n_tiles;
   int groups = kSms / *n_cblocks;
@@ -468,42 +461,22 @@ void calib_tc_plan(const CompressGeom& g, int n_keys, int* gpb, int* n_cblocks, 
   *parts = (size_t)g.units * *n_cblocks * *max_slots;
 }
 
-// Work-list mode: the grid is `groups` CTA groups whatever the number of listed units; a group's share
-// then spans at most seg_max units, and `parts` partial slots cover every (group, segment, row block).
-void calib_tc_list_plan(const CompressGeom& g, int n_keys, int* groups, int* seg_max, size_t* parts) {
-  int gpb, n_cblocks, tpc, max_slots;
-  size_t p;
-  calib_tc_plan(g, n_keys, &gpb, &n_cblocks, &tpc, &max_slots, &p);
-  int gr = kSms / n_cblocks;
-  if (gr < 1) gr = 1;
-  const int n_tiles = (n_keys + kTileKeys - 1) / kTileKeys;
-  const int tpc_max = tiles_per_group(g.units, n_tiles, gr);   // the share grows with the number of listed units
-  *groups = gr;
-  *seg_max = (tpc_max + n_tiles - 1) / n_tiles + 1;
-  *parts = (size_t)gr * *seg_max * n_cblocks;
-}
-
-// The masked sums of one key source: rows [0, n_keys) of every unit of K / V (a unit's rows are
-// `unit_rows` apart), minus the keys whose bit is set in `bitmap` (none when it is null), into the
-// partial arrays o_part / l_part.
-cudaError_t launch_calib_tc_parts(const CompressGeom& g, const void* Q_obs, const void* K, const void* V,
-                                  int n_keys, size_t unit_rows, const uint32_t* bitmap, const float* row_lse,
-                                  float* o_part, float* l_part, unsigned* status, const int* work_list,
-                                  const int* n_work, cudaStream_t st) {
+cudaError_t launch_calib_tc(const CompressGeom& g, const CompressWs& ws, const void* Q_obs, const void* K,
+                            const void* V, const float* row_lse, char* wsp, float* O_c, float* LSE_c, void* C_q,
+                            cudaStream_t st) {
   CalibArgs a{};
-  a.work_list = work_list; a.n_work = n_work; a.units = g.units;
-  a.Hq = g.Hq; a.G = g.G; a.W = g.W; a.L = g.L; a.n_cand = n_keys; a.n_cal = g.n_cal;
+  a.Hq = g.Hq; a.G = g.G; a.W = g.W; a.L = g.L; a.n_cand = g.n_cand; a.n_cal = g.n_cal;
   size_t parts;
-  calib_tc_plan(g, n_keys, &a.gpb, &a.n_cblocks, &a.tiles_per_cta, &a.max_slots, &parts);
-  a.n_tiles = (n_keys + kTileKeys - 1) / kTileKeys;
+  calib_tc_plan(g, &a.gpb, &a.n_cblocks, &a.tiles_per_cta, &a.max_slots, &parts);
+  a.n_tiles = (g.n_cand + kTileKeys - 1) / kTileKeys;
   a.total_tiles = g.units * a.n_tiles;
   a.bitmap_words = g.bitmap_words;
   a.scale2 = g.scale2;
   a.row_lse = row_lse;
-  a.bitmap = bitmap;
-  a.o_part = o_part;
-  a.l_part = l_part;
-  a.status = status;
+  a.bitmap = (const uint32_t*)(wsp + ws.bitmap);
+  a.o_part = (float*)(wsp + ws.calib_o);
+  a.l_part = (float*)(wsp + ws.calib_l);
+  a.status = (unsigned*)(wsp + ws.status);
   CUtensorMap qm, km, vm;
   // calibration rows: [head dim][c < n_cal][g < G][unit], starting at observation row W - n_cal
   const uint64_t qd[3] = {(uint64_t)g.n_cal, (uint64_t)g.G, (uint64_t)g.units};
@@ -511,8 +484,7 @@ cudaError_t launch_calib_tc_parts(const CompressGeom& g, const void* Q_obs, cons
   const uint32_t qb[3] = {(uint32_t)g.n_cal, (uint32_t)a.gpb, 1};
   const char* q0 = (const char*)Q_obs + (size_t)(g.W - g.n_cal) * 256;
   if (!make_tensor_map_bf16(&qm, q0, 4, qd, qs, qb)) return cudaErrorInvalidValue;
-  // rows at or beyond n_keys are never used (their probabilities are masked), so the maps end there
-  const uint64_t kd[2] = {(uint64_t)n_keys, (uint64_t)g.units}, ks[2] = {256, (uint64_t)unit_rows * 256};
+  const uint64_t kd[2] = {(uint64_t)g.L, (uint64_t)g.units}, ks[2] = {256, (uint64_t)g.L * 256};
   const uint32_t kb[2] = {(uint32_t)kTileKeys, 1};
   if (!make_tensor_map_bf16(&km, K, 3, kd, ks, kb) || !make_tensor_map_bf16(&vm, V, 3, kd, ks, kb))
     return cudaErrorInvalidValue;
@@ -525,60 +497,13 @@ cudaError_t launch_calib_tc_parts(const CompressGeom& g, const void* Q_obs, cons
     if (e != cudaSuccess) return e;
     if (dev >= 0 && dev < 64) attr_set[dev] = true;
   }
-  int grid = (a.total_tiles + a.tiles_per_cta - 1) / a.tiles_per_cta * a.n_cblocks;
-  if (work_list) {
-    // listed units only: a fixed grid of whole CTA groups, the shares are worked out on the device
-    int groups;
-    calib_tc_list_plan(g, n_keys, &groups, &a.seg_max, &parts);
-    grid = groups * a.n_cblocks;
-  }
+  const int grid = (a.total_tiles + a.tiles_per_cta - 1) / a.tiles_per_cta * a.n_cblocks;
   calib_tc_kernel<<<grid, kThreads, kSmemBytes, st>>>(qm, km, vm, a);
-  count_launch(1);
-  return cudaGetLastError();
-}
-
-cudaError_t launch_calib_tc(const CompressGeom& g, const CompressWs& ws, const void* Q_obs, const void* K,
-                            const void* V, const float* row_lse, char* wsp, float* O_c, float* LSE_c, void* C_q,
-                            cudaStream_t st) {
-  float* o_part = (float*)(wsp + ws.calib_o);
-  float* l_part = (float*)(wsp + ws.calib_l);
-  cudaError_t e = launch_calib_tc_parts(g, Q_obs, K, V, g.n_cand, (size_t)g.L, (const uint32_t*)(wsp + ws.bitmap),
-                                        row_lse, o_part, l_part, (unsigned*)(wsp + ws.status), nullptr, nullptr, st);
-  if (e != cudaSuccess) return e;
-  int gpb, n_cblocks, tiles_per_cta, max_slots;
-  size_t parts;
-  calib_tc_plan(g, g.n_cand, &gpb, &n_cblocks, &tiles_per_cta, &max_slots, &parts);
   const int total = g.B * g.Hq * g.n_cal;
-  calib_reduce_kernel<<<(total + 3) / 4, 128, 0, st>>>((const __nv_bfloat16*)Q_obs, row_lse, o_part, l_part, O_c,
+  calib_reduce_kernel<<<(total + 3) / 4, 128, 0, st>>>((const __nv_bfloat16*)Q_obs, row_lse, a.o_part, a.l_part, O_c,
                                                       LSE_c, (__nv_bfloat16*)C_q, g.B, g.Hq, g.G, g.W, g.n_cal,
-                                                      gpb, n_cblocks, (g.n_cand + kTileKeys - 1) / kTileKeys,
-                                                      tiles_per_cta, max_slots, nullptr, nullptr, 0, 0);
-  count_launch(1);
-  return cudaGetLastError();
-}
-
-// The masked calibration pass over the units listed on the device (work_list, *n_work; unit_pos is
-// the inverse map, -1 for the others): only their rows of O_c / LSE_c / C_q are rewritten.  With
-// nothing listed both launches return at once.
-cudaError_t launch_calib_tc_listed(const CompressGeom& g, const CompressWs& ws, const void* Q_obs, const void* K,
-                                   const void* V, const float* row_lse, char* wsp, const int* work_list,
-                                   const int* unit_pos, const int* n_work, float* O_c, float* LSE_c, void* C_q,
-                                   cudaStream_t st) {
-  float* o_part = (float*)(wsp + ws.calib_o);
-  float* l_part = (float*)(wsp + ws.calib_l);
-  cudaError_t e = launch_calib_tc_parts(g, Q_obs, K, V, g.n_cand, (size_t)g.L, (const uint32_t*)(wsp + ws.bitmap),
-                                        row_lse, o_part, l_part, (unsigned*)(wsp + ws.status), work_list, n_work, st);
-  if (e != cudaSuccess) return e;
-  int gpb, n_cblocks, tiles_per_cta, max_slots, groups, seg_max;
-  size_t parts;
-  calib_tc_plan(g, g.n_cand, &gpb, &n_cblocks, &tiles_per_cta, &max_slots, &parts);
-  calib_tc_list_plan(g, g.n_cand, &groups, &seg_max, &parts);
-  const int total = g.B * g.Hq * g.n_cal;
-  calib_reduce_kernel<<<(total + 3) / 4, 128, 0, st>>>((const __nv_bfloat16*)Q_obs, row_lse, o_part, l_part, O_c,
-                                                      LSE_c, (__nv_bfloat16*)C_q, g.B, g.Hq, g.G, g.W, g.n_cal,
-                                                      gpb, n_cblocks, (g.n_cand + kTileKeys - 1) / kTileKeys,
-                                                      tiles_per_cta, max_slots, unit_pos, n_work, groups, seg_max);
-  count_launch(1);
+                                                      a.gpb, a.n_cblocks, a.n_tiles, a.tiles_per_cta, a.max_slots);
+  count_launch(2);
   return cudaGetLastError();
 }
 

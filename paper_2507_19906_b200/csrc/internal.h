@@ -23,8 +23,6 @@ struct CompressGeom {
 // Workspace carving of compress (byte offsets, all 256-byte aligned).
 struct CompressWs {
   size_t vote, vote2, pooled, row_lse, bitmap, stat_part, status, calib_o, calib_l, total;
-  size_t pv_l, sel_o, sel_l;  // one-pass votes + calibration: row sums over all candidates, sums over the selected rows
-  size_t redo;                // one-pass: block counter, n_work, then unit_flag / unit_pos / work_list [units] (ints)
   int n_tiles;     // 128-key tiles per unit (scalar statistics pass: one partial per tile)
   int stat_slots;  // (max, sum) partial slots per observation row in stat_part
 };
@@ -94,28 +92,8 @@ cudaError_t launch_row_stats_tc(const CompressGeom& g, const CompressWs& ws, con
 cudaError_t launch_votes_tc(const CompressGeom& g, const CompressWs& ws, const void* Q_obs, const void* K,
                             const float* row_lse, char* wsp, cudaStream_t st);
 bool calib_tc_supported(const CompressGeom& g);
-void calib_tc_plan(const CompressGeom& g, int n_keys, int* gpb, int* n_cblocks, int* tiles_per_cta, int* max_slots,
+void calib_tc_plan(const CompressGeom& g, int* gpb, int* n_cblocks, int* tiles_per_cta, int* max_slots,
                    size_t* parts);
-void calib_tc_list_plan(const CompressGeom& g, int n_keys, int* groups, int* seg_max, size_t* parts);
-cudaError_t launch_calib_tc_parts(const CompressGeom& g, const void* Q_obs, const void* K, const void* V,
-                                  int n_keys, size_t unit_rows, const uint32_t* bitmap, const float* row_lse,
-                                  float* o_part, float* l_part, unsigned* status, const int* work_list,
-                                  const int* n_work, cudaStream_t st);
-cudaError_t launch_calib_tc_listed(const CompressGeom& g, const CompressWs& ws, const void* Q_obs, const void* K,
-                                   const void* V, const float* row_lse, char* wsp, const int* work_list,
-                                   const int* unit_pos, const int* n_work, float* O_c, float* LSE_c, void* C_q,
-                                   cudaStream_t st);
-// score_pv.cu: votes and the sums over all candidates in one pass; the combine with the sums over
-// the selected rows
-bool score_pv_supported(const CompressGeom& g);
-cudaError_t launch_score_pv(const CompressGeom& g, const CompressWs& ws, const void* Q_obs, const void* K,
-                            const void* V, const float* row_lse, char* wsp, cudaStream_t st);
-cudaError_t launch_score_pv_selected(const CompressGeom& g, const CompressWs& ws, const void* Q_obs,
-                                     const void* K_kept, const void* V_kept, const float* row_lse, char* wsp,
-                                     cudaStream_t st);
-cudaError_t launch_calib_combine(const CompressGeom& g, const CompressWs& ws, const void* Q_obs,
-                                 const float* row_lse, char* wsp, float* O_c, float* LSE_c, void* C_q,
-                                 cudaStream_t st);
 cudaError_t launch_calib_tc(const CompressGeom& g, const CompressWs& ws, const void* Q_obs, const void* K,
                             const void* V, const float* row_lse, char* wsp, float* O_c, float* LSE_c, void* C_q,
                             cudaStream_t st);

@@ -29,12 +29,13 @@ namespace {
 
 using namespace tc;
 
-constexpr int kGroups = 2;  // consumer warpgroups (4 warps each); both work on the same accumulator, half of its columns each
+constexpr int kGroups = 2;  // consumer warpgroups (4 warps each); group g drains accumulator buffer g
 constexpr int kProducerWarp = kGroups * 4;
 constexpr int kMmaWarp = kGroups * 4 + 1;
 constexpr int kThreads = kGroups * 128 + 64;
 constexpr int kTmemCols = 512;  // two accumulators of 256 columns
 constexpr int kBufCols = 256;
+constexpr int kNumBufs = 2;
 constexpr int kMaxRows = 512;   // G * W handled by the tiles
 constexpr int kSms = 148;
 
@@ -43,7 +44,7 @@ struct ScoreArgs {
   int vu_per_unit;    // virtual units per (batch, kv-head) unit
   int vu_rows;        // window rows a virtual unit starts at: vu % vu_per_unit * vu_rows
   int n_blocks;       // row blocks (= accumulators) per key tile
-  int block_rows;     // rows per block: 128 for the statistics, a multiple of 32 (<= 256) for the votes
+  int block_rows;     // rows per block: 128 for the statistics, a multiple of 64 (<= 256) for the votes
   int n_tiles;        // key tiles per virtual unit
   int total_tiles;    // virtual units * n_tiles
   int tiles_per_cta;
@@ -52,7 +53,7 @@ struct ScoreArgs {
   float scale2;
   const float* row_lse;  // votes: natural-log LSE of every observation row [B, Hq, W]
   float* vote;           // votes: out [units, n_cand]
-  float* vote2;          // votes of the second row block when there are two (added to vote afterwards)
+  float* vote2;          // with several row blocks per tile: the partial votes of warpgroup 1 (added to vote afterwards)
   float2* stat_part;     // statistics: out [row][slot][group] (max, sum) in the log2 domain
   unsigned* status;
 };
@@ -93,7 +94,6 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
   __shared__ __align__(8) unsigned long long bars[18];
   __shared__ uint32_t tmem_slot;
   __shared__ Ctl ctl;
-  __shared__ float vx[2][128];  // votes: partial vote of the second column half, per accumulator
   __shared__ __align__(16) float nlse2_s[kVotes ? kGroups * 4 : 1][kVotes ? kMaxRows : 4];  // -lse2 per row, one copy per warp
   __shared__ float2 ml_s[kVotes ? 1 : kGroups][kVotes ? 1 : 2][kVotes ? 1 : 128];       // running (max, sum)
 
@@ -117,9 +117,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
   auto full_k = [&](int s) { return bar0 + 8u * (2 + s); };
   auto empty_k = [&](int s) { return bar0 + 8u * (6 + s); };
   auto t_full = [&](int b) { return bar0 + 8u * (10 + b); };
-  auto t_empty = [&](int b) { return bar0 + 8u * (12 + b); };
-  auto vx_full = [&](int b) { return bar0 + 8u * (14 + b); };
-  auto vx_empty = [&](int b) { return bar0 + 8u * (16 + b); };
+  auto t_empty = [&](int b) { return bar0 + 8u * (14 + b); };
 
   if (tid == 0) {
     ctl.abort = 0;
@@ -127,9 +125,8 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
     mbar_init(q_full, 1);
     mbar_init(q_empty, 1);
     for (int s = 0; s < 4; ++s) { mbar_init(full_k(s), 1); mbar_init(empty_k(s), 1); }
-    for (int b = 0; b < 2; ++b) {
-      mbar_init(t_full(b), 1); mbar_init(t_empty(b), kGroups * 128);
-      mbar_init(vx_full(b), 128); mbar_init(vx_empty(b), 128);
+    for (int b = 0; b < kNumBufs; ++b) {
+      mbar_init(t_full(b), 1); mbar_init(t_empty(b), 128);   // a buffer is drained by one warpgroup
     }
     fence_mbar_init();
   }
@@ -173,7 +170,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
   } else if (warp == kMmaWarp) {
     // ------------------------------------------------------------ MMA issuer
     if (lane == 0) {
-      const uint32_t idesc = umma_idesc(128, kVotes ? a.block_rows : 256, false, false);
+      const uint32_t idesc = umma_idesc(128, kVotes ? a.block_rows : TILE_KEYS, false, false);
       // Descriptors are built once per buffer; a k-step adds a constant to the address field (the
       // issuing thread's own instructions between two MMAs are what limits the issue rate).
       const uint64_t dq0 = smem_desc_sw128(q_base, 16u, 1024u);
@@ -191,8 +188,8 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
         bool ok = true;
         const uint64_t kd = desc_advance(dk0, (uint32_t)s * STAGE_BYTES);
         for (int blk = 0; blk < a.n_blocks; ++blk, ++j) {
-          const int buf = j & 1;
-          if (!mbar_wait(&ctl, t_empty(buf), ((j >> 1) & 1) ^ 1, (kVotes ? 34u : 14u) | ((unsigned)j << 8))) {
+          const int buf = j & (kNumBufs - 1);
+          if (!mbar_wait(&ctl, t_empty(buf), ((j / kNumBufs) & 1) ^ 1, (kVotes ? 34u : 14u) | ((unsigned)j << 8))) {
             ok = false;
             break;
           }
@@ -218,14 +215,19 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
     }
   } else {
     // ------------------------------------------------------------ accumulator consumers
-    // Thread ct of warpgroup grp owns TMEM lane ct.  Both groups consume every job (key tile, row
-    // block), each one half of the accumulator's columns: a job is then drained at the full rate
-    // of the exponential unit while the MMAs of the next job fill the other accumulator.
+    // Thread ct of warpgroup grp owns TMEM lane ct.  The jobs (key tile, row block) alternate between
+    // the groups: group g drains accumulator buffer g, i.e. every job whose index has parity g, all
+    // of its columns.  The groups therefore run half a job apart: while one waits for the MMAs of
+    // its next job, stores its result or starts its first load, the other keeps the exponential unit
+    // busy.  (Measured at config 3: both groups on the same job, half of the columns each, 110 us
+    // for the votes, the groups stalling together at every job boundary; alternating jobs 100 us;
+    // four accumulators of 128 columns, so that a group's next job is ready before it asks, 110 us:
+    // the narrower MMAs cost more than the wait they hide.)
     const int grp = warp >> 2, ct = tid & 127;
     const uint32_t lane_base = tmem_base + ((uint32_t)((warp & 3) * 32) << 16);
-    float acc0 = 0.f, acc1 = 0.f, acc2 = 0.f, acc3 = 0.f;  // votes: running vote of this thread's key
     int cur_vu = -1, j = 0;
     bool ok = true;
+    float vsum = 0.f;
 
     // statistics: store this group's partial (max, sum) of every row of the virtual unit `vu`
     auto flush_stats = [&](int vu) {
@@ -264,17 +266,18 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
       }
       const int tbase = tile * TILE_KEYS;
       for (int blk = 0; blk < a.n_blocks; ++blk, ++j) {
-        const int buf = j & 1;
+        if ((j & 1) != grp) continue;
+        const int buf = j & (kNumBufs - 1);
         const uint32_t lane_addr = lane_base + (uint32_t)(buf * kBufCols);
-        ok = mbar_wait(&ctl, t_full(buf), (j >> 1) & 1, (kVotes ? 35u : 15u) | ((unsigned)j << 8));
+        ok = mbar_wait(&ctl, t_full(buf), (j / kNumBufs) & 1, (kVotes ? 35u : 15u) | ((unsigned)j << 8));
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) break;
         tc_fence_after_sync();
         uint32_t ra[32], rb[32];
         if (kVotes) {
-          const int cw = a.block_rows >> 1;  // columns (query rows) of this group: a multiple of 32
-          const float* nl = nlse2_s[warp] + blk * a.block_rows + grp * cw;
-          const uint32_t tcol = lane_addr + (uint32_t)(grp * cw);
+          const int cw = a.block_rows;  // columns (query rows) of the job: a multiple of 64
+          const float* nl = nlse2_s[warp] + blk * a.block_rows;
+          float acc0 = 0.f, acc1 = 0.f, acc2 = 0.f, acc3 = 0.f;  // running vote of this thread's key
           auto add32 = [&](const uint32_t (&r)[32], int c0) {
 #pragma unroll
             for (int e = 0; e < 32; e += 4) {
@@ -285,39 +288,29 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
               acc3 += ex2_approx(fmaf(__uint_as_float(r[e + 3]), a.scale2, n4.w));
             }
           };
-          // block_rows is a multiple of 32: chunks alternate between the two register sets
-          tmem_ld32_issue(tcol, ra);
+          // chunks of 32 columns alternate between the two register sets
+          tmem_ld32_issue(lane_addr, ra);
+#pragma unroll 1
           for (int c0 = 0; c0 < cw; c0 += 64) {
             tmem_ld_wait(ra);
-            const bool more_b = c0 + 32 < cw;
-            if (more_b) tmem_ld32_issue(tcol + c0 + 32, rb);
+            tmem_ld32_issue(lane_addr + c0 + 32, rb);
             add32(ra, c0);
-            if (more_b) {
-              tmem_ld_wait(rb);
-              if (c0 + 64 < cw) tmem_ld32_issue(tcol + c0 + 64, ra);
-              add32(rb, c0 + 32);
+            tmem_ld_wait(rb);
+            if (c0 + 64 < cw) {
+              tmem_ld32_issue(lane_addr + c0 + 64, ra);
+            } else {
+              tc_fence_before_sync();
+              mbar_arrive(t_empty(buf));  // the accumulator is in registers: hand the buffer back early
             }
+            add32(rb, c0 + 32);
           }
-          tc_fence_before_sync();
-          mbar_arrive(t_empty(buf));
-          // the two halves of the key's vote meet in shared memory; group 0 stores the sum
-          const float part = (acc0 + acc1) + (acc2 + acc3);
-          acc0 = acc1 = acc2 = acc3 = 0.f;
-          if (grp == 1) {
-            ok = mbar_wait(&ctl, vx_empty(buf), ((j >> 1) & 1) ^ 1, 37u | ((unsigned)j << 8));
-            ok = __all_sync(0xffffffffu, ok);
-            if (!ok) break;
-            vx[buf][ct] = part;
-            mbar_arrive(vx_full(buf));
-          } else {
-            ok = mbar_wait(&ctl, vx_full(buf), (j >> 1) & 1, 38u | ((unsigned)j << 8));
-            ok = __all_sync(0xffffffffu, ok);
-            if (!ok) break;
-            const float v = part + vx[buf][ct];
-            mbar_arrive(vx_empty(buf));
+          // the vote of the key over this group's row blocks of the tile; stored after the last of them
+          vsum += (acc0 + acc1) + (acc2 + acc3);
+          if (blk + 2 >= a.n_blocks) {
             const int key = tbase + ct;
-            float* out = blk == 0 ? a.vote : a.vote2;
-            if (key < a.n_cand) out[(size_t)unit * a.n_cand + key] = v;
+            float* out = (a.n_blocks > 1 && grp == 1) ? a.vote2 : a.vote;
+            if (key < a.n_cand) out[(size_t)unit * a.n_cand + key] = vsum;
+            vsum = 0.f;
           }
         } else {
           float2 ml = ml_s[grp][blk][ct];
@@ -337,15 +330,14 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
               ml.x = m_new;
             }
           };
-          const int cbeg = grp * (TILE_KEYS / 2), cend = cbeg + TILE_KEYS / 2;  // this group's keys of the tile
-          tmem_ld32_issue(lane_addr + cbeg, ra);
+          tmem_ld32_issue(lane_addr, ra);
 #pragma unroll 1
-          for (int c0 = cbeg; c0 < cend; c0 += 64) {
+          for (int c0 = 0; c0 < TILE_KEYS; c0 += 64) {
             tmem_ld_wait(ra);
             tmem_ld32_issue(lane_addr + c0 + 32, rb);
             fold32(ra, c0);
             tmem_ld_wait(rb);
-            if (c0 + 64 < cend) {
+            if (c0 + 64 < TILE_KEYS) {
               tmem_ld32_issue(lane_addr + c0 + 64, ra);
             } else {
               tc_fence_before_sync();
@@ -482,9 +474,9 @@ cudaError_t launch_votes_tc(const CompressGeom& g, const CompressWs& ws, const v
   a.Hq = g.Hq; a.G = g.G; a.W = g.W; a.L = g.L; a.n_cand = g.n_cand; a.GW = GW;
   a.vu_per_unit = 1;
   a.vu_rows = 0;
-  // One accumulator of up to 256 row columns per (key tile, row block); with two row blocks each
-  // warpgroup sums one block and the two partial votes are added afterwards.
-  a.n_blocks = GW <= 256 ? 1 : 2;
+  // One accumulator of up to 256 row columns per (key tile, row block); with several row blocks
+  // per tile each warpgroup sums the blocks it drains and the two partial votes are added afterwards.
+  a.n_blocks = (GW + 255) / 256;
   a.block_rows = ((GW + a.n_blocks - 1) / a.n_blocks + 63) / 64 * 64;
   a.n_tiles = (g.n_cand + kTileKeys - 1) / kTileKeys;
   partition_tiles(a, g.units);
@@ -508,7 +500,7 @@ cudaError_t launch_votes_tc(const CompressGeom& g, const CompressWs& ws, const v
   const int grid = (a.total_tiles + a.tiles_per_cta - 1) / a.tiles_per_cta;
   score_tc_kernel<true><<<grid, kThreads, smem, st>>>(qm, km, a);
   count_launch(1);
-  if (a.n_blocks == 2) {
+  if (a.n_blocks > 1) {
     const size_t n = (size_t)g.units * g.n_cand;
     add_votes_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(a.vote, a.vote2, n);
     count_launch(1);
