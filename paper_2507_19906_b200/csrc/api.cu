@@ -106,16 +106,6 @@ int device_supported() {
   return major_of[dev] == 10;
 }
 
-// CALIDROP_COMPRESS_PATH=scalar (read once) routes compress through the CUDA-core kernels, for
-// diagnosis of the tensor-core path.
-bool scalar_path_forced() {
-  static const bool forced = [] {
-    const char* v = getenv("CALIDROP_COMPRESS_PATH");
-    return v && strcmp(v, "scalar") == 0;
-  }();
-  return forced;
-}
-
 // Split-K factor of the decode launch: one CTA per SM at most (a CTA's ring takes most of an SM's
 // shared memory), never fewer than 32 rows per split.
 int decode_nsplit(int units_total, int n_kv) {
@@ -253,7 +243,7 @@ int calidrop_compress(const calidrop_params* p, const void* Q_obs, const void* K
   if (e != cudaSuccess) return cuda_fail(e);
   // The contractions run on the tensor cores whenever the tiles cover the shape; the scalar
   // kernels remain for the rest (more than 512 window rows per kv head, budget >= L).
-  const bool tc_path = score_tc_supported(g) && !scalar_path_forced();
+  const bool tc_path = score_tc_supported(g);
   const float* row_lse = lse_obs;
   if (!g.keep_all) {
     if (!row_lse) {
@@ -264,8 +254,8 @@ int calidrop_compress(const calidrop_params* p, const void* Q_obs, const void* K
     e = tc_path ? launch_votes_tc(g, ws, Q_obs, K, row_lse, wsp, st) : launch_votes(g, ws, Q_obs, K, row_lse, wsp, st);
     if (e != cudaSuccess) return cuda_fail(e);
   }
-  e = (select_cluster_supported(g) && !scalar_path_forced()) ? launch_pool_select_cluster(g, ws, wsp, kept_idx, st)
-                                                             : launch_pool_select(g, ws, wsp, kept_idx, st);
+  e = select_cluster_supported(g) ? launch_pool_select_cluster(g, ws, wsp, kept_idx, st)
+                                  : launch_pool_select(g, ws, wsp, kept_idx, st);
   if (e != cudaSuccess) return cuda_fail(e);
   e = launch_gather(g, K, V, kept_idx, K_kept, V_kept, st);
   if (e != cudaSuccess) return cuda_fail(e);
@@ -295,7 +285,7 @@ int calidrop_calibrate(const calidrop_params* p, const void* Q_obs, const void* 
   char* wsp = (char*)workspace;
   cudaError_t e = cudaMemsetAsync(wsp + ws.status, 0, 4, st);
   if (e != cudaSuccess) return cuda_fail(e);
-  const bool tc_path = score_tc_supported(g) && !scalar_path_forced();
+  const bool tc_path = score_tc_supported(g);
   // the calibration probabilities refer to the full-row softmax: its row LSE comes from the caller
   // or from the statistics pass of the scoring
   const float* row_lse = lse_obs;

@@ -316,6 +316,26 @@ calib_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
     };
 
     const uint32_t* bm_all = a.bitmap;
+    // The four bitmap words of a tile are loaded RAW (nothing may touch a loaded value before the
+    // tile that uses it, or the thread waits for the load on the spot); the mask of the keys outside
+    // the candidates is worked out separately from the indices.
+    auto load_words = [&](int unit, int tile, uint32_t (&raw)[4], uint32_t (&msk)[4]) {
+      const uint32_t* bm = bm_all + (size_t)unit * a.bitmap_words;
+      const int tbase = tile * kTileKeys;
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        const int kb = tbase + 32 * q;
+        raw[q] = __ldg(bm + min(kb >> 5, a.bitmap_words - 1));   // always a valid word; the mask decides
+        msk[q] = kb >= a.n_cand ? 0xffffffffu : (kb + 32 > a.n_cand ? 0xffffffffu << (a.n_cand - kb) : 0u);
+      }
+    };
+    uint32_t next_raw[4] = {0u, 0u, 0u, 0u}, next_msk[4] = {0xffffffffu, 0xffffffffu, 0xffffffffu, 0xffffffffu};
+    {
+      // this group's first tile is local tile `grp`
+      int t0 = tile_begin + grp, u0 = unit_begin;
+      while (t0 >= a.n_tiles) { t0 -= a.n_tiles; ++u0; }
+      if (grp < nt) load_words(u0, t0, next_raw, next_msk);
+    }
     int vu = vu_begin, tile = tile_begin, unit = unit_begin;
     for (int i = 0; i < nt; ++i, ++tile) {
       if (tile == a.n_tiles) { tile = 0; ++unit; vu += a.n_cblocks; }
@@ -330,19 +350,16 @@ calib_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
         ++seg;
       }
       if ((i & 1) != grp) continue;
-      // kept-key bits of the tile's 128 keys (bit set = the key does not contribute), fetched
-      // before the wait so that the loads are off the critical path
-      const uint32_t* bm = bm_all + (size_t)unit * a.bitmap_words;
-      const int tbase = tile * kTileKeys;
+      // kept-key bits of the tile's 128 keys (bit set = the key does not contribute).  The words of
+      // this group's NEXT tile are requested now and used a whole tile later: a load consumed in the
+      // tile that issued it stalled the group for an L2 round trip on every tile.
       uint32_t word[4];
 #pragma unroll
-      for (int q = 0; q < 4; ++q) {
-        const int kb = tbase + 32 * q;
-        word[q] = 0xffffffffu;
-        if (kb < a.n_cand) {
-          word[q] = __ldg(bm + (kb >> 5));
-          if (kb + 32 > a.n_cand) word[q] |= 0xffffffffu << (a.n_cand - kb);
-        }
+      for (int q = 0; q < 4; ++q) word[q] = next_raw[q] | next_msk[q];
+      {
+        int t2 = tile + 2, u2 = unit;
+        while (t2 >= a.n_tiles) { t2 -= a.n_tiles; ++u2; }
+        if (i + 2 < nt) load_words(u2, t2, next_raw, next_msk);
       }
       ok = mbar_wait(&ctl, s_full(grp), (i >> 1) & 1, 28u | ((unsigned)i << 8));
       ok = __all_sync(0xffffffffu, ok);
