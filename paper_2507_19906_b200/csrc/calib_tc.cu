@@ -10,15 +10,17 @@
 //             the candidates; row sums l kept in fp32; p rounded to bf16 and stored into tensor
 //             memory as the A operand of
 //     MMA 2   O += P V          V tile from TMA, read as the MN-major B operand
-// MMAs that accumulate into the same tensor-memory tile execute one after the other (about 150
-// cycles each for a 128x128x16 step, twice its math time), so the issuer interleaves the eight
-// k-steps of S(i+2) with the eight of P.V(i): two independent accumulation chains keep the pipe
-// busy.  lse2[row] is the row's LSE over ALL the keys it sees (from the statistics pass or the
-// caller), so every p <= 1 and no running maximum or rescaling is needed: the partial (O, l) of
-// the key ranges simply add up.  calib_reduce_kernel sums them in a fixed order and writes
-// O_c = O / l, LSE_c = lse + log l, C_q.
+// lse2[row] is the row's LSE over ALL the keys it sees (from the statistics pass or the caller), so
+// every p <= 1 and no running maximum or rescaling is needed: the partial (O, l) of the key ranges
+// simply add up.  calib_reduce_kernel sums them in a fixed order and writes O_c = O / l,
+// LSE_c = lse + log l, C_q.
 // Warp roles: two softmax warpgroups (group g owns S buffer g and P buffer g, i.e. the tiles with
-// local index i % 2 == g), one TMA producer warp, one warp that allocates TMEM and issues MMAs.
+// local index i % 2 == g), two TMA producer warps (Q_c and K; V), and two MMA-issuing warps, one for
+// S and one for P.V: a single thread's dependent scalar instructions cost several cycles each, and
+// with the waits and commits of both chains on one thread the issue, not the tensor pipe, set the
+// pace (a lone chain of eight 128x128x16 MMAs runs at the pipe's 64 cycles each once its descriptors
+// are prepared; no interleaving of chains is needed).  S(i+2) is issued as soon as S(i) has been read
+// out of the buffer they share, not when P(i) is complete.
 // Tensor memory: S buffers at columns 0 and 128, O at 256, P buffers (64 columns each) at 384, 448.
 #include <type_traits>
 
