@@ -35,8 +35,9 @@ import numpy as np  # noqa: E402
 METRIC = "decode attn HBM GB/s (% of peak); compress+calibrate ms/layer (% TC peak)"
 UNIT = "GB/s"
 FALLBACK_HBM_GBS, FALLBACK_BF16_TFLOPS = 6650.0, 1590.0
-# dram__bytes_read.sum + dram__bytes_write.sum per decode launch at config 3 from the committed ncu
-# capture (profiles/decode_kernel_config3.md); reported only for that workload.
+# dram__bytes_read.sum + dram__bytes_write.sum per decode launch at config 3, n_cal 64, from one ncu
+# capture of the decode kernel (cold caches: every launch of the capture reads its whole cache from
+# DRAM); reported only for that workload.
 DECODE_DRAM_TRAFFIC_PER_LAUNCH = 35872128
 
 
@@ -99,6 +100,13 @@ def compress_bytes(cfg):
     """Minimum bytes: K once, V once, the gather's read and write of the kept rows."""
     kv = cfg.B * cfg.Hkv * cfg.L * cfg.D * 2
     return 2 * kv + 4 * cfg.B * cfg.Hkv * cfg.budget * cfg.D * 2
+
+
+def compress_floors(cfg, n_cal, lse_supplied, peaks):
+    """Microseconds per layer that each of the three co-limiting resources needs on its own."""
+    return {"tensor": compress_flops(cfg, n_cal) / (peaks["bf16_tflops_sustained"] * 1e12) * 1e6,
+            "hbm": compress_bytes(cfg) / (peaks["hbm_gbs"] * 1e9) * 1e6,
+            "exp": compress_exps(cfg, n_cal, lse_supplied) / (XU_PER_CLK_PER_SM * N_SMS * SM_MAX_HZ) * 1e6}
 
 
 class ClockSampler:
@@ -286,6 +294,8 @@ def run_gpu(args):
     t_dec = sum(e[1].elapsed_time(e[2]) for e in ev)
     t_tot = sum(e[0].elapsed_time(e[2]) for e in ev)
     t_comp, t_dec, t_tot = max_over_ranks([t_comp, t_dec, t_tot], world, "cuda")
+    dec_step_ms = sorted(e[1].elapsed_time(e[2]) for e in ev)      # this rank's timed repetitions of the decode phase
+    comp_step_ms = sorted(e[0].elapsed_time(e[1]) for e in ev)
 
     dec_bytes_step = sum(decode_bytes(cfg, n_cal, cfg.budget + t + 1) for t in range(T)) * S
     dec_launches = T * (1 if args.batched_decode else S) * args.steps
@@ -393,8 +403,21 @@ def run_gpu(args):
                    "parallelism": "replicas only" if world > 1 else "single GPU"},
         "decode": {"us_per_launch": avg_launch_s * 1e6, "gbs": dec_gbs, "launches": dec_launches,
                    "bytes_per_launch": bytes_per_launch,
+                   # spread over the timed repetitions of the decode phase (each T x states launches)
+                   "us_per_launch_median": dec_step_ms[len(dec_step_ms) // 2] * 1e3 / (dec_launches / args.steps),
+                   "us_per_launch_min": dec_step_ms[0] * 1e3 / (dec_launches / args.steps),
+                   "us_per_launch_max": dec_step_ms[-1] * 1e3 / (dec_launches / args.steps),
+                   "repetitions": args.steps,
                    "frac_of_measured_hbm": dec_gbs / peaks["hbm_gbs"], "frac_of_nominal_8tbs": dec_gbs / 8000.0},
-        "compress": {"ms_per_layer": comp_ms_layer, "algorithmic_tflops": comp_tflops,
+        "compress": {"ms_per_layer": comp_ms_layer,
+                     "ms_per_layer_median": comp_step_ms[len(comp_step_ms) // 2] / S,
+                     # the three floors of the step (tensor pipe at the sustained bf16 peak, copy bandwidth on
+                     # the minimum bytes, special-function pipe on the exponentials); the step is bound by
+                     # the largest, and frac_of_bound = that floor / measured time
+                     "floor_us": compress_floors(cfg, n_cal, args.lse_obs, peaks),
+                     "frac_of_bound": max(compress_floors(cfg, n_cal, args.lse_obs, peaks).values())
+                     / (comp_ms_layer * 1e3),
+                     "algorithmic_tflops": comp_tflops,
                      "frac_of_bf16_peak_burst": comp_tflops / peaks["bf16_tflops"],
                      "frac_of_bf16_peak_sustained": comp_tflops / peaks["bf16_tflops_sustained"],
                      "min_bytes_gbs": comp_gbs, "frac_of_measured_hbm": comp_gbs / peaks["hbm_gbs"],
@@ -507,10 +530,23 @@ def run_reference(args):
     }))
 
 
-def main():
+def replica_command(n_gpus, argv, port):
+    """The command line that runs this file as n_gpus processes on this node, one rank per GPU."""
+    return [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n_gpus}",
+            "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + list(argv)
+
+
+def spawn_replicas(n_gpus, argv, run=None):
+    """`bench.py --gpus N` without a launcher: start the N replicas (the path has no exchange step, so
+    the ranks only meet in the barrier and the max-over-ranks of the timing) and pass their output on."""
+    port = 29500 + os.getpid() % 1000
+    return (run or subprocess.call)(replica_command(n_gpus, argv, port))
+
+
+def main(argv=None):
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=3)
+    ap.add_argument("--steps", type=int, default=5)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", type=int, default=3)
@@ -530,12 +566,16 @@ def main():
                     help="supply the row log-sum-exp of the prefill attention to calidrop_compress (as a prefill "
                          "kernel would), so the statistics pass is skipped; not the default workload")
     ap.add_argument("--no-graph", action="store_true", help="launch every call eagerly instead of replaying CUDA graphs")
-    args = ap.parse_args()
+    args = ap.parse_args(argv)
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        # started as a plain process: become the launcher of N replica processes, one per GPU
+        return spawn_replicas(args.gpus, sys.argv[1:] if argv is None else list(argv))
     if args.impl == "reference":
         run_reference(args)
     else:
         run_gpu(args)
+    return 0
 
 
 if __name__ == "__main__":
-    main()
+    sys.exit(main())

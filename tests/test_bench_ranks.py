@@ -47,3 +47,23 @@ def test_single_rank_is_the_identity():
     import bench
     assert bench.max_over_ranks([1.5, 2.5], 1, "cpu") == [1.5, 2.5]
     assert bench.whole_job_rate(10.0, 1, 5.0) == pytest.approx(2000.0)
+
+
+def test_gpus_flag_without_a_launcher_starts_the_replicas(monkeypatch):
+    """`bench.py --gpus 2` started as a plain process re-launches itself as two ranks (one per GPU)
+    with the same arguments; under a launcher (WORLD_SIZE set) it runs as a rank instead."""
+    import bench
+    monkeypatch.delenv("WORLD_SIZE", raising=False)
+    seen = []
+    monkeypatch.setattr(bench.subprocess, "call", lambda cmd: seen.append(cmd) or 0)
+    argv = ["--gpus", "2", "--steps", "4", "--warmup", "3"]
+    assert bench.main(argv) == 0
+    (cmd,) = seen
+    assert cmd[1:3] == ["-m", "torch.distributed.run"] and "--nproc-per-node=2" in cmd and "--nnodes=1" in cmd
+    assert cmd[cmd.index("--master-addr") + 1] == "127.0.0.1"
+    assert cmd[-len(argv):] == argv and cmd[-len(argv) - 1].endswith("bench.py")
+    # as a rank of a launched job the same flags do not spawn again
+    monkeypatch.setenv("WORLD_SIZE", "2")
+    ran = []
+    monkeypatch.setattr(bench, "run_gpu", lambda args: ran.append(args.gpus))
+    assert bench.main(argv) == 0 and ran == [2] and len(seen) == 1
