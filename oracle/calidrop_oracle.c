@@ -25,6 +25,13 @@
  *     textbook routine in the tests).
  *   - n_cal > 1 (several calibration queries, decode picks the most similar one, ties to
  *     the most recent) is an extension; n_cal = 1 is Algorithm 1 verbatim.
+ *   - The "calibration size" of Section 4.4 (Efficiency Optimization; Fig. 3c): the evicted
+ *     tokens are ranked by importance and only the first m are kept for calibration and
+ *     offloading.  Importance is read as the pooled vote the eviction rule already ranks by,
+ *     with the same tie rule (lower index first), so the calibrated set is the next m
+ *     candidates after the selected ones in one and the same order.  PARITY UNPINNED for the
+ *     choice of the importance measure (the paper names none); m >= |E| is Algorithm 1 as
+ *     printed.
  */
 #include <math.h>
 #include <stdint.h>
@@ -171,6 +178,7 @@ void oracle_topk(const double* score, int64_t n, int64_t k, int32_t* out_sorted)
  */
 static void unit_calibrate(const uint16_t* Qobs, const uint16_t* K, const uint16_t* V,
                            const int32_t* kept, int64_t n_kept,
+                           const int32_t* calib_set, int64_t n_set, /* NULL: every evicted candidate */
                            int G, int W, int64_t L, int D, int n_cal, int64_t cap, double scale,
                            uint16_t* K_kept, uint16_t* V_kept,
                            double* O_c /* [G, n_cal, D] */, double* LSE_c /* [G, n_cal] */,
@@ -188,6 +196,11 @@ static void unit_calibrate(const uint16_t* Qobs, const uint16_t* K, const uint16
     int64_t n_e = 0;
     for (int64_t t = 0; t < n_cand; ++t)
         if (!is_kept[t]) evicted[n_e++] = (int32_t)t;
+    if (calib_set) {   /* calibration size: only the listed evicted tokens take part */
+        n_e = 0;
+        for (int64_t i = 0; i < n_set; ++i)
+            if (!is_kept[calib_set[i]]) evicted[n_e++] = calib_set[i];
+    }
     for (int g = 0; g < G; ++g) {
         for (int c = 0; c < n_cal; ++c) {
             const uint16_t* q = Qobs + ((int64_t)g * W + (W - n_cal + c)) * D;
@@ -206,6 +219,9 @@ static void unit_calibrate(const uint16_t* Qobs, const uint16_t* K, const uint16
  * n_kept = min(budget, L); K_kept,V_kept [B,Hkv,cap,D]; O_c [B,Hq,n_cal,D], LSE_c
  * [B,Hq,n_cal] (double); C_q [B,Hq,n_cal,D] (bf16 bits); vote, pooled [B,Hkv,L-W] and
  * row_lse [B,Hq,W] (double; may be NULL).
+ * calib_size < 0: every evicted candidate is calibrated (Algorithm 1 as printed).  Otherwise only
+ * the m = min(calib_size, number evicted) evicted candidates of highest pooled vote (ties to the
+ * lower index) are; their ascending indices go to calib_idx [B,Hkv,m] when it is not NULL.
  * Returns 0, or -1 for arguments the method does not define (budget <= window < L).
  */
 int oracle_compress(const uint16_t* Q_obs, const uint16_t* K, const uint16_t* V,
@@ -213,7 +229,8 @@ int oracle_compress(const uint16_t* Q_obs, const uint16_t* K, const uint16_t* V,
                     int n_cal, int64_t cap, double scale,
                     int32_t* kept_idx, uint16_t* K_kept, uint16_t* V_kept,
                     double* O_c, double* LSE_c, uint16_t* C_q,
-                    double* vote_out, double* pooled_out, double* row_lse_out) {
+                    double* vote_out, double* pooled_out, double* row_lse_out,
+                    int64_t calib_size, int32_t* calib_idx) {
     if (Hq % Hkv != 0 || n_cal < 1 || n_cal > W || pool < 1 || pool % 2 == 0) return -1;
     int keep_all = budget >= L;
     if (!keep_all && (budget <= W || L < W)) return -1;
@@ -229,6 +246,8 @@ int oracle_compress(const uint16_t* Q_obs, const uint16_t* K, const uint16_t* V,
         const uint16_t* Vu = V + (int64_t)u * L * D;
         const uint16_t* Qu = Q_obs + ((int64_t)b * Hq + (int64_t)h * G) * W * D;
         int32_t* kept = kept_idx + (int64_t)u * n_kept;
+        int32_t* cset = NULL;
+        int64_t m = 0;
         if (keep_all) {
             for (int64_t t = 0; t < L; ++t) kept[t] = (int32_t)t;
         } else {
@@ -239,6 +258,18 @@ int oracle_compress(const uint16_t* Q_obs, const uint16_t* K, const uint16_t* V,
             oracle_pool(vote, n_cand, pool, pooled);
             oracle_topk(pooled, n_cand, k_sel, kept);
             for (int j = 0; j < W; ++j) kept[k_sel + j] = (int32_t)(n_cand + j);
+            if (calib_size >= 0) {
+                /* the next m candidates in the same order: rank the candidates again with the
+                 * selected ones pushed below every vote (votes are non-negative) */
+                m = calib_size < n_cand - k_sel ? calib_size : n_cand - k_sel;
+                double* rest = (double*)malloc((size_t)n_cand * sizeof(double));
+                memcpy(rest, pooled, (size_t)n_cand * sizeof(double));
+                for (int64_t i = 0; i < k_sel; ++i) rest[kept[i]] = -1.0;
+                cset = (int32_t*)malloc((size_t)(m > 0 ? m : 1) * sizeof(int32_t));
+                oracle_topk(rest, n_cand, m, cset);
+                if (calib_idx) memcpy(calib_idx + (int64_t)u * m, cset, (size_t)m * sizeof(int32_t));
+                free(rest);
+            }
             if (vote_out) memcpy(vote_out + (int64_t)u * n_cand, vote, (size_t)n_cand * sizeof(double));
             if (pooled_out) memcpy(pooled_out + (int64_t)u * n_cand, pooled, (size_t)n_cand * sizeof(double));
             if (row_lse_out)
@@ -246,11 +277,12 @@ int oracle_compress(const uint16_t* Q_obs, const uint16_t* K, const uint16_t* V,
                        (size_t)G * W * sizeof(double));
             free(vote); free(pooled); free(row_lse);
         }
-        unit_calibrate(Qu, Ku, Vu, kept, n_kept, G, W, L, D, n_cal, cap, scale,
+        unit_calibrate(Qu, Ku, Vu, kept, n_kept, cset, m, G, W, L, D, n_cal, cap, scale,
                        K_kept + (int64_t)u * cap * D, V_kept + (int64_t)u * cap * D,
                        O_c + ((int64_t)b * Hq + (int64_t)h * G) * n_cal * D,
                        LSE_c + ((int64_t)b * Hq + (int64_t)h * G) * n_cal,
                        C_q + ((int64_t)b * Hq + (int64_t)h * G) * n_cal * D);
+        free(cset);
     }
     return 0;
 }
@@ -270,7 +302,7 @@ int oracle_calibrate_given_indices(const uint16_t* Q_obs, const uint16_t* K, con
         int b = u / Hkv, h = u % Hkv;
         int64_t qoff = (int64_t)b * Hq + (int64_t)h * G;
         unit_calibrate(Q_obs + qoff * W * D, K + (int64_t)u * L * D, V + (int64_t)u * L * D,
-                       kept_idx + (int64_t)u * n_kept, n_kept, G, W, L, D, n_cal, cap, scale,
+                       kept_idx + (int64_t)u * n_kept, n_kept, NULL, 0, G, W, L, D, n_cal, cap, scale,
                        K_kept + (int64_t)u * cap * D, V_kept + (int64_t)u * cap * D,
                        O_c + qoff * n_cal * D, LSE_c + qoff * n_cal, C_q + qoff * n_cal * D);
     }

@@ -86,8 +86,11 @@ def topk(score, k):
     return out
 
 
-def compress(Q_obs, K, V, *, window, pool, budget, n_cal=1, cap=None, scale=None):
-    """Oracle compress-and-calibrate.  Q_obs [B,Hq,W,D], K,V [B,Hkv,L,D] bf16 bits."""
+def compress(Q_obs, K, V, *, window, pool, budget, n_cal=1, cap=None, scale=None, calib_size=None):
+    """Oracle compress-and-calibrate.  Q_obs [B,Hq,W,D], K,V [B,Hkv,L,D] bf16 bits.
+    calib_size: None = every evicted token is calibrated (Algorithm 1 as printed); m >= 0 = only the
+    m evicted tokens of highest pooled vote (the "calibration size" of the paper's Section 4.4),
+    whose ascending indices are returned as calib_idx [B,Hkv,min(m, number evicted)]."""
     Q_obs, K, V = _u16(Q_obs), _u16(K), _u16(V)
     B, Hq, W, D = Q_obs.shape
     _, Hkv, L, _ = K.shape
@@ -105,14 +108,18 @@ def compress(Q_obs, K, V, *, window, pool, budget, n_cal=1, cap=None, scale=None
         vote=np.zeros((B, Hkv, n_cand), dtype=np.float64),
         pooled=np.zeros((B, Hkv, n_cand), dtype=np.float64),
         row_lse=np.zeros((B, Hq, W), dtype=np.float64),
-        n_kept=n_kept, cap=cap,
+        n_kept=n_kept, cap=cap, calib_idx=None,
     )
+    m = -1
+    if calib_size is not None and budget < L:
+        m = min(int(calib_size), n_cand - (budget - W))
+        r.calib_idx = np.zeros((B, Hkv, m), dtype=np.int32)
     rc = _load().oracle_compress(
         _p(Q_obs), _p(K), _p(V), C.c_int(B), C.c_int(Hq), C.c_int(Hkv), C.c_int64(L), C.c_int(D),
         C.c_int(W), C.c_int(pool), C.c_int64(budget), C.c_int(n_cal), C.c_int64(cap),
         C.c_double(scale or default_scale(D)),
         _p(r.kept_idx), _p(r.K_kept), _p(r.V_kept), _p(r.O_c), _p(r.LSE_c), _p(r.C_q),
-        _p(r.vote), _p(r.pooled), _p(r.row_lse))
+        _p(r.vote), _p(r.pooled), _p(r.row_lse), C.c_int64(m), _p(r.calib_idx))
     if rc != 0:
         raise ValueError("oracle_compress: arguments outside the method's definition")
     return r

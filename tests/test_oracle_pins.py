@@ -230,6 +230,47 @@ def test_single_evicted_token_closed_form():
         np.testing.assert_allclose(r.O_c[0, h, 0], f64(V[0, h, t]), atol=1e-15)
 
 
+def test_calibration_size_takes_the_next_most_important_evicted_tokens():
+    """Section 4.4's calibration size m: the calibrated (and offloaded) set is the m evicted candidates
+    of highest pooled vote, i.e. ranks k_sel .. k_sel+m-1 of ONE stable ordering; the term is plain
+    attention over exactly those rows.  m >= |E| is Algorithm 1 as printed, m = 0 no calibration."""
+    cfg = wl.small_config(L=150, window=8, budget=28, n_heavy=12)
+    Q, (K, V) = wl.gen_q_obs(cfg), wl.gen_kv(cfg)
+    full = oracle.compress(Q, K, V, window=8, pool=5, budget=28, n_cal=2)
+    n_cand, k_sel = 150 - 8, 28 - 8
+    n_e = n_cand - k_sel
+    for m in (0, 1, 7, n_e, n_e + 50):
+        r = oracle.compress(Q, K, V, window=8, pool=5, budget=28, n_cal=2, calib_size=m)
+        np.testing.assert_array_equal(r.kept_idx, full.kept_idx)        # the selection does not depend on m
+        np.testing.assert_array_equal(r.K_kept, full.K_kept)
+        m_eff = min(m, n_e)
+        assert r.calib_idx.shape == (1, cfg.Hkv, m_eff)
+        for h in range(cfg.Hkv):
+            # one stable ordering of the candidates by (pooled desc, index asc), from numpy
+            order = np.argsort(-full.pooled[0, h], kind="stable")
+            np.testing.assert_array_equal(np.sort(order[:k_sel]), full.kept_idx[0, h, :k_sel])
+            want = np.sort(order[k_sel:k_sel + m_eff])
+            np.testing.assert_array_equal(r.calib_idx[0, h], want)
+            for g in range(cfg.G):
+                hq = h * cfg.G + g
+                for c in range(2):
+                    if m_eff == 0:
+                        assert np.isneginf(r.LSE_c[0, hq, c]) and np.all(r.O_c[0, hq, c] == 0)
+                        continue
+                    q = Q[0, hq, 8 - 2 + c][None]
+                    o, l = np_attention(q, K[0, h][want], V[0, h][want], 1 / math.sqrt(128))
+                    np.testing.assert_allclose(r.O_c[0, hq, c], o[0], atol=1e-13)
+                    np.testing.assert_allclose(r.LSE_c[0, hq, c], l[0], atol=1e-12)
+        if m >= n_e:
+            np.testing.assert_array_equal(r.O_c, full.O_c)
+            np.testing.assert_array_equal(r.LSE_c, full.LSE_c)
+    # ties: with a constant vote vector the order is the index order
+    Kc = np.zeros_like(K)
+    rc = oracle.compress(Q, Kc, V, window=8, pool=1, budget=28, n_cal=1, calib_size=5)
+    np.testing.assert_array_equal(rc.kept_idx[0, 0, :k_sel], np.arange(k_sel))
+    np.testing.assert_array_equal(rc.calib_idx[0, 0], np.arange(k_sel, k_sel + 5))
+
+
 def test_calibrate_given_indices_agrees_and_uses_supplied_set():
     cfg = wl.small_config(L=100, window=8, budget=20)
     Q, (K, V) = wl.gen_q_obs(cfg), wl.gen_kv(cfg)
