@@ -67,6 +67,12 @@ typedef struct calidrop_params {
   float   softmax_scale;        /* 0 => 1/sqrt(D)                                              */
   float   theta1, theta2;       /* decode: rho < theta1 raises needs_recompute; rho > theta2   */
                                 /* applies the calibration; theta2 <= -1 always applies it     */
+  int32_t calib_size;           /* compress: the "calibration size" of the paper's Section 4.4 */
+                                /* (Efficiency Optimization): 0 = every evicted row takes part */
+                                /* in the calibration (Algorithm 1 as printed); m > 0 = only   */
+                                /* the m evicted rows of highest pooled vote (ties: lowest     */
+                                /* index), the rest are dropped for good; -1 = none (O_c = 0,  */
+                                /* LSE_c = -inf).  A zero-initialised struct gives 0.          */
 } calidrop_params;
 
 /*
@@ -85,7 +91,9 @@ size_t calidrop_compress_workspace_bytes(const calidrop_params* p);
  *   pooled[t] = (1/pool) sum_{|d| <= pool/2} vote[t+d]   (zero padding, constant divisor);
  *   kept      = the budget-W candidates with the largest pooled[t] (ties: lowest index),
  *               in ascending order, followed by the window rows L-W .. L-1;
- *   E         = [0, L-W) \ kept, the evicted rows;
+ *   E         = [0, L-W) \ kept, the evicted rows; with calib_size = m > 0 only the m of them
+ *               with the largest pooled[t] (the candidates of rank budget-W .. budget-W+m-1 in the
+ *               same order), with calib_size = -1 none;
  *   for c < n_cal, q_c = Q_obs[b, h*G+g, W-n_cal+c]:
  *     LSE_c[c] = log sum_{t in E} exp(q_c.k_t * scale),  O_c[c] = Att(q_c, K_E, V_E),
  *     C_q[c] = q_c.                                       (lines 5-8 of Algorithm 1)
@@ -146,7 +154,12 @@ int calidrop_calibrate(const calidrop_params* p,
  *             kept_idx does not list, ascending
  *   K_evict, V_evict out [B, Hkv, n_evict, D] bf16: bit copies of those rows
  *   workspace as for calidrop_compress (its kept bitmap is rebuilt from kept_idx)
- * INVALID_ARG also when budget >= L (nothing is evicted).
+ * With calib_size = m > 0 the rows are the m calibrated ones (n_evict = min(m, L - budget)): which
+ * they are depends on the votes, so `workspace` must then be the workspace of the calidrop_compress
+ * call that wrote kept_idx (same parameters), not used for anything else in between; that call
+ * leaves the list there.
+ * INVALID_ARG also when budget >= L (nothing is evicted) or calib_size = -1 (nothing is kept for
+ * calibration).
  */
 int calidrop_gather_evicted(const calidrop_params* p, const void* K, const void* V, const int32_t* kept_idx,
                             int32_t* evict_idx, void* K_evict, void* V_evict,

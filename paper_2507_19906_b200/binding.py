@@ -36,7 +36,8 @@ EXPORTS = [
 class Params(C.Structure):
     _fields_ = [(n, C.c_int32) for n in
                 ("B", "Hq", "Hkv", "D", "L", "window", "pool", "budget", "n_cal", "cap")] + \
-               [("softmax_scale", C.c_float), ("theta1", C.c_float), ("theta2", C.c_float)]
+               [("softmax_scale", C.c_float), ("theta1", C.c_float), ("theta2", C.c_float),
+                ("calib_size", C.c_int32)]
 
 
 class CompressLayout(C.Structure):
@@ -104,9 +105,10 @@ def load():
 
 
 def make_params(*, B, Hq, Hkv, L=1, window=1, pool=1, budget=1, n_cal=1, cap, D=128,
-                softmax_scale=0.0, theta1=0.7, theta2=0.85) -> Params:
+                softmax_scale=0.0, theta1=0.7, theta2=0.85, calib_size=0) -> Params:
     return Params(B=B, Hq=Hq, Hkv=Hkv, D=D, L=L, window=window, pool=pool, budget=budget,
-                  n_cal=n_cal, cap=cap, softmax_scale=softmax_scale, theta1=theta1, theta2=theta2)
+                  n_cal=n_cal, cap=cap, softmax_scale=softmax_scale, theta1=theta1, theta2=theta2,
+                  calib_size=calib_size)
 
 
 def _ptr(t):

@@ -46,6 +46,7 @@ int check_compress(const calidrop_params* p) {
   if (p->budget < p->L && (p->budget <= p->window || p->L < p->window)) return CALIDROP_INVALID_ARG;
   const int n_kept = p->budget < p->L ? p->budget : p->L;
   if (p->cap < n_kept) return CALIDROP_INVALID_ARG;
+  if (p->calib_size < -1) return CALIDROP_INVALID_ARG;
   return CALIDROP_OK;
 }
 
@@ -65,6 +66,10 @@ CompressGeom make_geom(const calidrop_params* p) {
   g.units = p->B * p->Hkv;
   g.bitmap_words = (p->L + 31) / 32;
   g.scale2 = scale2_of(p);
+  // calibration size: how many of the n_cand - k_sel evicted candidates are calibrated
+  const int n_evict = g.keep_all ? 0 : g.n_cand - g.k_sel;
+  g.sized = !g.keep_all && p->calib_size != 0;
+  g.n_calib = p->calib_size == 0 ? n_evict : (p->calib_size < 0 ? 0 : (p->calib_size < n_evict ? p->calib_size : n_evict));
   return g;
 }
 
@@ -77,6 +82,8 @@ CompressWs make_ws(const CompressGeom& g) {
   w.pooled = off;  off = align_up(off + (size_t)g.units * n_cand * 4, 256);
   w.row_lse = off; off = align_up(off + (size_t)g.B * g.Hq * g.W * 4, 256);
   w.bitmap = off;  off = align_up(off + (size_t)g.units * g.bitmap_words * 4, 256);
+  w.bitmap2 = off; off = align_up(off + (g.sized ? (size_t)g.units * g.bitmap_words * 4 : 0), 256);
+  w.calib_mask = g.sized ? w.bitmap2 : w.bitmap;
   w.n_tiles = (g.L + 127) / 128;
   w.stat_slots = w.n_tiles > 320 ? w.n_tiles : 320;
   w.stat_part = off; off = align_up(off + (size_t)g.B * g.Hq * g.W * w.stat_slots * 8, 256);
@@ -236,6 +243,8 @@ int calidrop_compress(const calidrop_params* p, const void* Q_obs, const void* K
   const CompressWs ws = make_ws(g);
   if (workspace_bytes < ws.total) return CALIDROP_WORKSPACE_TOO_SMALL;
   if (!device_supported()) return CALIDROP_UNSUPPORTED;
+  // a sized calibration takes its second threshold in the cluster selection kernel
+  if (g.sized && g.n_calib > 0 && !select_cluster_supported(g)) return CALIDROP_UNSUPPORTED;
 
   cudaStream_t st = (cudaStream_t)stream;
   char* wsp = (char*)workspace;
@@ -259,9 +268,12 @@ int calidrop_compress(const calidrop_params* p, const void* Q_obs, const void* K
   if (e != cudaSuccess) return cuda_fail(e);
   e = launch_gather(g, K, V, kept_idx, K_kept, V_kept, st);
   if (e != cudaSuccess) return cuda_fail(e);
-  e = (tc_path && calib_tc_supported(g))
-          ? launch_calib_tc(g, ws, Q_obs, K, V, row_lse, wsp, O_c, LSE_c, C_q, st)
-          : launch_calib_direct(g, ws, Q_obs, K, V, wsp, O_c, LSE_c, C_q, st);
+  if (g.sized && g.n_calib == 0)
+    e = launch_calib_none(g, Q_obs, O_c, LSE_c, C_q, st);
+  else
+    e = (tc_path && calib_tc_supported(g))
+            ? launch_calib_tc(g, ws, Q_obs, K, V, row_lse, wsp, O_c, LSE_c, C_q, st)
+            : launch_calib_direct(g, ws, Q_obs, K, V, wsp, O_c, LSE_c, C_q, st);
   if (e != cudaSuccess) return cuda_fail(e);
   return CALIDROP_OK;
 }
@@ -276,6 +288,7 @@ int calidrop_calibrate(const calidrop_params* p, const void* Q_obs, const void* 
     if (!q || !aligned16(q)) return CALIDROP_INVALID_ARG;
   if (lse_obs && !aligned16(lse_obs)) return CALIDROP_INVALID_ARG;
   if (reinterpret_cast<uintptr_t>(workspace) & 255u) return CALIDROP_INVALID_ARG;
+  if (p->calib_size != 0) return CALIDROP_INVALID_ARG;   // no votes here to rank the evicted rows by
   const CompressGeom g = make_geom(p);
   const CompressWs ws = make_ws(g);
   if (workspace_bytes < ws.total) return CALIDROP_WORKSPACE_TOO_SMALL;
@@ -315,17 +328,19 @@ int calidrop_gather_evicted(const calidrop_params* p, const void* K, const void*
     if (!q || !aligned16(q)) return CALIDROP_INVALID_ARG;
   if (reinterpret_cast<uintptr_t>(workspace) & 255u) return CALIDROP_INVALID_ARG;
   const CompressGeom g = make_geom(p);
-  if (g.keep_all) return CALIDROP_INVALID_ARG;  // nothing is evicted
+  if (g.keep_all || g.n_calib == 0) return CALIDROP_INVALID_ARG;  // nothing is evicted / kept for calibration
   const CompressWs ws = make_ws(g);
   if (workspace_bytes < ws.total) return CALIDROP_WORKSPACE_TOO_SMALL;
   if (!device_supported()) return CALIDROP_UNSUPPORTED;
   cudaStream_t st = (cudaStream_t)stream;
   char* wsp = (char*)workspace;
-  cudaError_t e = launch_bitmap_from_indices(g, ws, wsp, kept_idx, st);
+  cudaError_t e = cudaSuccess;
+  // sized calibration: the mask of the calibrated rows is the one calidrop_compress left in this workspace
+  if (!g.sized) e = launch_bitmap_from_indices(g, ws, wsp, kept_idx, st);
   if (e != cudaSuccess) return cuda_fail(e);
   e = launch_evicted_indices(g, ws, wsp, evict_idx, st);
   if (e != cudaSuccess) return cuda_fail(e);
-  const int n_evict = g.L - g.n_kept;
+  const int n_evict = g.n_calib;
   e = launch_gather_rows(g, K, V, evict_idx, n_evict, n_evict, K_evict, V_evict, st);
   return e == cudaSuccess ? CALIDROP_OK : cuda_fail(e);
 }

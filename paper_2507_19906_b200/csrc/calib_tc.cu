@@ -492,7 +492,7 @@ cudaError_t launch_calib_tc(const CompressGeom& g, const CompressWs& ws, const v
   a.bitmap_words = g.bitmap_words;
   a.scale2 = g.scale2;
   a.row_lse = row_lse;
-  a.bitmap = (const uint32_t*)(wsp + ws.bitmap);
+  a.bitmap = (const uint32_t*)(wsp + ws.calib_mask);
   a.o_part = (float*)(wsp + ws.calib_o);
   a.l_part = (float*)(wsp + ws.calib_l);
   a.status = (unsigned*)(wsp + ws.status);

@@ -229,7 +229,7 @@ cudaError_t launch_calib_direct(const CompressGeom& g, const CompressWs& ws, con
   const int total = g.B * g.Hq * g.n_cal;
   calib_direct_kernel<<<(total + 3) / 4, 128, 0, st>>>(
       (const __nv_bfloat16*)Q_obs, (const __nv_bfloat16*)K, (const __nv_bfloat16*)V,
-      (const uint32_t*)(wsp + ws.bitmap), O_c, LSE_c, (__nv_bfloat16*)C_q, g.B, g.Hq, g.Hkv, g.G, g.W,
+      (const uint32_t*)(wsp + ws.calib_mask), O_c, LSE_c, (__nv_bfloat16*)C_q, g.B, g.Hq, g.Hkv, g.G, g.W,
       g.L, g.n_cand, g.n_cal, g.bitmap_words, g.scale2);
   count_launch(1);
   return cudaGetLastError();

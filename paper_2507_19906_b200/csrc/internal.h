@@ -18,11 +18,16 @@ struct CompressGeom {
   int units;    // B * Hkv
   int bitmap_words;  // ceil(L / 32) per unit
   float scale2;      // softmax scale * log2(e)
+  // calibration size: n_calib of the evicted candidates take part in the calibration (all of them
+  // unless `sized`); the masked passes then read the bitmap at ws.calib_mask
+  int sized, n_calib;
 };
 
 // Workspace carving of compress (byte offsets, all 256-byte aligned).
 struct CompressWs {
   size_t vote, vote2, pooled, row_lse, bitmap, stat_part, status, calib_o, calib_l, total;
+  size_t bitmap2;     // sized calibration: bit set = the row is NOT one of the calibrated evicted rows
+  size_t calib_mask;  // the bitmap the calibration passes mask with: bitmap, or bitmap2 when sized
   int n_tiles;     // 128-key tiles per unit (scalar statistics pass: one partial per tile)
   int stat_slots;  // (max, sum) partial slots per observation row in stat_part
 };
@@ -120,6 +125,9 @@ cudaError_t launch_decode(const DecodeArgsT<kDecodeMaxLayers>& a, cudaStream_t s
 cudaError_t launch_recalibrate(const DecodeArgsT<1>& a, cudaStream_t st);
 cudaError_t launch_evicted_indices(const CompressGeom& g, const CompressWs& ws, char* wsp, int32_t* evict_idx,
                                    cudaStream_t st);
+// Calibration size -1: no row is calibrated (O_c = 0, LSE_c = -inf, C_q = the calibration queries).
+cudaError_t launch_calib_none(const CompressGeom& g, const void* Q_obs, float* O_c, float* LSE_c, void* C_q,
+                              cudaStream_t st);
 
 void count_launch(int n = 1);
 

@@ -260,8 +260,31 @@ evicted_indices_kernel(const uint32_t* __restrict__ bitmap, int32_t* __restrict_
 
 cudaError_t launch_evicted_indices(const CompressGeom& g, const CompressWs& ws, char* wsp, int32_t* evict_idx,
                                    cudaStream_t st) {
-  evicted_indices_kernel<<<g.units, kSelThreads, 0, st>>>((const uint32_t*)(wsp + ws.bitmap), evict_idx, g.n_cand,
-                                                          g.L - g.n_kept, g.bitmap_words);
+  // the zero bits below n_cand of the kept bitmap, or of the calibration mask when the calibration is sized
+  evicted_indices_kernel<<<g.units, kSelThreads, 0, st>>>((const uint32_t*)(wsp + ws.calib_mask), evict_idx, g.n_cand,
+                                                          g.n_calib, g.bitmap_words);
+  count_launch(1);
+  return cudaGetLastError();
+}
+
+// No calibrated rows: zeros, -inf and the calibration queries.  One warp per (b, hq, c).
+__global__ void __launch_bounds__(128)
+calib_none_kernel(const __nv_bfloat16* __restrict__ Q_obs, float* __restrict__ O_c, float* __restrict__ LSE_c,
+                  __nv_bfloat16* __restrict__ C_q, int rows, int W, int n_cal) {
+  const int lane = threadIdx.x & 31, row = blockIdx.x * 4 + (threadIdx.x >> 5);
+  if (row >= rows) return;
+  const int c = row % n_cal, bhq = row / n_cal;
+  reinterpret_cast<float4*>(O_c + (size_t)row * kD)[lane] = make_float4(0.f, 0.f, 0.f, 0.f);
+  if (lane == 0) LSE_c[row] = -INFINITY;
+  reinterpret_cast<uint2*>(C_q + (size_t)row * kD)[lane] =
+      reinterpret_cast<const uint2*>(Q_obs + ((size_t)bhq * W + (W - n_cal + c)) * kD)[lane];
+}
+
+cudaError_t launch_calib_none(const CompressGeom& g, const void* Q_obs, float* O_c, float* LSE_c, void* C_q,
+                              cudaStream_t st) {
+  const int rows = g.B * g.Hq * g.n_cal;
+  calib_none_kernel<<<(rows + 3) / 4, 128, 0, st>>>((const __nv_bfloat16*)Q_obs, O_c, LSE_c, (__nv_bfloat16*)C_q, rows,
+                                                   g.W, g.n_cal);
   count_launch(1);
   return cudaGetLastError();
 }

@@ -29,12 +29,13 @@ template <int ROWS>
 __global__ void __cluster_dims__(kClu, 1, 1) __launch_bounds__(kT)
 pool_select_cluster_kernel(const float* __restrict__ vote, float* __restrict__ pooled,
                            uint32_t* __restrict__ bitmap, int32_t* __restrict__ kept_idx, int n_cand, int L,
-                           int pool, int k_sel, int n_kept, int bitmap_words) {
+                           int pool, int k_sel, int n_kept, int bitmap_words, uint32_t* __restrict__ mask2,
+                           int n_calib) {
   __shared__ unsigned hist[kW][256];
   __shared__ unsigned mine[2][256];   // this CTA's histogram of the current pass (double-buffered)
   __shared__ unsigned total[256];
   __shared__ unsigned sel_bin, sel_k;
-  __shared__ unsigned cnt[2];         // this CTA's counts of keys > T and == T
+  __shared__ unsigned cnt[2][2];      // this CTA's counts of keys > T and == T, for the two thresholds
   __shared__ unsigned wsum[ROWS * kW][2];
 
   cg::cluster_group cluster = cg::this_cluster();
@@ -68,103 +69,123 @@ pool_select_cluster_kernel(const float* __restrict__ vote, float* __restrict__ p
   }
 
   // 2. radix select, most significant byte first; the histograms of the eight CTAs are summed
-  // through distributed shared memory
-  unsigned prefix = 0, k = (unsigned)k_sel;
-  for (int pass = 0; pass < 4; ++pass) {
-    const int shift = 24 - 8 * pass;
-    for (int i = tid; i < kW * 256; i += kT) (&hist[0][0])[i] = 0;
-    __syncthreads();
+  // through distributed shared memory.  Returns the bit pattern T of the kk-th largest pooled vote
+  // and how many candidates equal to T are still taken (those at the lowest positions).
+  auto radix_select = [&](unsigned kk, unsigned& T_out, unsigned& need_out) {
+    unsigned prefix = 0, k = kk;
+    for (int pass = 0; pass < 4; ++pass) {
+      const int shift = 24 - 8 * pass;
+      for (int i = tid; i < kW * 256; i += kT) (&hist[0][0])[i] = 0;
+      __syncthreads();
+#pragma unroll
+      for (int i = 0; i < ROWS; ++i) {
+        const int t = rank * chunk + i * kT + tid;
+        const bool in = t < n_cand && ((pass == 0) || ((key[i] >> (shift + 8)) == prefix));
+        if (in) atomicAdd(&hist[warp][(key[i] >> shift) & 255u], 1u);
+      }
+      __syncthreads();
+      if (tid < 256) {
+        unsigned s = 0;
+#pragma unroll 8
+        for (int w = 0; w < kW; ++w) s += hist[w][tid];
+        mine[pass & 1][tid] = s;
+      }
+      cluster.sync();
+      if (tid < 256) {
+        unsigned s = 0;
+        for (int r = 0; r < kClu; ++r) s += cluster.map_shared_rank(&mine[pass & 1][0], r)[tid];
+        total[tid] = s;
+      }
+      __syncthreads();
+      if (warp == 0) {
+        // lane 0 owns the 8 highest bins; walk bins downwards until k candidates are covered
+        const int base = 255 - 8 * lane;
+        unsigned c[8], s = 0;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) { c[j] = total[base - j]; s += c[j]; }
+        unsigned incl = s;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+          unsigned n = __shfl_up_sync(0xffffffffu, incl, o);
+          if (lane >= o) incl += n;
+        }
+        const unsigned ball = __ballot_sync(0xffffffffu, incl >= k);
+        const int target = __ffs(ball) - 1;  // always found: the candidates number at least k
+        if (lane == target) {
+          unsigned run = incl - s;
+#pragma unroll
+          for (int j = 0; j < 8; ++j) {
+            if (run + c[j] >= k) { sel_bin = (unsigned)(base - j); sel_k = k - run; break; }
+            run += c[j];
+          }
+        }
+      }
+      __syncthreads();
+      prefix = (prefix << 8) | sel_bin;
+      k = sel_k;
+    }
+    // (the two passes that still use mine[] of this call lie at least two cluster barriers behind
+    // when the next call writes them again)
+    T_out = prefix;
+    need_out = k;
+  };
+  unsigned T, need_eq;
+  radix_select((unsigned)k_sel, T, need_eq);
+
+  // 3. ordered compaction.  Per (row, warp): how many keys are above T / equal to T; the exclusive
+  // scan of those counts in index order, over the cluster, gives every key the number of keys
+  // above / equal to the threshold that precede it.
+  unsigned gt_mask[ROWS], eq_mask[ROWS];
+  unsigned before_gt = 0, before_eq = 0;  // keys of the lower-ranked CTAs
+  auto scan_threshold = [&](unsigned Tx, int slot) {
 #pragma unroll
     for (int i = 0; i < ROWS; ++i) {
       const int t = rank * chunk + i * kT + tid;
-      const bool in = t < n_cand && ((pass == 0) || ((key[i] >> (shift + 8)) == prefix));
-      if (in) atomicAdd(&hist[warp][(key[i] >> shift) & 255u], 1u);
+      const bool valid = t < n_cand;
+      gt_mask[i] = __ballot_sync(0xffffffffu, valid && key[i] > Tx);
+      eq_mask[i] = __ballot_sync(0xffffffffu, valid && key[i] == Tx);
+      if (lane == 0) {
+        wsum[i * kW + warp][0] = __popc(gt_mask[i]);
+        wsum[i * kW + warp][1] = __popc(eq_mask[i]);
+      }
     }
     __syncthreads();
-    if (tid < 256) {
-      unsigned s = 0;
-#pragma unroll 8
-      for (int w = 0; w < kW; ++w) s += hist[w][tid];
-      mine[pass & 1][tid] = s;
+    // exclusive scan of the ROWS * 32 warp counts in index order (row-major), by the first warp
+    if (warp == 0) {
+      unsigned run_gt = 0, run_eq = 0;
+      for (int base = 0; base < ROWS * kW; base += 32) {
+        const unsigned g0 = wsum[base + lane][0], e0 = wsum[base + lane][1];
+        unsigned ig = g0, ie = e0;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+          const unsigned a = __shfl_up_sync(0xffffffffu, ig, o);
+          const unsigned b = __shfl_up_sync(0xffffffffu, ie, o);
+          if (lane >= o) { ig += a; ie += b; }
+        }
+        wsum[base + lane][0] = run_gt + ig - g0;
+        wsum[base + lane][1] = run_eq + ie - e0;
+        run_gt += __shfl_sync(0xffffffffu, ig, 31);
+        run_eq += __shfl_sync(0xffffffffu, ie, 31);
+      }
+      if (lane == 0) { cnt[slot][0] = run_gt; cnt[slot][1] = run_eq; }
     }
     cluster.sync();
-    if (tid < 256) {
-      unsigned s = 0;
-      for (int r = 0; r < kClu; ++r) s += cluster.map_shared_rank(&mine[pass & 1][0], r)[tid];
-      total[tid] = s;
+    before_gt = before_eq = 0;
+    for (int r = 0; r < rank; ++r) {
+      const unsigned* c = cluster.map_shared_rank(&cnt[slot][0], r);
+      before_gt += c[0];
+      before_eq += c[1];
     }
-    __syncthreads();
-    if (warp == 0) {
-      // lane 0 owns the 8 highest bins; walk bins downwards until k candidates are covered
-      const int base = 255 - 8 * lane;
-      unsigned c[8], s = 0;
-#pragma unroll
-      for (int j = 0; j < 8; ++j) { c[j] = total[base - j]; s += c[j]; }
-      unsigned incl = s;
-#pragma unroll
-      for (int o = 1; o < 32; o <<= 1) {
-        unsigned n = __shfl_up_sync(0xffffffffu, incl, o);
-        if (lane >= o) incl += n;
-      }
-      const unsigned ball = __ballot_sync(0xffffffffu, incl >= k);
-      const int target = __ffs(ball) - 1;  // always found: the candidates number at least k
-      if (lane == target) {
-        unsigned run = incl - s;
-#pragma unroll
-        for (int j = 0; j < 8; ++j) {
-          if (run + c[j] >= k) { sel_bin = (unsigned)(base - j); sel_k = k - run; break; }
-          run += c[j];
-        }
-      }
-    }
-    __syncthreads();
-    prefix = (prefix << 8) | sel_bin;
-    k = sel_k;
-  }
-  const unsigned T = prefix;   // bit pattern of the k-th largest pooled vote
-  const unsigned need_eq = k;  // how many candidates equal to T are taken (lowest positions)
-
-  // 3. ordered compaction.  Per (row, warp): how many keys are above T / equal to T.
-  unsigned gt_mask[ROWS], eq_mask[ROWS];
-#pragma unroll
-  for (int i = 0; i < ROWS; ++i) {
-    const int t = rank * chunk + i * kT + tid;
-    const bool valid = t < n_cand;
-    gt_mask[i] = __ballot_sync(0xffffffffu, valid && key[i] > T);
-    eq_mask[i] = __ballot_sync(0xffffffffu, valid && key[i] == T);
-    if (lane == 0) {
-      wsum[i * kW + warp][0] = __popc(gt_mask[i]);
-      wsum[i * kW + warp][1] = __popc(eq_mask[i]);
-    }
-  }
-  __syncthreads();
-  // exclusive scan of the ROWS * 32 warp counts in index order (row-major), by the first warp
-  if (warp == 0) {
-    unsigned run_gt = 0, run_eq = 0;
-    for (int base = 0; base < ROWS * kW; base += 32) {
-      const unsigned g0 = wsum[base + lane][0], e0 = wsum[base + lane][1];
-      unsigned ig = g0, ie = e0;
-#pragma unroll
-      for (int o = 1; o < 32; o <<= 1) {
-        const unsigned a = __shfl_up_sync(0xffffffffu, ig, o);
-        const unsigned b = __shfl_up_sync(0xffffffffu, ie, o);
-        if (lane >= o) { ig += a; ie += b; }
-      }
-      wsum[base + lane][0] = run_gt + ig - g0;
-      wsum[base + lane][1] = run_eq + ie - e0;
-      run_gt += __shfl_sync(0xffffffffu, ig, 31);
-      run_eq += __shfl_sync(0xffffffffu, ie, 31);
-    }
-    if (lane == 0) { cnt[0] = run_gt; cnt[1] = run_eq; }
-  }
-  cluster.sync();
-  unsigned before_gt = 0, before_eq = 0;  // keys of the lower-ranked CTAs
-  for (int r = 0; r < rank; ++r) {
-    const unsigned* c = cluster.map_shared_rank(&cnt[0], r);
-    before_gt += c[0];
-    before_eq += c[1];
-  }
+  };
+  // is key (row i, this thread) among the first `need` keys equal to Tx or above Tx ?
   const unsigned lt = (1u << lane) - 1u;
+  auto taken = [&](int i, unsigned Tx, unsigned need) {
+    const unsigned eq_before = before_eq + wsum[i * kW + warp][1] + __popc(eq_mask[i] & lt);
+    return key[i] > Tx || (key[i] == Tx && eq_before < need);
+  };
+
+  scan_threshold(T, 0);
+  unsigned take_bits = 0;   // bit i: this thread's key of row i was selected
 #pragma unroll
   for (int i = 0; i < ROWS; ++i) {
     const int t = rank * chunk + i * kT + tid;
@@ -172,12 +193,12 @@ pool_select_cluster_kernel(const float* __restrict__ vote, float* __restrict__ p
     const unsigned eq_before = before_eq + wsum[i * kW + warp][1] + __popc(eq_mask[i] & lt);
     bool take = false;
     if (t < n_cand) {
-      if (key[i] > T) take = true;
-      else if (key[i] == T) take = eq_before < need_eq;
+      take = taken(i, T, need_eq);
       if (take) kept[gt_before + min(eq_before, need_eq)] = t;
     } else if (t < L) {
       take = true;  // observation-window rows are always kept
     }
+    take_bits |= (take ? 1u : 0u) << i;
     const unsigned word = __ballot_sync(0xffffffffu, take);
     const int t0 = rank * chunk + i * kT + warp * 32;
     if (lane == 0 && t0 < L) bm[t0 >> 5] = word;
@@ -185,6 +206,24 @@ pool_select_cluster_kernel(const float* __restrict__ vote, float* __restrict__ p
   // the window rows close the kept list
   if (rank == 0)
     for (int j = tid; j < L - n_cand; j += kT) kept[k_sel + j] = n_cand + j;
+
+  // 4. calibration size: the next n_calib candidates in the same order, i.e. those among the first
+  // k_sel + n_calib that were not selected.  mask2: bit set = the row is NOT one of them.
+  if (mask2) {
+    uint32_t* bm2 = mask2 + (size_t)unit * bitmap_words;
+    unsigned T2, need2;
+    __syncthreads();   // wsum and the flags of step 3 have been read by every thread of this CTA
+    radix_select((unsigned)(k_sel + n_calib), T2, need2);
+    scan_threshold(T2, 1);
+#pragma unroll
+    for (int i = 0; i < ROWS; ++i) {
+      const int t = rank * chunk + i * kT + tid;
+      const bool member = t < n_cand && !((take_bits >> i) & 1u) && taken(i, T2, need2);
+      const unsigned word = ~__ballot_sync(0xffffffffu, member);
+      const int t0 = rank * chunk + i * kT + warp * 32;
+      if (lane == 0 && t0 < L) bm2[t0 >> 5] = word;
+    }
+  }
   cluster.sync();  // no CTA leaves while another may still read its shared memory
 }
 
@@ -192,7 +231,8 @@ template <int ROWS>
 void launch_rows(const CompressGeom& g, const CompressWs& ws, char* wsp, int32_t* kept_idx, cudaStream_t st) {
   pool_select_cluster_kernel<ROWS><<<dim3(kClu, g.units), kT, 0, st>>>(
       (const float*)(wsp + ws.vote), (float*)(wsp + ws.pooled), (uint32_t*)(wsp + ws.bitmap), kept_idx, g.n_cand,
-      g.L, g.pool, g.k_sel, g.n_kept, g.bitmap_words);
+      g.L, g.pool, g.k_sel, g.n_kept, g.bitmap_words, (g.sized && g.n_calib > 0) ? (uint32_t*)(wsp + ws.bitmap2) : nullptr,
+      g.n_calib);
 }
 
 }  // namespace

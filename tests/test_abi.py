@@ -55,7 +55,7 @@ def test_size_queries_and_status_strings(lib):
     assert cd.status_string(cd.OK) == "ok"
     assert "workspace" in cd.status_string(cd.WORKSPACE_TOO_SMALL)
     assert cd.calidrop_version() >= 100
-    assert ctypes.sizeof(cd.Params) == 13 * 4
+    assert ctypes.sizeof(cd.Params) == 14 * 4
 
 
 def test_null_arguments_are_rejected_before_any_cuda_call(lib):

@@ -76,6 +76,52 @@ def test_single_cta_selection_for_very_long_prompts(cuda_lib):
     decode_steps_compare(g, ref, q, kn, vn, steps=2)
 
 
+@pytest.mark.parametrize("calib_size", [1, 40, 300, 10 ** 6, -1])
+def test_calibration_size(cuda_lib, calib_size):
+    """Section 4.4's calibration size m: only the m evicted rows of highest pooled vote are calibrated
+    (and offloaded); m >= the number evicted is Algorithm 1 as printed, -1 switches the calibration off."""
+    from paper_2507_19906_b200 import binding as cd
+    B, Hq, Hkv, L, W, pool, budget, n_cal = 2, 8, 2, 1500, 16, 7, 200, 16
+    cfg = wl.small_config(B=B, Hq=Hq, Hkv=Hkv, L=L, window=W, pool=pool, budget=budget, steps=3, n_sink=2, n_heavy=40)
+    Q, K, V = _inputs(cfg)
+    m = None if calib_size == 10 ** 6 else max(calib_size, 0)
+    orc = oracle.compress(Q, K, V, window=W, pool=pool, budget=budget, n_cal=n_cal, cap=budget + 3, calib_size=m)
+    p = cd.make_params(B=B, Hq=Hq, Hkv=Hkv, L=L, window=W, pool=pool, budget=budget, n_cal=n_cal, cap=budget + 3,
+                       calib_size=calib_size)
+    st = cd.alloc_layer_state(p)
+    dQ, dK, dV = to_dev(Q), to_dev(K), to_dev(V)
+    cd.calidrop_compress(p, dQ, dK, dV, None, st.kept_idx, st.K_kept, st.V_kept, st.O_c, st.LSE_c, st.C_q,
+                         st.ws_compress)
+    torch.cuda.synchronize()
+    np.testing.assert_array_equal(st.kept_idx.cpu().numpy(), orc.kept_idx)      # no near-tie in this input
+    np.testing.assert_array_equal(to_bits(st.C_q), orc.C_q)
+    assert_close_lse(st.LSE_c.cpu().numpy(), orc.LSE_c, "LSE_c")
+    assert_close_out(st.O_c.cpu().numpy(), orc.O_c, "O_c")
+    if calib_size == -1:
+        assert np.all(np.isneginf(st.LSE_c.cpu().numpy()))
+        return
+    # the calibrated rows, compacted for offloading: the same list and bit copies of the rows
+    n_e = min(calib_size, L - budget)
+    ev_idx = torch.empty((B, Hkv, n_e), dtype=torch.int32, device="cuda")
+    K_e = torch.empty((B, Hkv, n_e, 128), dtype=torch.bfloat16, device="cuda")
+    V_e = torch.empty_like(K_e)
+    cd.calidrop_gather_evicted(p, dK, dV, st.kept_idx, ev_idx, K_e, V_e, st.ws_compress)
+    torch.cuda.synchronize()
+    want = orc.calib_idx if m is not None else np.stack(
+        [[np.setdiff1d(np.arange(L - W), orc.kept_idx[b, h]) for h in range(Hkv)] for b in range(B)])
+    np.testing.assert_array_equal(ev_idx.cpu().numpy(), want)
+    for b in range(B):
+        for h in range(Hkv):
+            np.testing.assert_array_equal(to_bits(K_e)[b, h], K[b, h][want[b, h]])
+            np.testing.assert_array_equal(to_bits(V_e)[b, h], V[b, h][want[b, h]])
+    # and decode goes on as usual with the smaller calibration term
+    g = type("R", (), {})()
+    g.p, g.st, g.n_kept = p, st, budget
+    ref = orc
+    q, kn, vn = wl.gen_decode_inputs(cfg, Q, steps=3)
+    decode_steps_compare(g, ref, q, kn, vn, steps=3)
+
+
 def test_supplied_row_lse_matches_self_computed(cuda_lib):
     cfg = wl.small_config(B=1, Hq=4, Hkv=2, L=400, window=16, pool=7, budget=64)
     Q, K, V = _inputs(cfg)
