@@ -373,7 +373,48 @@ def run_gpu(args):
             torch.cuda.synchronize()
         ev_bytes = 2 * cfg.B * cfg.Hkv * n_e * cfg.D * 2
         t_g, t_r = evs[0].elapsed_time(evs[1]), evs[1].elapsed_time(evs[2]) / reps
+        # offload to and reload from page-locked host memory on a copy stream (Algorithm 1 line 4,
+        # Algorithm 2 line 4), alone and with decode steps running on the compute stream
+        K_h = torch.empty(K_e.shape, dtype=torch.bfloat16).pin_memory()
+        V_h = torch.empty(V_e.shape, dtype=torch.bfloat16).pin_memory()
+        side = torch.cuda.Stream()
+        c0, c1, c2 = (torch.cuda.Event(enable_timing=True) for _ in range(3))
+        for it in range(2):
+            torch.cuda.synchronize()
+            c0.record(side)
+            cd.calidrop_offload_evicted(p, n_e, K_e, V_e, K_h, V_h, side)
+            c1.record(side)
+            cd.calidrop_reload_evicted(p, n_e, K_h, V_h, K_e, V_e, side)
+            c2.record(side)
+            torch.cuda.synchronize()
+        t_off, t_rel = c0.elapsed_time(c1), c1.elapsed_time(c2)
+        n_dec = min(T, 32)
+
+        def some_decode_steps():
+            for t in range(n_dec):
+                for s_, st_ in enumerate(states):
+                    cd.calidrop_decode(p, dq[t], None, None, st_.K_kept, st_.V_kept, cfg.budget, st_.O_c, st_.LSE_c,
+                                       st_.C_q, outs[s_], lses[s_], flgs[s_], st_.ws_decode)
+
+        d0, d1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        some_decode_steps()
+        torch.cuda.synchronize()
+        d0.record(); some_decode_steps(); d1.record()
+        torch.cuda.synchronize()
+        t_dec_alone = d0.elapsed_time(d1)
+        c0.record(side)
+        cd.calidrop_reload_evicted(p, n_e, K_h, V_h, K_e, V_e, side)
+        c1.record(side)
+        d0.record(); some_decode_steps(); d1.record()
+        torch.cuda.synchronize()
+        t_dec_busy, t_rel_busy = d0.elapsed_time(d1), c0.elapsed_time(c1)
         recompute = {"n_evict": n_e, "gather_evicted_ms": t_g,
+                     "offload_ms": t_off, "offload_gbs": ev_bytes / (t_off * 1e-3) / 1e9,
+                     "reload_ms": t_rel, "reload_gbs": ev_bytes / (t_rel * 1e-3) / 1e9,
+                     "reload_beside_decode": {
+                         "decode_launches": n_dec * S, "decode_ms_alone": t_dec_alone, "decode_ms_with_reload": t_dec_busy,
+                         "reload_ms_with_decode": t_rel_busy,
+                         "note": "eager decode launches on the compute stream while the reload runs on a copy stream"},
                      "gather_evicted_gbs": 2 * ev_bytes / (t_g * 1e-3) / 1e9,     # rows read and written
                      "recalibrate_us": t_r * 1e3, "recalibrate_gbs": ev_bytes / (t_r * 1e-3) / 1e9,
                      "recalibrate_frac_of_measured_hbm": ev_bytes / (t_r * 1e-3) / 1e9 / peaks["hbm_gbs"]}

@@ -166,6 +166,30 @@ int calidrop_gather_evicted(const calidrop_params* p, const void* K, const void*
                             void* workspace, size_t workspace_bytes, void* stream);
 
 /*
+ * Offload and reload of the compacted evicted rows ("Offload KV_evict" in Algorithm 1, line 4;
+ * "reload" in Algorithm 2, line 4; Section 3.2: the evicted entries move to CPU memory and come
+ * back when a recomputation is due).  Each call enqueues one asynchronous copy per tensor on
+ * `copy_stream`, a stream of the caller's that is normally NOT the compute stream, so that the
+ * transfer runs beside the decode steps:
+ *   calidrop_offload_evicted   K_evict, V_evict (device) -> K_host, V_host (HOST)
+ *   calidrop_reload_evicted    K_host, V_host (HOST) -> K_evict, V_evict (device)
+ *
+ *   K_evict, V_evict  device [B, Hkv, n_evict, D] bf16 (as written by calidrop_gather_evicted)
+ *   K_host, V_host    HOST buffers of the same size; page-locked (cudaHostAlloc / cudaHostRegister)
+ *                     if the copy is to be asynchronous with respect to the host
+ *   wait_event        cudaEvent_t or NULL: copy_stream waits for it first (e.g. recorded on the
+ *                     compute stream after calidrop_gather_evicted, or after the last use of the rows)
+ *   done_event        cudaEvent_t or NULL: recorded on copy_stream behind the copies; the compute
+ *                     stream waits for it (cudaStreamWaitEvent) before calidrop_recalibrate reads the rows
+ * The library keeps neither the events nor the pointers.  Errors: INVALID_ARG (null pointer,
+ * n_evict < 1), CUDA_ERROR.
+ */
+int calidrop_offload_evicted(const calidrop_params* p, int32_t n_evict, const void* K_evict, const void* V_evict,
+                             void* K_host, void* V_host, void* copy_stream, void* wait_event, void* done_event);
+int calidrop_reload_evicted(const calidrop_params* p, int32_t n_evict, const void* K_host, const void* V_host,
+                            void* K_evict, void* V_evict, void* copy_stream, void* wait_event, void* done_event);
+
+/*
  * Recompute one calibration entry with the current query (Algorithm 2, lines 4-6, taken when
  * rho < theta1; the printed "Q_-1" is read as the current query Q_t, which line 6 stores):
  * per (b, query head hq of kv head h)

@@ -24,7 +24,7 @@ MAX_LAYERS = 32
 
 EXPORTS = [
     "calidrop_compress_workspace_bytes", "calidrop_compress", "calidrop_calibrate", "calidrop_gather_evicted",
-    "calidrop_recalibrate",
+    "calidrop_recalibrate", "calidrop_offload_evicted", "calidrop_reload_evicted",
     "calidrop_compress_workspace_layout",
     "calidrop_decode_workspace_bytes", "calidrop_decode_workspace_init",
     "calidrop_decode_workspace_status_offset", "calidrop_decode",
@@ -79,6 +79,9 @@ def load():
     lib.calidrop_recalibrate.restype = C.c_int
     lib.calidrop_recalibrate.argtypes = [C.POINTER(Params), vp, vp, vp, C.c_int32, C.c_int32, vp, vp, vp, vp,
                                          C.c_size_t, vp]
+    for f in (lib.calidrop_offload_evicted, lib.calidrop_reload_evicted):
+        f.restype = C.c_int
+        f.argtypes = [C.POINTER(Params), C.c_int32, vp, vp, vp, vp, vp, vp, vp]
     lib.calidrop_calibrate.restype = C.c_int
     lib.calidrop_calibrate.argtypes = [C.POINTER(Params)] + [vp] * 11 + [C.c_size_t, vp]
     lib.calidrop_decode_workspace_status_offset.restype = C.c_size_t
@@ -194,6 +197,36 @@ def calidrop_recalibrate(p, q, K_evict, V_evict, n_evict, slot, O_c, LSE_c, C_q,
                                      workspace.numel() * workspace.element_size(), _stream())
     if check:
         _check(rc, "calidrop_recalibrate")
+    return rc
+
+
+def _handle(x):
+    """A CUDA stream or event of torch (or a raw handle, or None) as the integer the C-ABI takes."""
+    if x is None:
+        return None
+    if isinstance(x, torch.cuda.Stream):
+        return x.cuda_stream
+    if isinstance(x, torch.cuda.Event):
+        h = x.cuda_event                      # exists once the event has been recorded
+        return h.value if hasattr(h, "value") else int(h)
+    return int(x)
+
+
+def calidrop_offload_evicted(p, n_evict, K_evict, V_evict, K_host, V_host, copy_stream, wait_event=None,
+                             done_event=None, check=True) -> int:
+    rc = load().calidrop_offload_evicted(C.byref(p), int(n_evict), _ptr(K_evict), _ptr(V_evict), _ptr(K_host),
+                                         _ptr(V_host), _handle(copy_stream), _handle(wait_event), _handle(done_event))
+    if check:
+        _check(rc, "calidrop_offload_evicted")
+    return rc
+
+
+def calidrop_reload_evicted(p, n_evict, K_host, V_host, K_evict, V_evict, copy_stream, wait_event=None,
+                            done_event=None, check=True) -> int:
+    rc = load().calidrop_reload_evicted(C.byref(p), int(n_evict), _ptr(K_host), _ptr(V_host), _ptr(K_evict),
+                                        _ptr(V_evict), _handle(copy_stream), _handle(wait_event), _handle(done_event))
+    if check:
+        _check(rc, "calidrop_reload_evicted")
     return rc
 
 

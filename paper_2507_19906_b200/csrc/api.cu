@@ -345,6 +345,36 @@ int calidrop_gather_evicted(const calidrop_params* p, const void* K, const void*
   return e == cudaSuccess ? CALIDROP_OK : cuda_fail(e);
 }
 
+namespace {
+// One asynchronous copy per tensor on the caller's copy stream, between the caller's two events.
+int move_evicted(const calidrop_params* p, int32_t n_evict, const void* K_src, const void* V_src, void* K_dst,
+                 void* V_dst, cudaMemcpyKind kind, void* copy_stream, void* wait_event, void* done_event) {
+  int rc = check_common(p);
+  if (rc != CALIDROP_OK) return rc;
+  if (!K_src || !V_src || !K_dst || !V_dst || n_evict < 1) return CALIDROP_INVALID_ARG;
+  cudaStream_t cs = (cudaStream_t)copy_stream;
+  const size_t bytes = (size_t)p->B * p->Hkv * n_evict * kD * 2;
+  cudaError_t e;
+  if (wait_event && (e = cudaStreamWaitEvent(cs, (cudaEvent_t)wait_event, 0)) != cudaSuccess) return cuda_fail(e);
+  if ((e = cudaMemcpyAsync(K_dst, K_src, bytes, kind, cs)) != cudaSuccess) return cuda_fail(e);
+  if ((e = cudaMemcpyAsync(V_dst, V_src, bytes, kind, cs)) != cudaSuccess) return cuda_fail(e);
+  if (done_event && (e = cudaEventRecord((cudaEvent_t)done_event, cs)) != cudaSuccess) return cuda_fail(e);
+  return CALIDROP_OK;
+}
+}  // namespace
+
+int calidrop_offload_evicted(const calidrop_params* p, int32_t n_evict, const void* K_evict, const void* V_evict,
+                             void* K_host, void* V_host, void* copy_stream, void* wait_event, void* done_event) {
+  return move_evicted(p, n_evict, K_evict, V_evict, K_host, V_host, cudaMemcpyDeviceToHost, copy_stream, wait_event,
+                      done_event);
+}
+
+int calidrop_reload_evicted(const calidrop_params* p, int32_t n_evict, const void* K_host, const void* V_host,
+                            void* K_evict, void* V_evict, void* copy_stream, void* wait_event, void* done_event) {
+  return move_evicted(p, n_evict, K_host, V_host, K_evict, V_evict, cudaMemcpyHostToDevice, copy_stream, wait_event,
+                      done_event);
+}
+
 int calidrop_recalibrate(const calidrop_params* p, const void* q, const void* K_evict, const void* V_evict,
                          int32_t n_evict, int32_t slot, float* O_c, float* LSE_c, void* C_q, void* workspace,
                          size_t workspace_bytes, void* stream) {

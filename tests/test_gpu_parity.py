@@ -608,6 +608,76 @@ def test_gather_evicted_and_recalibrate(cuda_lib, B, Hq, Hkv, L, W, budget, n_ca
             assert_close_out(got[b, hq], o[0], "decode after the recompute vs attention over the whole prompt")
 
 
+def test_offload_and_reload_of_the_evicted_rows_beside_decode(cuda_lib):
+    """Algorithm 1 line 4 / Algorithm 2 line 4: the compacted evicted rows go to page-locked host
+    memory on a copy stream and come back on it, bit for bit, while decode steps run on the compute
+    stream; the decode outputs are the same as without the transfer, and a recompute from the
+    reloaded rows equals one from the rows that never left."""
+    cd = cuda_lib
+    B, Hq, Hkv, L, W, budget, n_cal = 2, 8, 2, 6000, 32, 512, 32
+    cfg = wl.small_config(B=B, Hq=Hq, Hkv=Hkv, L=L, window=W, pool=7, budget=budget, steps=6, n_sink=4, n_heavy=100)
+    Q, K, V = _inputs(cfg)
+    T = 6
+    g = gpu_compress(Q, K, V, window=W, pool=7, budget=budget, n_cal=n_cal, cap=budget + T, keep_inputs=True)
+    p, st = g.p, g.st
+    n_e = L - budget
+    ev_idx = torch.empty((B, Hkv, n_e), dtype=torch.int32, device="cuda")
+    K_e = torch.empty((B, Hkv, n_e, 128), dtype=torch.bfloat16, device="cuda")
+    V_e = torch.empty_like(K_e)
+    K_h = torch.empty(K_e.shape, dtype=torch.bfloat16).pin_memory()
+    V_h = torch.empty(V_e.shape, dtype=torch.bfloat16).pin_memory()
+    main, side = torch.cuda.current_stream(), torch.cuda.Stream()
+    gathered, offloaded, reloaded = torch.cuda.Event(), torch.cuda.Event(), torch.cuda.Event()
+    cd.calidrop_gather_evicted(p, g.dK, g.dV, st.kept_idx, ev_idx, K_e, V_e, st.ws_compress)
+    gathered.record(main)
+    offloaded.record(side); reloaded.record(side)          # (creates the handles; they are recorded again below)
+    cd.calidrop_offload_evicted(p, n_e, K_e, V_e, K_h, V_h, side, wait_event=gathered, done_event=offloaded)
+    offloaded.synchronize()
+    K_ref, V_ref = K_e.clone(), V_e.clone()
+    assert torch.equal(K_h, K_ref.cpu()) and torch.equal(V_h, V_ref.cpu())
+    # decode steps without any transfer, on copies of the cache
+    q, kn, vn = wl.gen_decode_inputs(cfg, Q, steps=T)
+    dq, dk, dv = [to_dev(x) for x in q], [to_dev(x) for x in kn], [to_dev(x) for x in vn]
+
+    def run_steps(Kc, Vc):
+        outs = []
+        for t in range(T):
+            o = torch.empty((B, Hq, 128), dtype=torch.bfloat16, device="cuda")
+            cd.calidrop_decode(p, dq[t], dk[t], dv[t], Kc, Vc, budget + t, st.O_c, st.LSE_c, st.C_q, o, None, None,
+                               st.ws_decode)
+            outs.append(o)
+        return outs
+
+    quiet = run_steps(st.K_kept.clone(), st.V_kept.clone())
+    torch.cuda.synchronize()
+    # the device copy is dropped (overwritten), then reloaded on the side stream while decode runs
+    K_e.zero_(); V_e.zero_()
+    torch.cuda.synchronize()
+    cd.calidrop_reload_evicted(p, n_e, K_h, V_h, K_e, V_e, side, wait_event=None, done_event=reloaded)
+    busy = run_steps(st.K_kept.clone(), st.V_kept.clone())
+    main.wait_event(reloaded)                              # the compute stream may read the rows from here on
+    assert torch.equal(K_e, K_ref) and torch.equal(V_e, V_ref)
+    for a, b in zip(quiet, busy):
+        assert torch.equal(a, b)
+    off = cd.calidrop_decode_workspace_status_offset(p)
+    assert int(st.ws_decode[off:off + 4].view(torch.int32).item()) == 0
+    # a recompute from the reloaded rows
+    rng = np.random.Generator(np.random.Philox(key=[12, L]))
+    qr = wl.f32_to_bf16_bits(rng.standard_normal((B, Hq, 128)).astype(np.float32))
+    cd.calidrop_recalibrate(p, to_dev(qr), K_e, V_e, n_e, 5, st.O_c, st.LSE_c, st.C_q, st.ws_decode)
+    torch.cuda.synchronize()
+    ev = ev_idx.cpu().numpy()
+    for b in range(B):
+        for hq in range(Hq):
+            h = hq // (Hq // Hkv)
+            o, l = oracle.full_attention(qr[b, hq][None], K[b, h][ev[b, h]], V[b, h][ev[b, h]])
+            assert_close_out(st.O_c[b, hq, 5].cpu().numpy(), o[0], "O_c recomputed from the reloaded rows")
+            assert abs(float(st.LSE_c[b, hq, 5]) - l[0]) < 1e-3
+    # argument checks
+    assert cd.calidrop_offload_evicted(p, 0, K_e, V_e, K_h, V_h, side, check=False) == cd.INVALID_ARG
+    assert cd.calidrop_reload_evicted(p, n_e, None, V_h, K_e, V_e, side, check=False) == cd.INVALID_ARG
+
+
 # ---------------------------------------------------------------- seeded random shapes
 def _random_shapes(n, seed):
     rng = np.random.Generator(np.random.Philox(key=[seed, 1]))
