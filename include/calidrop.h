@@ -145,6 +145,32 @@ int calidrop_calibrate(const calidrop_params* p,
                        void* workspace, size_t workspace_bytes, void* stream);
 
 /*
+ * Kept lists of two other eviction rules, written on the device for calidrop_calibrate (the paper's
+ * Section 4.1.2 applies CaliDrop on top of StreamingLLM, H2O and SnapKV alike; Section 4.1.3 gives
+ * their settings: StreamingLLM with 32 sink tokens plus the most recent ones, H2O with half of the
+ * budget for the heavy hitters of the accumulated attention score and half for the most recent).
+ *
+ * calidrop_select_streaming: kept = the first n_sink prompt rows and the last n_kept - n_sink ones,
+ *   n_kept = min(budget, L).  INVALID_ARG unless 0 <= n_sink <= n_kept - min(window, n_kept) (the
+ *   observation-window rows are part of the recent ones).
+ * calidrop_select_from_scores: kept = the budget - tail rows of [0, L - tail) with the largest
+ *   pooled score (zero-padded average pool of kernel `pool` of `p`, 1 for none; ties to the lowest
+ *   index) and the last `tail` rows.  With the accumulated attention score of the prefill (its
+ *   column sums over all queries, a by-product of the prefill attention that this library does not
+ *   compute) and tail = budget / 2 this is H2O's rule; with the window votes and tail = window it is
+ *   the selection step of calidrop_compress.
+ *     scores in [B, Hkv, L] f32, finite and non-negative (they are ordered by their bit patterns);
+ *            entries at and beyond L - tail are not read
+ *     tail   window <= tail < budget < L
+ *     workspace: a calidrop_compress workspace for `p` (the pooled scores and a bitmap go there)
+ *   UNSUPPORTED beyond 262144 prompt rows.
+ *   kept_idx out [B, Hkv, n_kept] i32, ascending.
+ */
+int calidrop_select_streaming(const calidrop_params* p, int32_t n_sink, int32_t* kept_idx, void* stream);
+int calidrop_select_from_scores(const calidrop_params* p, const float* scores, int32_t tail, int32_t* kept_idx,
+                                void* workspace, size_t workspace_bytes, void* stream);
+
+/*
  * The complement of calidrop_compress's gather: the evicted candidate rows, compacted, for the
  * caller to offload ("offload them to the CPU", Algorithm 1 line 4) and to hand back to
  * calidrop_recalibrate when a decode step raises needs_recompute.

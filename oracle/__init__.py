@@ -1,5 +1,6 @@
 """CPU oracle (test infrastructure only): see oracle.py and calidrop_oracle.c."""
 from .oracle import (  # noqa: F401
+    accumulated_attention,
     build_oracle,
     calibrate_given_indices,
     compress,
@@ -7,5 +8,7 @@ from .oracle import (  # noqa: F401
     full_attention,
     max_threads,
     pool_votes,
+    select_from_scores,
+    streaming_indices,
     topk,
 )

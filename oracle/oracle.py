@@ -185,3 +185,38 @@ def decode(q, k_new, v_new, K_kept, V_kept, kv_len, O_c, LSE_c, C_q, *,
         C.c_double(theta1), C.c_double(theta2), _p(force_c), _p(force_apply),
         _p(r.out), _p(r.lse), _p(r.lse_a), _p(r.rho), _p(r.flags))
     return r
+
+
+def streaming_indices(L, budget, n_sink):
+    """StreamingLLM's rule (Section 4.1.3): the first n_sink prompt rows and the most recent ones, min(budget, L) in all."""
+    n_kept = min(budget, L)
+    n_sink = min(n_sink, n_kept)
+    return np.concatenate([np.arange(n_sink), np.arange(L - (n_kept - n_sink), L)]).astype(np.int32)
+
+
+def select_from_scores(scores, *, tail, budget, pool=1):
+    """Kept list from per-row scores [L]: the last `tail` rows plus the budget - tail rows of [0, L - tail) with
+    the largest (pooled) score, ties to the lower index; ascending.  With H2O's accumulated attention score and
+    tail = budget / 2 this is H2O's rule (Section 4.1.3)."""
+    scores = np.ascontiguousarray(scores, dtype=np.float64)
+    L = scores.shape[-1]
+    assert 0 < tail < budget < L
+    pooled = pool_votes(scores[:L - tail], pool)
+    return np.concatenate([topk(pooled, budget - tail), np.arange(L - tail, L)]).astype(np.int32)
+
+
+def accumulated_attention(Q_full, K, scale=None):
+    """H2O's importance: for one kv head, the causal softmax attention of every prompt query of its query group
+    (Q_full [G, L, D], K [L, D], bf16 bits), summed over the queries and the group: score[t] = sum_g sum_{i >= t} a[g,i,t]."""
+    Q_full, K = _u16(Q_full), _u16(K)
+    G, L, D = Q_full.shape
+    scale = scale or default_scale(D)
+    Kf = (K.astype(np.uint32) << 16).view(np.float32).astype(np.float64)
+    score = np.zeros((L,), dtype=np.float64)
+    for g in range(G):
+        Qf = (Q_full[g].astype(np.uint32) << 16).view(np.float32).astype(np.float64)
+        for i in range(L):
+            s = (Kf[:i + 1] @ Qf[i]) * scale
+            e = np.exp(s - s.max())
+            score[:i + 1] += e / e.sum()
+    return score

@@ -25,6 +25,7 @@ MAX_LAYERS = 32
 EXPORTS = [
     "calidrop_compress_workspace_bytes", "calidrop_compress", "calidrop_calibrate", "calidrop_gather_evicted",
     "calidrop_recalibrate", "calidrop_offload_evicted", "calidrop_reload_evicted",
+    "calidrop_select_streaming", "calidrop_select_from_scores",
     "calidrop_compress_workspace_layout",
     "calidrop_decode_workspace_bytes", "calidrop_decode_workspace_init",
     "calidrop_decode_workspace_status_offset", "calidrop_decode",
@@ -82,6 +83,10 @@ def load():
     for f in (lib.calidrop_offload_evicted, lib.calidrop_reload_evicted):
         f.restype = C.c_int
         f.argtypes = [C.POINTER(Params), C.c_int32, vp, vp, vp, vp, vp, vp, vp]
+    lib.calidrop_select_streaming.restype = C.c_int
+    lib.calidrop_select_streaming.argtypes = [C.POINTER(Params), C.c_int32, vp, vp]
+    lib.calidrop_select_from_scores.restype = C.c_int
+    lib.calidrop_select_from_scores.argtypes = [C.POINTER(Params), vp, C.c_int32, vp, vp, C.c_size_t, vp]
     lib.calidrop_calibrate.restype = C.c_int
     lib.calidrop_calibrate.argtypes = [C.POINTER(Params)] + [vp] * 11 + [C.c_size_t, vp]
     lib.calidrop_decode_workspace_status_offset.restype = C.c_size_t
@@ -197,6 +202,21 @@ def calidrop_recalibrate(p, q, K_evict, V_evict, n_evict, slot, O_c, LSE_c, C_q,
                                      workspace.numel() * workspace.element_size(), _stream())
     if check:
         _check(rc, "calidrop_recalibrate")
+    return rc
+
+
+def calidrop_select_streaming(p, n_sink, kept_idx, check=True) -> int:
+    rc = load().calidrop_select_streaming(C.byref(p), int(n_sink), _ptr(kept_idx), _stream())
+    if check:
+        _check(rc, "calidrop_select_streaming")
+    return rc
+
+
+def calidrop_select_from_scores(p, scores, tail, kept_idx, workspace, check=True) -> int:
+    rc = load().calidrop_select_from_scores(C.byref(p), _ptr(scores), int(tail), _ptr(kept_idx), _ptr(workspace),
+                                            workspace.numel() * workspace.element_size(), _stream())
+    if check:
+        _check(rc, "calidrop_select_from_scores")
     return rc
 
 

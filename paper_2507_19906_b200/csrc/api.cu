@@ -318,6 +318,37 @@ int calidrop_calibrate(const calidrop_params* p, const void* Q_obs, const void* 
   return CALIDROP_OK;
 }
 
+int calidrop_select_streaming(const calidrop_params* p, int32_t n_sink, int32_t* kept_idx, void* stream) {
+  int rc = check_compress(p);
+  if (rc != CALIDROP_OK) return rc;
+  if (!kept_idx || !aligned16(kept_idx)) return CALIDROP_INVALID_ARG;
+  const CompressGeom g = make_geom(p);
+  const int recent_min = p->window < g.n_kept ? p->window : g.n_kept;
+  if (n_sink < 0 || n_sink > g.n_kept - recent_min) return CALIDROP_INVALID_ARG;
+  if (!device_supported()) return CALIDROP_UNSUPPORTED;
+  cudaError_t e = launch_streaming_indices(g, n_sink, kept_idx, (cudaStream_t)stream);
+  return e == cudaSuccess ? CALIDROP_OK : cuda_fail(e);
+}
+
+int calidrop_select_from_scores(const calidrop_params* p, const float* scores, int32_t tail, int32_t* kept_idx,
+                                void* workspace, size_t workspace_bytes, void* stream) {
+  int rc = check_compress(p);
+  if (rc != CALIDROP_OK) return rc;
+  if (!scores || !kept_idx || !workspace || !aligned16(scores) || !aligned16(kept_idx)) return CALIDROP_INVALID_ARG;
+  if (reinterpret_cast<uintptr_t>(workspace) & 255u) return CALIDROP_INVALID_ARG;
+  if (p->budget >= p->L || tail < p->window || tail >= p->budget) return CALIDROP_INVALID_ARG;
+  const CompressGeom g0 = make_geom(p);
+  const CompressWs ws = make_ws(g0);   // sized for window <= tail: the pooled scores of L - tail rows fit
+  if (workspace_bytes < ws.total) return CALIDROP_WORKSPACE_TOO_SMALL;
+  // the selection's geometry: `tail` rows are always kept, the rest compete
+  CompressGeom g = g0;
+  g.W = tail; g.n_cand = p->L - tail; g.k_sel = p->budget - tail; g.sized = 0; g.n_calib = 0;
+  if (!select_cluster_supported(g)) return CALIDROP_UNSUPPORTED;
+  if (!device_supported()) return CALIDROP_UNSUPPORTED;
+  cudaError_t e = launch_pool_select_scores(g, ws, (char*)workspace, scores, (size_t)p->L, kept_idx, (cudaStream_t)stream);
+  return e == cudaSuccess ? CALIDROP_OK : cuda_fail(e);
+}
+
 int calidrop_gather_evicted(const calidrop_params* p, const void* K, const void* V, const int32_t* kept_idx,
                             int32_t* evict_idx, void* K_evict, void* V_evict, void* workspace,
                             size_t workspace_bytes, void* stream) {

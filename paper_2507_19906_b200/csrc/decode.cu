@@ -117,6 +117,26 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
   }
   return true;
 }
+// The same wait without the shortcut on the CTA's abort flag: only its own time limit ends it early.
+// For waits that must be sat out even in a CTA that is giving up, because other CTAs still write
+// into (or read from) this CTA's shared memory until the awaited phase completes.
+__device__ __forceinline__ bool mbar_wait_sit_out(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                                  unsigned* status, unsigned code) {
+  long long t0 = 0;
+  unsigned polls = 0;
+  while (!mbar_try_wait(bar, parity)) {
+    if ((++polls & 255u) == 0u) {
+      const long long now = clock64();
+      if (t0 == 0) t0 = now;
+      if (now - t0 > kWaitLimitCycles) {
+        *abort_flag = 1;
+        atomicCAS(status, 0u, code);
+        return false;
+      }
+    }
+  }
+  return true;
+}
 __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1,
                                             int c2, uint64_t pol) {
   asm volatile(
@@ -647,8 +667,11 @@ decode_kernel(const __grid_constant__ DecodeArgsT<NL> args) {
   }
   // (B) everything pushed to this CTA has arrived when its byte count is complete.  No cluster
   // barrier: a CTA waits for its own data only, and it cannot leave before the others have read its
-  // s_best, because their pushes, which it waits for, come after those reads.
-  mbar_wait(smem_u32(&s_push), 0, abort_flag, a.status, 0x300u);
+  // s_best, because their pushes, which it waits for, come after those reads.  That argument needs
+  // the wait to be sat out: a CTA whose earlier wait ran out (abort flag raised) must not skip it,
+  // or its peers, which always reach their pushes, would read and write the shared memory of a
+  // CTA that has left.  Only the wait's own time limit remains as the way out.
+  mbar_wait_sit_out(smem_u32(&s_push), 0, abort_flag, a.status, 0x300u);
 
   // ---- (6) finish: reduce the splits for this CTA's output slice (local data only from here on,
   // so no CTA has to wait for another before it leaves)

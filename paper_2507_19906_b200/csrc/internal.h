@@ -109,6 +109,9 @@ cudaError_t launch_pool_select(const CompressGeom& g, const CompressWs& ws, char
 bool select_cluster_supported(const CompressGeom& g);
 cudaError_t launch_pool_select_cluster(const CompressGeom& g, const CompressWs& ws, char* wsp, int32_t* kept_idx,
                                        cudaStream_t st);
+cudaError_t launch_pool_select_scores(const CompressGeom& g, const CompressWs& ws, char* wsp, const float* scores,
+                                      size_t stride, int32_t* kept_idx, cudaStream_t st);
+cudaError_t launch_streaming_indices(const CompressGeom& g, int n_sink, int32_t* kept_idx, cudaStream_t st);
 cudaError_t launch_bitmap_from_indices(const CompressGeom& g, const CompressWs& ws, char* wsp,
                                        const int32_t* kept_idx, cudaStream_t st);
 cudaError_t launch_gather_rows(const CompressGeom& g, const void* K, const void* V, const int32_t* idx, int n_rows,

@@ -184,6 +184,7 @@ gather_kernel(const uint4* __restrict__ K, const uint4* __restrict__ V,
   const int chunk = threadIdx.x & 15;
   if (i >= n_kept) return;
   const int t = kept_idx[(size_t)unit * n_kept + i];
+  if (t < 0 || t >= L) return;   // a caller's list may hold anything: rows outside the prompt are skipped
   const size_t src = ((size_t)unit * L + t) * 16 + chunk;
   const size_t dst = ((size_t)unit * cap + i) * 16 + chunk;
   K_kept[dst] = __ldg(K + src);
@@ -226,6 +227,10 @@ evicted_indices_kernel(const uint32_t* __restrict__ bitmap, int32_t* __restrict_
     if (rem < 32) z &= (1u << rem) - 1u;
     return z;
   };
+  // entries that no zero bit fills (a kept list with fewer candidates than expected leaves fewer
+  // evicted rows than n_evict) hold -1, which the gather skips
+  for (int i = tid; i < n_evict; i += kSelThreads) out[i] = -1;
+  __syncthreads();
   unsigned cnt = 0;
   for (int w = w0; w < w1; ++w) cnt += __popc(zeros_of(w));
   unsigned incl = cnt;

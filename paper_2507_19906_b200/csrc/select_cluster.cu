@@ -30,7 +30,7 @@ __global__ void __cluster_dims__(kClu, 1, 1) __launch_bounds__(kT)
 pool_select_cluster_kernel(const float* __restrict__ vote, float* __restrict__ pooled,
                            uint32_t* __restrict__ bitmap, int32_t* __restrict__ kept_idx, int n_cand, int L,
                            int pool, int k_sel, int n_kept, int bitmap_words, uint32_t* __restrict__ mask2,
-                           int n_calib) {
+                           int n_calib, size_t vote_stride) {
   __shared__ unsigned hist[kW][256];
   __shared__ unsigned mine[2][256];   // this CTA's histogram of the current pass (double-buffered)
   __shared__ unsigned total[256];
@@ -43,7 +43,7 @@ pool_select_cluster_kernel(const float* __restrict__ vote, float* __restrict__ p
   const int unit = blockIdx.y;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int chunk = ROWS * kT;
-  const float* v = vote + (size_t)unit * n_cand;
+  const float* v = vote + (size_t)unit * vote_stride;
   float* pl = pooled + (size_t)unit * n_cand;
   uint32_t* bm = bitmap + (size_t)unit * bitmap_words;
   int32_t* kept = kept_idx + (size_t)unit * n_kept;
@@ -228,11 +228,12 @@ pool_select_cluster_kernel(const float* __restrict__ vote, float* __restrict__ p
 }
 
 template <int ROWS>
-void launch_rows(const CompressGeom& g, const CompressWs& ws, char* wsp, int32_t* kept_idx, cudaStream_t st) {
+void launch_rows(const CompressGeom& g, const CompressWs& ws, char* wsp, const float* scores, size_t stride,
+                 int32_t* kept_idx, cudaStream_t st) {
   pool_select_cluster_kernel<ROWS><<<dim3(kClu, g.units), kT, 0, st>>>(
-      (const float*)(wsp + ws.vote), (float*)(wsp + ws.pooled), (uint32_t*)(wsp + ws.bitmap), kept_idx, g.n_cand,
+      scores, (float*)(wsp + ws.pooled), (uint32_t*)(wsp + ws.bitmap), kept_idx, g.n_cand,
       g.L, g.pool, g.k_sel, g.n_kept, g.bitmap_words, (g.sized && g.n_calib > 0) ? (uint32_t*)(wsp + ws.bitmap2) : nullptr,
-      g.n_calib);
+      g.n_calib, stride);
 }
 
 }  // namespace
@@ -240,15 +241,34 @@ void launch_rows(const CompressGeom& g, const CompressWs& ws, char* wsp, int32_t
 // The cluster kernel keeps at most 32 keys per thread: 8 CTAs x 1024 threads x 32.
 bool select_cluster_supported(const CompressGeom& g) { return !g.keep_all && g.L <= kClu * kT * 32; }
 
+// Selection from per-candidate scores [units][stride] (the window votes of the workspace, or a
+// caller's scores).
+cudaError_t launch_pool_select_scores(const CompressGeom& g, const CompressWs& ws, char* wsp, const float* scores,
+                                      size_t stride, int32_t* kept_idx, cudaStream_t st) {
+  const int rows = (g.L + kClu * kT - 1) / (kClu * kT);
+  if (rows <= 1) launch_rows<1>(g, ws, wsp, scores, stride, kept_idx, st);
+  else if (rows <= 2) launch_rows<2>(g, ws, wsp, scores, stride, kept_idx, st);
+  else if (rows <= 4) launch_rows<4>(g, ws, wsp, scores, stride, kept_idx, st);
+  else if (rows <= 8) launch_rows<8>(g, ws, wsp, scores, stride, kept_idx, st);
+  else if (rows <= 16) launch_rows<16>(g, ws, wsp, scores, stride, kept_idx, st);
+  else launch_rows<32>(g, ws, wsp, scores, stride, kept_idx, st);
+  count_launch(1);
+  return cudaGetLastError();
+}
+
 cudaError_t launch_pool_select_cluster(const CompressGeom& g, const CompressWs& ws, char* wsp, int32_t* kept_idx,
                                        cudaStream_t st) {
-  const int rows = (g.L + kClu * kT - 1) / (kClu * kT);
-  if (rows <= 1) launch_rows<1>(g, ws, wsp, kept_idx, st);
-  else if (rows <= 2) launch_rows<2>(g, ws, wsp, kept_idx, st);
-  else if (rows <= 4) launch_rows<4>(g, ws, wsp, kept_idx, st);
-  else if (rows <= 8) launch_rows<8>(g, ws, wsp, kept_idx, st);
-  else if (rows <= 16) launch_rows<16>(g, ws, wsp, kept_idx, st);
-  else launch_rows<32>(g, ws, wsp, kept_idx, st);
+  return launch_pool_select_scores(g, ws, wsp, (const float*)(wsp + ws.vote), (size_t)g.n_cand, kept_idx, st);
+}
+
+// Sink-plus-recent index rule: the first n_sink rows and the last n_kept - n_sink.
+__global__ void streaming_indices_kernel(int32_t* __restrict__ kept_idx, int L, int n_kept, int n_sink) {
+  const int unit = blockIdx.y, i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < n_kept) kept_idx[(size_t)unit * n_kept + i] = i < n_sink ? i : L - (n_kept - i);
+}
+
+cudaError_t launch_streaming_indices(const CompressGeom& g, int n_sink, int32_t* kept_idx, cudaStream_t st) {
+  streaming_indices_kernel<<<dim3((g.n_kept + 255) / 256, g.units), 256, 0, st>>>(kept_idx, g.L, g.n_kept, n_sink);
   count_launch(1);
   return cudaGetLastError();
 }

@@ -309,8 +309,11 @@ def test_config2_full(cuda_lib, n_cal):
     assert st["applied"] > 0.5 * st["total"]
 
 
-def _sampled_units_check(cfg, layer, n_cal, units, steps, step_ids):
-    """Full-size GPU run; the oracle evaluates only the sampled (batch, kv-head) units."""
+def _sampled_units_check(cfg, layer, n_cal, units, steps, step_ids, compress_units=None):
+    """Full-size GPU run through the C-ABI.  The oracle evaluates compress-and-calibrate on
+    `compress_units` (default: `units`) and the decode steps `step_ids` on `units`; the sampled units
+    go to the oracle as one batch, so that its loop over units runs on all host cores.
+    Returns (number of heads that applied the calibration, number that did not) over the checked steps."""
     Q, K, V = _inputs(cfg, layer)
     T = steps
     g = gpu_compress(Q, K, V, window=cfg.window, pool=cfg.pool, budget=cfg.budget, n_cal=n_cal,
@@ -331,20 +334,32 @@ def _sampled_units_check(cfg, layer, n_cal, units, steps, step_ids):
             torch.cuda.synchronize()
             rec[t] = (wl.bf16_bits_to_f64(to_bits(out)), lse.cpu().numpy(), flags.cpu().numpy())
     torch.cuda.synchronize()
-    applied = 0
+    off = cd.calidrop_decode_workspace_status_offset(p)
+    assert int(st.ws_decode[off:off + 4].view(torch.int32).item()) == 0, "a wait of the decode kernel ran out"
+
+    # the sampled units as a batch of single-kv-head problems: [n, G, W, D] queries, [n, 1, L, D] keys/values
+    cu = list(compress_units if compress_units is not None else units)
+    assert set(units) <= set(cu)
+    hsl = lambda h: slice(h * G, (h + 1) * G)
+    Qs = np.ascontiguousarray(np.stack([Q[b, hsl(h)] for b, h in cu]))
+    Ks = np.ascontiguousarray(np.stack([K[b, h:h + 1] for b, h in cu]))
+    Vs = np.ascontiguousarray(np.stack([V[b, h:h + 1] for b, h in cu]))
+    sub = type("R", (), {})()
+    sub.kept_idx = np.stack([g.kept_idx[b, h:h + 1] for b, h in cu])
+    sub.K_kept = np.stack([g.K_kept[b, h:h + 1] for b, h in cu])
+    sub.V_kept = np.stack([g.V_kept[b, h:h + 1] for b, h in cu])
+    sub.O_c = np.stack([g.O_c[b, hsl(h)] for b, h in cu])
+    sub.LSE_c = np.stack([g.LSE_c[b, hsl(h)] for b, h in cu])
+    sub.C_q = np.stack([g.C_q[b, hsl(h)] for b, h in cu])
+    sub.n_kept, sub.cap = g.n_kept, g.cap
+    ref, swaps = compare_compress(sub, Qs, Ks, Vs, window=cfg.window, pool=cfg.pool, budget=cfg.budget, n_cal=n_cal)
+
+    applied = not_applied = 0
     for (b, h) in units:
-        hs = slice(h * G, (h + 1) * G)
-        Qs, Ks, Vs = Q[b:b + 1, hs], K[b:b + 1, h:h + 1], V[b:b + 1, h:h + 1]
-        orc = oracle.compress(Qs, Ks, Vs, window=cfg.window, pool=cfg.pool, budget=cfg.budget, n_cal=n_cal,
-                              cap=cfg.budget + T)
-        sub = type("R", (), {})()
-        sub.kept_idx = g.kept_idx[b:b + 1, h:h + 1]
-        sub.K_kept, sub.V_kept = g.K_kept[b:b + 1, h:h + 1], g.V_kept[b:b + 1, h:h + 1]
-        sub.O_c, sub.LSE_c, sub.C_q = g.O_c[b:b + 1, hs], g.LSE_c[b:b + 1, hs], g.C_q[b:b + 1, hs]
-        sub.n_kept, sub.cap = g.n_kept, g.cap
-        ref, swaps = compare_compress(sub, Qs, Ks, Vs, window=cfg.window, pool=cfg.pool, budget=cfg.budget,
-                                      n_cal=n_cal, orc=orc)
-        Kk, Vk = ref.K_kept.copy(), ref.V_kept.copy()
+        i = cu.index((b, h))
+        hs = hsl(h)
+        Kk, Vk = ref.K_kept[i:i + 1].copy(), ref.V_kept[i:i + 1].copy()
+        Oc, Lc, Cq = ref.O_c[i:i + 1], ref.LSE_c[i:i + 1], ref.C_q[i:i + 1]
         for t in range(T):
             qs = np.ascontiguousarray(q[t, b:b + 1, hs])
             kns = np.ascontiguousarray(kn[t, b:b + 1, h:h + 1])
@@ -352,22 +367,54 @@ def _sampled_units_check(cfg, layer, n_cal, units, steps, step_ids):
             if t not in step_ids:
                 Kk[0, 0, cfg.budget + t], Vk[0, 0, cfg.budget + t] = kns[0, 0], vns[0, 0]
                 continue
-            o = oracle.decode(qs, kns, vns, Kk, Vk, cfg.budget + t, ref.O_c, ref.LSE_c, ref.C_q)
+            o = oracle.decode(qs, kns, vns, Kk, Vk, cfg.budget + t, Oc, Lc, Cq)
             gout, glse, gfl = rec[t]
             gf = gfl[b, hs]
             if not np.array_equal(gf, o.flags[0]):
                 fc = (gf >> 2).astype(np.int32)[None]
                 fa = (gf & 1).astype(np.int32)[None]
-                for i in np.nonzero(gf != o.flags[0])[0]:
-                    rho = o.rho[0, i]
-                    assert abs(rho[gf[i] >> 2] - rho.max()) < 1e-4
-                    assert (gf[i] & 1) == (o.flags[0, i] & 1) or abs(rho.max() - 0.85) < 1e-3
-                o = oracle.decode(qs, None, None, Kk, Vk, cfg.budget + t + 1, ref.O_c, ref.LSE_c, ref.C_q,
+                for k in np.nonzero(gf != o.flags[0])[0]:
+                    rho = o.rho[0, k]
+                    assert abs(rho[gf[k] >> 2] - rho.max()) < 1e-4
+                    assert (gf[k] & 1) == (o.flags[0, k] & 1) or abs(rho.max() - 0.85) < 1e-3
+                o = oracle.decode(qs, None, None, Kk, Vk, cfg.budget + t + 1, Oc, Lc, Cq,
                                   force_c=fc, force_apply=fa)
-            assert_close_out(gout[b, hs], o.out[0], f"unit ({b},{h}) step {t}")
-            assert_close_lse(glse[b, hs], o.lse[0], f"unit ({b},{h}) step {t} lse")
+            assert_close_out(gout[b, hs], o.out[0], f"layer {layer} unit ({b},{h}) step {t}")
+            assert_close_lse(glse[b, hs], o.lse[0], f"layer {layer} unit ({b},{h}) step {t} lse")
             applied += int((gf & 1).sum())
-    return applied
+            not_applied += int((1 - (gf & 1)).sum())
+    return applied, not_applied
+
+
+# ---------------------------------------------------------------- the configurations at full size
+def test_config3_every_unit_and_every_decode_step(cuda_lib):
+    """Config 3 as benchmarked (n_cal = W = 64): compress-and-calibrate of all 32 units against the
+    oracle, and all 128 decode steps on four units (one per batch element)."""
+    cfg = wl.CONFIGS[3]
+    every = [(b, h) for b in range(cfg.B) for h in range(cfg.Hkv)]
+    applied, _ = _sampled_units_check(cfg, 0, n_cal=64, units=[(0, 0), (1, 3), (2, 6), (3, 7)], steps=cfg.steps,
+                                      step_ids=set(range(cfg.steps)), compress_units=every)
+    assert applied > 0
+
+
+def test_config4_every_layer(cuda_lib):
+    """Config 4: each of the 32 layers at full size on the GPU, two units per layer against the oracle
+    (the units move with the layer so that every batch element and kv head is visited)."""
+    cfg = wl.CONFIGS[4]
+    for layer in range(cfg.layers):
+        units = [(layer % cfg.B, (layer // 4) % cfg.Hkv), ((layer + 3) % cfg.B, (layer + 5) % cfg.Hkv)]
+        _sampled_units_check(cfg, layer, n_cal=32, units=units, steps=4, step_ids={0, 3})
+
+
+def test_config5_every_unit_and_the_drift_across_the_gate(cuda_lib):
+    """Config 5: all four units of the 131072-token prompt, and decode steps spread over the whole run
+    of 512: the query noise grows with the step, so early steps apply the calibration and late steps,
+    past the point where the similarity falls below theta2, do not.  Both must occur."""
+    cfg = wl.CONFIGS[5]
+    every = [(0, h) for h in range(cfg.Hkv)]
+    applied, not_applied = _sampled_units_check(cfg, 0, n_cal=64, units=every, steps=cfg.steps,
+                                                step_ids={0, 100, 200, 300, 400, 480, 511})
+    assert applied > 0 and not_applied > 0
 
 
 def test_config3_sampled_units(cuda_lib):
@@ -380,15 +427,9 @@ def test_config3_sampled_units_last_query_only(cuda_lib):
     _sampled_units_check(cfg, 0, n_cal=1, units=[(1, 7)], steps=2, step_ids={1})
 
 
-def test_config4_layers_sampled_units(cuda_lib):
-    cfg = wl.CONFIGS[4]
-    for layer in (0, 31):
-        _sampled_units_check(cfg, layer, n_cal=32, units=[(0, 0), (7, 7), (4, 3)], steps=4, step_ids={0, 3})
-
-
-def test_config5_sampled_unit(cuda_lib):
+def test_config5_last_query_only(cuda_lib):
     cfg = wl.CONFIGS[5]
-    _sampled_units_check(cfg, 0, n_cal=64, units=[(0, 2)], steps=4, step_ids={3})
+    _sampled_units_check(cfg, 0, n_cal=1, units=[(0, 2)], steps=4, step_ids={3})
 
 
 # ---------------------------------------------------------------- decode on hand-built states
@@ -676,6 +717,53 @@ def test_offload_and_reload_of_the_evicted_rows_beside_decode(cuda_lib):
     # argument checks
     assert cd.calidrop_offload_evicted(p, 0, K_e, V_e, K_h, V_h, side, check=False) == cd.INVALID_ARG
     assert cd.calidrop_reload_evicted(p, n_e, None, V_h, K_e, V_e, side, check=False) == cd.INVALID_ARG
+
+
+def test_streaming_and_h2o_kept_lists_from_the_library_feed_the_calibration(cuda_lib):
+    """The paper applies CaliDrop on top of StreamingLLM and H2O too (Sections 4.1.2-4.1.3): their kept
+    lists, written on the device by the library, equal the oracle's, and calidrop_calibrate on them
+    matches the oracle's calibration over the rows those rules evict."""
+    cd = cuda_lib
+    B, Hq, Hkv, L, W, budget, n_cal = 2, 4, 2, 700, 16, 128, 4
+    G = Hq // Hkv
+    cfg = wl.small_config(B=B, Hq=Hq, Hkv=Hkv, L=L, window=W, pool=1, budget=budget, steps=2, n_sink=4, n_heavy=14)
+    Q, K, V = _inputs(cfg)
+    p = cd.make_params(B=B, Hq=Hq, Hkv=Hkv, L=L, window=W, pool=1, budget=budget, n_cal=n_cal, cap=budget + 2)
+    st = cd.alloc_layer_state(p)
+    dQ, dK, dV = to_dev(Q), to_dev(K), to_dev(V)
+    # H2O's accumulated attention needs every prompt query: a seeded full-query tensor whose last W rows are Q_obs
+    rng = np.random.Generator(np.random.Philox(key=[31, 7]))
+    scores = np.zeros((B, Hkv, L), dtype=np.float32)
+    for b in range(B):
+        for h in range(Hkv):
+            Qfull = wl.f32_to_bf16_bits(rng.standard_normal((G, L, 128)).astype(np.float32))
+            Qfull[:, L - W:] = Q[b, h * G:(h + 1) * G]
+            scores[b, h] = oracle.accumulated_attention(Qfull, K[b, h]).astype(np.float32)
+    lists = {}
+    cd.calidrop_select_streaming(p, 32, st.kept_idx)
+    torch.cuda.synchronize()
+    lists["streaming"] = st.kept_idx.cpu().numpy().copy()
+    np.testing.assert_array_equal(lists["streaming"], np.broadcast_to(oracle.streaming_indices(L, budget, 32), (B, Hkv, budget)))
+    cd.calidrop_select_from_scores(p, torch.from_numpy(scores).cuda(), budget // 2, st.kept_idx, st.ws_compress)
+    torch.cuda.synchronize()
+    lists["h2o"] = st.kept_idx.cpu().numpy().copy()
+    for b in range(B):
+        for h in range(Hkv):
+            # fp32 scores on both sides: the order is the same bit for bit
+            np.testing.assert_array_equal(lists["h2o"][b, h], oracle.select_from_scores(scores[b, h], tail=budget // 2, budget=budget))
+    for name, kept in lists.items():
+        st.kept_idx.copy_(torch.from_numpy(kept))
+        cd.calidrop_calibrate(p, dQ, dK, dV, None, st.kept_idx, st.K_kept, st.V_kept, st.O_c, st.LSE_c, st.C_q,
+                              st.ws_compress)
+        torch.cuda.synchronize()
+        ref = oracle.calibrate_given_indices(Q, K, V, kept, n_cal=n_cal, cap=budget + 2)
+        np.testing.assert_array_equal(to_bits(st.K_kept)[:, :, :budget], ref.K_kept[:, :, :budget])
+        assert_close_lse(st.LSE_c.cpu().numpy(), ref.LSE_c, f"{name}: LSE_c")
+        assert_close_out(st.O_c.cpu().numpy(), ref.O_c, f"{name}: O_c")
+    # argument checks
+    assert cd.calidrop_select_streaming(p, budget, st.kept_idx, check=False) == cd.INVALID_ARG
+    assert cd.calidrop_select_from_scores(p, torch.from_numpy(scores).cuda(), W - 1, st.kept_idx, st.ws_compress,
+                                          check=False) == cd.INVALID_ARG
 
 
 # ---------------------------------------------------------------- seeded random shapes

@@ -271,6 +271,33 @@ def test_calibration_size_takes_the_next_most_important_evicted_tokens():
     np.testing.assert_array_equal(rc.calib_idx[0, 0], np.arange(k_sel, k_sel + 5))
 
 
+def test_other_eviction_rules_index_lists():
+    """StreamingLLM (sinks + recent) and H2O (half heavy hitters by accumulated attention, half recent):
+    the index rules against their plain definitions, the accumulated attention against a library softmax."""
+    # sinks + recent
+    np.testing.assert_array_equal(oracle.streaming_indices(100, 12, 4), [0, 1, 2, 3] + list(range(92, 100)))
+    np.testing.assert_array_equal(oracle.streaming_indices(10, 64, 32), np.arange(10))     # budget >= L keeps all
+    # heavy + local from scores: brute force with a stable numpy sort, planted ties
+    rng = np.random.Generator(np.random.Philox(key=[21, 1]))
+    sc = rng.random(200)
+    sc[[5, 17, 60]] = 0.99
+    sc[[3, 150]] = sc[40]                                   # ties with an unselected / a selected value
+    kept = oracle.select_from_scores(sc, tail=10, budget=30)
+    order = np.argsort(-sc[:190], kind="stable")[:20]
+    np.testing.assert_array_equal(kept, np.concatenate([np.sort(order), np.arange(190, 200)]))
+    # accumulated attention: column sums of the causal softmax (scipy), mass L per head, first query all on key 0
+    G, L, D = 2, 37, 128
+    Qf, K = rand_bits(rng, G, L, D), rand_bits(rng, L, D)
+    acc = oracle.accumulated_attention(Qf, K)
+    want = np.zeros(L)
+    for g in range(G):
+        s = f64(Qf[g]) @ f64(K).T / math.sqrt(D)
+        s[np.triu_indices(L, 1)] = -np.inf
+        want += softmax(s, axis=-1).sum(axis=0)
+    np.testing.assert_allclose(acc, want, atol=1e-12)
+    assert abs(acc.sum() - G * L) < 1e-9 and acc[0] >= G
+
+
 def test_calibrate_given_indices_agrees_and_uses_supplied_set():
     cfg = wl.small_config(L=100, window=8, budget=20)
     Q, (K, V) = wl.gen_q_obs(cfg), wl.gen_kv(cfg)

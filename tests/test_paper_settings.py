@@ -62,3 +62,18 @@ def test_oracle_with_the_papers_window_pool_and_budgets(budget):
     o = oracle.decode(q_far, None, None, r.K_kept.copy(), r.V_kept.copy(), budget, r.O_c, r.LSE_c, r.C_q,
                       theta1=s["theta1"][0], theta2=s["theta2"][0])
     assert np.all(o.flags & 1 == 0) and np.all(o.flags & 2 == 2)
+
+
+def test_other_baselines_settings_give_valid_kept_lists():
+    """StreamingLLM with the paper's 32 sinks and H2O with its even split, at the paper's budgets."""
+    s = _settings()
+    n_sink, frac = int(s["streamingllm_sinks"][0]), s["h2o_local_fraction"][0]
+    rng = np.random.Generator(np.random.Philox(key=[5, 5]))
+    for budget in (64, 128, 256, 512):
+        kept = oracle.streaming_indices(2000, budget, n_sink)
+        assert kept.size == budget and np.all(np.diff(kept) > 0)
+        assert np.array_equal(kept[:n_sink], np.arange(n_sink)) and kept[-1] == 1999 and kept[n_sink] == 2000 - (budget - n_sink)
+        tail = int(budget * frac)
+        kept = oracle.select_from_scores(rng.random(2000), tail=tail, budget=budget)
+        assert kept.size == budget and np.all(np.diff(kept) > 0)
+        assert np.array_equal(kept[budget - tail:], np.arange(2000 - tail, 2000)) and np.all(kept[:budget - tail] < 2000 - tail)
