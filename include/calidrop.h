@@ -20,8 +20,14 @@
  * Conventions
  *   - Unless a comment says HOST, every tensor pointer is a DEVICE pointer to a contiguous,
  *     16-byte aligned buffer on the current device.  "bf16" buffers hold bfloat16 values.
- *   - The library allocates nothing, owns nothing and keeps no pointer between calls.  All
- *     buffers, including the workspaces, belong to the caller.
+ *   - The library allocates nothing and owns no buffer: all of them, including the workspaces,
+ *     belong to the caller.  Two things outlast a call.  (1) calidrop_decode_static's built-in
+ *     scratch array (see there).  (2) Small per-thread and per-device tables of derived values:
+ *     whether a kernel's shared-memory attribute has been set on a device, the argument block of
+ *     the batched decode, and the TMA descriptors of the caches the decode entry points have
+ *     seen, keyed by the cache's addresses, capacity and unit count.  A descriptor is a pure
+ *     function of its key, so a table entry is never stale and is never dereferenced by the
+ *     library itself; freeing a cache needs no call into the library.
  *   - Every call validates its arguments on the host BEFORE enqueueing anything; a call that
  *     returns a non-zero status has had no effect.  Work is enqueued on `stream`
  *     (a cudaStream_t passed as void*; NULL is the default stream) and the call returns

@@ -392,8 +392,8 @@ decode_kernel(const __grid_constant__ DecodeArgsT<NL> args) {
 
   // One ring fill: rows [r0 + sb * 64, ...) of K and V into slot sb % 3.  Whole slots take four
   // 64-row boxes; the ragged last slot takes 16-row boxes for the row groups that hold valid rows,
-  // so a split never pulls more than 15 rows of its neighbour.  Rows at or beyond kv_len lie
-  // outside the tensor and arrive as zeros.
+  // so a split never pulls more than 15 rows of its neighbour.  Rows at or beyond n_kv (up to the
+  // cache's capacity) arrive as they lie in memory; the stream warps mask and clear them.
   auto fill = [&](int sb) {
     const int s = sb % kSlots, k = sb / kSlots;
     const uint32_t bar = smem_u32(&s_full[s][k & 1]);
@@ -533,8 +533,8 @@ decode_kernel(const __grid_constant__ DecodeArgsT<NL> args) {
       if (ok && row_base < r1) {
         const uint32_t sK = ring + s * kSlotBytes;
         const uint32_t sV = sK + 2 * kPlaneBytes;
-        // D1: the warp that meets row kv_len takes it from k_new / v_new (the cache row is
-        // outside the TMA tensor and arrived as zeros) and appends it to the cache
+        // D1: the warp that meets row kv_len takes it from k_new / v_new (the cache row has not
+        // been written yet: what arrived for it is stale) and appends it to the cache
         if (a.has_new && a.kv_len >= row_base && a.kv_len < row_base + kBlkRows) {
           const int chunk = lane & 15;
           const int rs = a.kv_len - (r0 + sb * kSlotRows);  // row inside the slot
@@ -546,6 +546,18 @@ decode_kernel(const __grid_constant__ DecodeArgsT<NL> args) {
           *reinterpret_cast<uint4*>(dstg) = v;
           *reinterpret_cast<uint4*>(ring_ptr + s * kSlotBytes + (lane < 16 ? 0 : 2 * kPlaneBytes) +
                                     plane_off(rs, chunk)) = v;
+          __syncwarp();
+        }
+        // The tensor maps cover the cache's whole capacity (so that they can be encoded once per
+        // cache and not once per call): the rows at or beyond n_kv of the last block hold whatever the
+        // caller's memory holds.  Their scores are masked below; their V rows are cleared here, since
+        // a zero probability times a NaN would still poison the product.
+        if (row_base + kBlkRows > r1 && r1 == a.n_kv) {
+          const int first_bad = r1 - (r0 + sb * kSlotRows);                 // row inside the slot
+          const int n_bad = (sub + 1) * kBlkRows - first_bad;               // 1..15 rows
+          for (int idx = lane; idx < n_bad * 16; idx += 32)
+            *reinterpret_cast<uint4*>(ring_ptr + s * kSlotBytes + 2 * kPlaneBytes +
+                                      plane_off(first_bad + (idx >> 4), idx & 15)) = make_uint4(0u, 0u, 0u, 0u);
           __syncwarp();
         }
         // S^T: two accumulators (even and odd k-steps) halve the dependent chain
@@ -769,15 +781,34 @@ decode_kernel(const __grid_constant__ DecodeArgsT<NL> args) {
 }  // namespace
 
 bool make_decode_maps(const DecodeCommon& c, const DecodeLayerPtrs& L, DecodeLayerMaps* out) {
-  // rows at or beyond kv_len are outside the tensor: the TMA unit delivers zeros for them
-  const uint64_t rows = (uint64_t)(c.kv_len > 0 ? c.kv_len : 1);
-  const uint64_t dims[2] = {rows, (uint64_t)c.units};
+  // The maps cover all `cap` rows of the cache, whatever kv_len is (the kernel masks and clears
+  // the rows beyond it), so one encoding serves every step on a cache.  Encoding the four maps
+  // costs more host time than the kernel runs; a small per-thread table keyed by everything the
+  // encoding depends on (the two base addresses, the capacity, the number of units) returns them
+  // on the following calls.  An entry can never be stale: equal keys encode equal maps.
+  struct Entry { const void* K; const void* V; int cap, units; DecodeLayerMaps maps; };
+  constexpr int kEntries = 64;
+  static thread_local Entry table[kEntries];
+  static thread_local int next = 0;
+  for (int i = 0; i < kEntries; ++i) {
+    const Entry& e = table[i];
+    if (e.K == L.K && e.V == L.V && e.cap == c.cap && e.units == c.units && e.K != nullptr) {
+      *out = e.maps;
+      return true;
+    }
+  }
+  const uint64_t dims[2] = {(uint64_t)c.cap, (uint64_t)c.units};
   const uint64_t strides[2] = {(uint64_t)kRowBytes, (uint64_t)c.cap * kRowBytes};
   const uint32_t box64[2] = {(uint32_t)kSlotRows, 1}, box16[2] = {(uint32_t)kBlkRows, 1};
-  return make_tensor_map_bf16(&out->k64, L.K, 3, dims, strides, box64) &&
-         make_tensor_map_bf16(&out->v64, L.V, 3, dims, strides, box64) &&
-         make_tensor_map_bf16(&out->k16, L.K, 3, dims, strides, box16) &&
-         make_tensor_map_bf16(&out->v16, L.V, 3, dims, strides, box16);
+  if (!(make_tensor_map_bf16(&out->k64, L.K, 3, dims, strides, box64) &&
+        make_tensor_map_bf16(&out->v64, L.V, 3, dims, strides, box64) &&
+        make_tensor_map_bf16(&out->k16, L.K, 3, dims, strides, box16) &&
+        make_tensor_map_bf16(&out->v16, L.V, 3, dims, strides, box16)))
+    return false;
+  Entry& e = table[next];
+  next = (next + 1) % kEntries;
+  e.K = L.K; e.V = L.V; e.cap = c.cap; e.units = c.units; e.maps = *out;
+  return true;
 }
 
 namespace {
