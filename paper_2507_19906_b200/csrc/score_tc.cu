@@ -29,7 +29,7 @@ namespace {
 
 using namespace tc;
 
-constexpr int kGroups = 2;  // consumer warpgroups (4 warps each); group g drains accumulator buffer g
+constexpr int kGroups = 4;  // consumer warpgroups (4 warps each), two pairs; pair p drains accumulator buffer p
 constexpr int kProducerWarp = kGroups * 4;
 constexpr int kMmaWarp = kGroups * 4 + 1;
 constexpr int kThreads = kGroups * 128 + 64;
@@ -91,10 +91,12 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
   constexpr int TILE_KEYS = kVotes ? 128 : 256;
   constexpr uint32_t STAGE_BYTES = TILE_KEYS * 256;
   extern __shared__ unsigned char smem_raw[];
-  __shared__ __align__(8) unsigned long long bars[18];
+  __shared__ __align__(8) unsigned long long bars[22];
   __shared__ uint32_t tmem_slot;
   __shared__ Ctl ctl;
-  __shared__ __align__(16) float nlse2_s[kVotes ? kGroups * 4 : 1][kVotes ? kMaxRows : 4];  // -lse2 per row, one copy per warp
+  // votes: -lse2 of the columns this warp reads (128 per row block at most), one copy per warp
+  __shared__ __align__(16) float nlse2_s[kVotes ? kGroups * 4 : 1][kVotes ? 256 : 4];
+  __shared__ float vx[2][128];  // votes: partial vote of the second column half, per pair
   __shared__ float2 ml_s[kVotes ? 1 : kGroups][kVotes ? 1 : 2][kVotes ? 1 : 128];       // running (max, sum)
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -118,6 +120,8 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
   auto empty_k = [&](int s) { return bar0 + 8u * (6 + s); };
   auto t_full = [&](int b) { return bar0 + 8u * (10 + b); };
   auto t_empty = [&](int b) { return bar0 + 8u * (14 + b); };
+  auto vx_full = [&](int b) { return bar0 + 8u * (18 + b); };
+  auto vx_empty = [&](int b) { return bar0 + 8u * (20 + b); };
 
   if (tid == 0) {
     ctl.abort = 0;
@@ -126,7 +130,8 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
     mbar_init(q_empty, 1);
     for (int s = 0; s < 4; ++s) { mbar_init(full_k(s), 1); mbar_init(empty_k(s), 1); }
     for (int b = 0; b < kNumBufs; ++b) {
-      mbar_init(t_full(b), 1); mbar_init(t_empty(b), 128);   // a buffer is drained by one warpgroup
+      mbar_init(t_full(b), 1); mbar_init(t_empty(b), 256);   // a buffer is drained by one pair of warpgroups
+      mbar_init(vx_full(b), 128); mbar_init(vx_empty(b), 128);
     }
     fence_mbar_init();
   }
@@ -215,15 +220,17 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
     }
   } else {
     // ------------------------------------------------------------ accumulator consumers
-    // Thread ct of warpgroup grp owns TMEM lane ct.  The jobs (key tile, row block) alternate between
-    // the groups: group g drains accumulator buffer g, i.e. every job whose index has parity g, all
-    // of its columns.  The groups therefore run half a job apart: while one waits for the MMAs of
-    // its next job, stores its result or starts its first load, the other keeps the exponential unit
-    // busy.  (Measured at config 3: both groups on the same job, half of the columns each, 110 us
-    // for the votes, the groups stalling together at every job boundary; alternating jobs 100 us;
-    // four accumulators of 128 columns, so that a group's next job is ready before it asks, 110 us:
-    // the narrower MMAs cost more than the wait they hide.)
+    // Thread ct of warpgroup grp owns TMEM lane ct.  The four groups form two pairs; the jobs (key
+    // tile, row block) alternate between the pairs: pair p drains accumulator buffer p, i.e. every
+    // job whose index has parity p, each of its two groups half of the columns.  The pairs run half
+    // a job apart: while one waits for the MMAs of its next job (which cannot start before the
+    // last columns of the current one have been read), the other, two warps per scheduler, keeps the
+    // exponential unit busy; one warp per scheduler alone reaches less than half of that unit's rate.
+    // (Measured at config 3, votes: two groups on the same job 110 us, the groups stalling together
+    // at every job boundary; two groups on alternate jobs 100 us; four accumulators of 128 columns
+    // 110 us, the narrower MMAs costing more than the wait they hide.)
     const int grp = warp >> 2, ct = tid & 127;
+    const int pair = grp >> 1, half = grp & 1;
     const uint32_t lane_base = tmem_base + ((uint32_t)((warp & 3) * 32) << 16);
     int cur_vu = -1, j = 0;
     bool ok = true;
@@ -254,9 +261,14 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
           // this warp's copy of -lse2 of the unit's window rows (-inf for the padding rows); warps
           // keep their own copy so that no barrier wider than a warp is needed here
           const int hq0 = (unit / Hkv) * a.Hq + (unit % Hkv) * a.G;
+          const int cwh = a.block_rows >> 1;   // this group's columns of a row block: [half * cwh, +cwh)
           __syncwarp();
-          for (int r = lane; r < kMaxRows; r += 32)
-            nlse2_s[warp][r] = r < a.GW ? -a.row_lse[(size_t)hq0 * a.W + r] * kLog2e : -INFINITY;
+          for (int idx = lane; idx < 256; idx += 32) {
+            const int blk = idx >> 7, c = idx & 127;
+            const int r = blk * a.block_rows + half * cwh + c;
+            nlse2_s[warp][idx] = (blk < a.n_blocks && c < cwh && r < a.GW) ? -a.row_lse[(size_t)hq0 * a.W + r] * kLog2e
+                                                                         : -INFINITY;
+          }
           __syncwarp();
         } else {
           if (cur_vu >= 0) flush_stats(cur_vu);
@@ -266,7 +278,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
       }
       const int tbase = tile * TILE_KEYS;
       for (int blk = 0; blk < a.n_blocks; ++blk, ++j) {
-        if ((j & 1) != grp) continue;
+        if ((j & 1) != pair) continue;
         const int buf = j & (kNumBufs - 1);
         const uint32_t lane_addr = lane_base + (uint32_t)(buf * kBufCols);
         ok = mbar_wait(&ctl, t_full(buf), (j / kNumBufs) & 1, (kVotes ? 35u : 15u) | ((unsigned)j << 8));
@@ -275,8 +287,9 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
         tc_fence_after_sync();
         uint32_t ra[32], rb[32];
         if (kVotes) {
-          const int cw = a.block_rows;  // columns (query rows) of the job: a multiple of 64
-          const float* nl = nlse2_s[warp] + blk * a.block_rows;
+          const int cw = a.block_rows >> 1;  // columns (query rows) of this group: a multiple of 32
+          const float* nl = nlse2_s[warp] + blk * 128;
+          const uint32_t tcol = lane_addr + (uint32_t)(half * cw);
           float acc0 = 0.f, acc1 = 0.f, acc2 = 0.f, acc3 = 0.f;  // running vote of this thread's key
           auto add32 = [&](const uint32_t (&r)[32], int c0) {
 #pragma unroll
@@ -288,29 +301,44 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
               acc3 += ex2_approx(fmaf(__uint_as_float(r[e + 3]), a.scale2, n4.w));
             }
           };
-          // chunks of 32 columns alternate between the two register sets
-          tmem_ld32_issue(lane_addr, ra);
+          // chunks of 32 columns alternate between the two register sets (cw is a multiple of 32)
+          tmem_ld32_issue(tcol, ra);
 #pragma unroll 1
           for (int c0 = 0; c0 < cw; c0 += 64) {
             tmem_ld_wait(ra);
-            tmem_ld32_issue(lane_addr + c0 + 32, rb);
+            const bool more_b = c0 + 32 < cw;
+            if (more_b) tmem_ld32_issue(tcol + c0 + 32, rb);
+            else { tc_fence_before_sync(); mbar_arrive(t_empty(buf)); }   // all of it is in registers
             add32(ra, c0);
-            tmem_ld_wait(rb);
-            if (c0 + 64 < cw) {
-              tmem_ld32_issue(lane_addr + c0 + 64, ra);
-            } else {
-              tc_fence_before_sync();
-              mbar_arrive(t_empty(buf));  // the accumulator is in registers: hand the buffer back early
+            if (more_b) {
+              tmem_ld_wait(rb);
+              if (c0 + 64 < cw) tmem_ld32_issue(tcol + c0 + 64, ra);
+              else { tc_fence_before_sync(); mbar_arrive(t_empty(buf)); }
+              add32(rb, c0 + 32);
             }
-            add32(rb, c0 + 32);
           }
-          // the vote of the key over this group's row blocks of the tile; stored after the last of them
-          vsum += (acc0 + acc1) + (acc2 + acc3);
-          if (blk + 2 >= a.n_blocks) {
-            const int key = tbase + ct;
-            float* out = (a.n_blocks > 1 && grp == 1) ? a.vote2 : a.vote;
-            if (key < a.n_cand) out[(size_t)unit * a.n_cand + key] = vsum;
-            vsum = 0.f;
+          // the two halves of the key's vote meet in shared memory; the first group stores the sum
+          const float part = (acc0 + acc1) + (acc2 + acc3);
+          const int jp = j >> 1;   // index of the job among this pair's jobs
+          if (half == 1) {
+            ok = mbar_wait(&ctl, vx_empty(pair), (jp & 1) ^ 1, 37u | ((unsigned)j << 8));
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+            vx[pair][ct] = part;
+            mbar_arrive(vx_full(pair));
+          } else {
+            ok = mbar_wait(&ctl, vx_full(pair), jp & 1, 38u | ((unsigned)j << 8));
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+            vsum += part + vx[pair][ct];
+            mbar_arrive(vx_empty(pair));
+            // the vote of the key over this pair's row blocks of the tile; stored after the last of them
+            if (blk + 2 >= a.n_blocks) {
+              const int key = tbase + ct;
+              float* out = (a.n_blocks > 1 && pair == 1) ? a.vote2 : a.vote;
+              if (key < a.n_cand) out[(size_t)unit * a.n_cand + key] = vsum;
+              vsum = 0.f;
+            }
           }
         } else {
           float2 ml = ml_s[grp][blk][ct];
@@ -330,14 +358,15 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
               ml.x = m_new;
             }
           };
-          tmem_ld32_issue(lane_addr, ra);
+          const int cbeg = half * (TILE_KEYS / 2), cend = cbeg + TILE_KEYS / 2;  // this group's keys of the tile
+          tmem_ld32_issue(lane_addr + cbeg, ra);
 #pragma unroll 1
-          for (int c0 = 0; c0 < TILE_KEYS; c0 += 64) {
+          for (int c0 = cbeg; c0 < cend; c0 += 64) {
             tmem_ld_wait(ra);
             tmem_ld32_issue(lane_addr + c0 + 32, rb);
             fold32(ra, c0);
             tmem_ld_wait(rb);
-            if (c0 + 64 < TILE_KEYS) {
+            if (c0 + 64 < cend) {
               tmem_ld32_issue(lane_addr + c0 + 64, ra);
             } else {
               tc_fence_before_sync();

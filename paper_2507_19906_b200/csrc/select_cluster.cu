@@ -25,8 +25,8 @@ constexpr int kClu = 8;
 constexpr int kT = 1024;
 constexpr int kW = kT / 32;
 
-template <int ROWS>
-__global__ void __cluster_dims__(kClu, 1, 1) __launch_bounds__(kT)
+template <int ROWS, bool kSized>
+__global__ void __cluster_dims__(kClu, 1, 1) __launch_bounds__(kT, ROWS <= 8 ? 2 : 1)  // two CTAs per SM where many units make more CTAs than SMs
 pool_select_cluster_kernel(const float* __restrict__ vote, float* __restrict__ pooled,
                            uint32_t* __restrict__ bitmap, int32_t* __restrict__ kept_idx, int n_cand, int L,
                            int pool, int k_sel, int n_kept, int bitmap_words, uint32_t* __restrict__ mask2,
@@ -71,7 +71,7 @@ pool_select_cluster_kernel(const float* __restrict__ vote, float* __restrict__ p
   // 2. radix select, most significant byte first; the histograms of the eight CTAs are summed
   // through distributed shared memory.  Returns the bit pattern T of the kk-th largest pooled vote
   // and how many candidates equal to T are still taken (those at the lowest positions).
-  auto radix_select = [&](unsigned kk, unsigned& T_out, unsigned& need_out) {
+  auto radix_select = [&](unsigned kk, unsigned& T_out, unsigned& need_out) __attribute__((always_inline)) {
     unsigned prefix = 0, k = kk;
     for (int pass = 0; pass < 4; ++pass) {
       const int shift = 24 - 8 * pass;
@@ -137,7 +137,7 @@ pool_select_cluster_kernel(const float* __restrict__ vote, float* __restrict__ p
   // above / equal to the threshold that precede it.
   unsigned gt_mask[ROWS], eq_mask[ROWS];
   unsigned before_gt = 0, before_eq = 0;  // keys of the lower-ranked CTAs
-  auto scan_threshold = [&](unsigned Tx, int slot) {
+  auto scan_threshold = [&](unsigned Tx, int slot) __attribute__((always_inline)) {
 #pragma unroll
     for (int i = 0; i < ROWS; ++i) {
       const int t = rank * chunk + i * kT + tid;
@@ -179,7 +179,7 @@ pool_select_cluster_kernel(const float* __restrict__ vote, float* __restrict__ p
   };
   // is key (row i, this thread) among the first `need` keys equal to Tx or above Tx ?
   const unsigned lt = (1u << lane) - 1u;
-  auto taken = [&](int i, unsigned Tx, unsigned need) {
+  auto taken = [&](int i, unsigned Tx, unsigned need) __attribute__((always_inline)) {
     const unsigned eq_before = before_eq + wsum[i * kW + warp][1] + __popc(eq_mask[i] & lt);
     return key[i] > Tx || (key[i] == Tx && eq_before < need);
   };
@@ -209,7 +209,7 @@ pool_select_cluster_kernel(const float* __restrict__ vote, float* __restrict__ p
 
   // 4. calibration size: the next n_calib candidates in the same order, i.e. those among the first
   // k_sel + n_calib that were not selected.  mask2: bit set = the row is NOT one of them.
-  if (mask2) {
+  if (kSized) {
     uint32_t* bm2 = mask2 + (size_t)unit * bitmap_words;
     unsigned T2, need2;
     __syncthreads();   // wsum and the flags of step 3 have been read by every thread of this CTA
@@ -230,10 +230,14 @@ pool_select_cluster_kernel(const float* __restrict__ vote, float* __restrict__ p
 template <int ROWS>
 void launch_rows(const CompressGeom& g, const CompressWs& ws, char* wsp, const float* scores, size_t stride,
                  int32_t* kept_idx, cudaStream_t st) {
-  pool_select_cluster_kernel<ROWS><<<dim3(kClu, g.units), kT, 0, st>>>(
-      scores, (float*)(wsp + ws.pooled), (uint32_t*)(wsp + ws.bitmap), kept_idx, g.n_cand,
-      g.L, g.pool, g.k_sel, g.n_kept, g.bitmap_words, (g.sized && g.n_calib > 0) ? (uint32_t*)(wsp + ws.bitmap2) : nullptr,
-      g.n_calib, stride);
+  if (g.sized && g.n_calib > 0)
+    pool_select_cluster_kernel<ROWS, true><<<dim3(kClu, g.units), kT, 0, st>>>(
+        scores, (float*)(wsp + ws.pooled), (uint32_t*)(wsp + ws.bitmap), kept_idx, g.n_cand, g.L, g.pool, g.k_sel,
+        g.n_kept, g.bitmap_words, (uint32_t*)(wsp + ws.bitmap2), g.n_calib, stride);
+  else
+    pool_select_cluster_kernel<ROWS, false><<<dim3(kClu, g.units), kT, 0, st>>>(
+        scores, (float*)(wsp + ws.pooled), (uint32_t*)(wsp + ws.bitmap), kept_idx, g.n_cand, g.L, g.pool, g.k_sel,
+        g.n_kept, g.bitmap_words, nullptr, 0, stride);
 }
 
 }  // namespace
