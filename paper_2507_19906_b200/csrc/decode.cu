@@ -392,8 +392,10 @@ decode_kernel(const __grid_constant__ DecodeArgsT<NL> args) {
 
   // One ring fill: rows [r0 + sb * 64, ...) of K and V into slot sb % 3.  Whole slots take four
   // 64-row boxes; the ragged last slot takes 16-row boxes for the row groups that hold valid rows,
-  // so a split never pulls more than 15 rows of its neighbour.  Rows at or beyond n_kv (up to the
-  // cache's capacity) arrive as they lie in memory; the stream warps mask and clear them.
+  // so a split never pulls more than 15 rows of its neighbour.  Only a 16-row box can reach past
+  // row kv_len: the V map of those boxes ends at kv_len, so such V rows arrive as zeros (a zero
+  // probability times whatever lies in the caller's memory could still be a NaN); the K rows
+  // arrive as they lie in memory and their scores are masked.
   auto fill = [&](int sb) {
     const int s = sb % kSlots, k = sb / kSlots;
     const uint32_t bar = smem_u32(&s_full[s][k & 1]);
@@ -546,18 +548,6 @@ decode_kernel(const __grid_constant__ DecodeArgsT<NL> args) {
           *reinterpret_cast<uint4*>(dstg) = v;
           *reinterpret_cast<uint4*>(ring_ptr + s * kSlotBytes + (lane < 16 ? 0 : 2 * kPlaneBytes) +
                                     plane_off(rs, chunk)) = v;
-          __syncwarp();
-        }
-        // The tensor maps cover the cache's whole capacity (so that they can be encoded once per
-        // cache and not once per call): the rows at or beyond n_kv of the last block hold whatever the
-        // caller's memory holds.  Their scores are masked below; their V rows are cleared here, since
-        // a zero probability times a NaN would still poison the product.
-        if (row_base + kBlkRows > r1 && r1 == a.n_kv) {
-          const int first_bad = r1 - (r0 + sb * kSlotRows);                 // row inside the slot
-          const int n_bad = (sub + 1) * kBlkRows - first_bad;               // 1..15 rows
-          for (int idx = lane; idx < n_bad * 16; idx += 32)
-            *reinterpret_cast<uint4*>(ring_ptr + s * kSlotBytes + 2 * kPlaneBytes +
-                                      plane_off(first_bad + (idx >> 4), idx & 15)) = make_uint4(0u, 0u, 0u, 0u);
           __syncwarp();
         }
         // S^T: two accumulators (even and odd k-steps) halve the dependent chain
@@ -781,29 +771,32 @@ decode_kernel(const __grid_constant__ DecodeArgsT<NL> args) {
 }  // namespace
 
 bool make_decode_maps(const DecodeCommon& c, const DecodeLayerPtrs& L, DecodeLayerMaps* out) {
-  // The maps cover all `cap` rows of the cache, whatever kv_len is (the kernel masks and clears
-  // the rows beyond it), so one encoding serves every step on a cache.  Encoding the four maps
-  // costs more host time than the kernel runs; a small per-thread table keyed by everything the
-  // encoding depends on (the two base addresses, the capacity, the number of units) returns them
-  // on the following calls.  An entry can never be stale: equal keys encode equal maps.
+  // Three of the four maps cover all `cap` rows of the cache, whatever kv_len is, so one encoding
+  // serves every step on a cache: a small per-thread table keyed by everything the encoding depends
+  // on (the two base addresses, the capacity, the number of units) returns them on the following
+  // calls (encoding all four on every call cost more host time than the kernel runs).  An entry can
+  // never be stale: equal keys encode equal maps.  The fourth, V in 16-row boxes, is the only one
+  // through which rows at or beyond kv_len can reach a product; it ends at kv_len, so the TMA unit
+  // delivers zeros for those rows, and is encoded per call.
   struct Entry { const void* K; const void* V; int cap, units; DecodeLayerMaps maps; };
   constexpr int kEntries = 64;
   static thread_local Entry table[kEntries];
   static thread_local int next = 0;
+  const uint64_t strides[2] = {(uint64_t)kRowBytes, (uint64_t)c.cap * kRowBytes};
+  const uint32_t box64[2] = {(uint32_t)kSlotRows, 1}, box16[2] = {(uint32_t)kBlkRows, 1};
+  const uint64_t dims_v16[2] = {(uint64_t)(c.kv_len > 0 ? c.kv_len : 1), (uint64_t)c.units};
   for (int i = 0; i < kEntries; ++i) {
     const Entry& e = table[i];
     if (e.K == L.K && e.V == L.V && e.cap == c.cap && e.units == c.units && e.K != nullptr) {
       *out = e.maps;
-      return true;
+      return make_tensor_map_bf16(&out->v16, L.V, 3, dims_v16, strides, box16);
     }
   }
   const uint64_t dims[2] = {(uint64_t)c.cap, (uint64_t)c.units};
-  const uint64_t strides[2] = {(uint64_t)kRowBytes, (uint64_t)c.cap * kRowBytes};
-  const uint32_t box64[2] = {(uint32_t)kSlotRows, 1}, box16[2] = {(uint32_t)kBlkRows, 1};
   if (!(make_tensor_map_bf16(&out->k64, L.K, 3, dims, strides, box64) &&
         make_tensor_map_bf16(&out->v64, L.V, 3, dims, strides, box64) &&
         make_tensor_map_bf16(&out->k16, L.K, 3, dims, strides, box16) &&
-        make_tensor_map_bf16(&out->v16, L.V, 3, dims, strides, box16)))
+        make_tensor_map_bf16(&out->v16, L.V, 3, dims_v16, strides, box16)))
     return false;
   Entry& e = table[next];
   next = (next + 1) % kEntries;

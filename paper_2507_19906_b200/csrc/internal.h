@@ -46,8 +46,9 @@ struct DecodeLayerPtrs {
   uint8_t* flags;
 };
 
-// TMA views of one layer's retained cache, [unit][row < kv_len][128] bf16 with 128-byte swizzle:
-// boxes of 64 rows for whole ring slots and of 16 rows for the ragged end of a split.
+// TMA views of one layer's retained cache, [unit][row][128] bf16 with 128-byte swizzle: boxes of
+// 64 rows for whole ring slots and of 16 rows for the ragged end of a split.  k64, v64 and k16 span
+// the cache's capacity; v16 ends at row kv_len (rows beyond it arrive as zeros).
 struct alignas(64) DecodeLayerMaps {
   CUtensorMap k64, v64, k16, v16;
 };
