@@ -14,14 +14,18 @@
 // every p <= 1 and no running maximum or rescaling is needed: the partial (O, l) of the key ranges
 // simply add up.  calib_reduce_kernel sums them in a fixed order and writes O_c = O / l,
 // LSE_c = lse + log l, C_q.
-// Warp roles: two softmax warpgroups (group g owns S buffer g and P buffer g, i.e. the tiles with
-// local index i % 2 == g), two TMA producer warps (Q_c and K; V), and two MMA-issuing warps, one for
-// S and one for P.V: a single thread's dependent scalar instructions cost several cycles each, and
-// with the waits and commits of both chains on one thread the issue, not the tensor pipe, set the
-// pace (a lone chain of eight 128x128x16 MMAs runs at the pipe's 64 cycles each once its descriptors
-// are prepared; no interleaving of chains is needed).  S(i+2) is issued as soon as S(i) has been read
-// out of the buffer they share, not when P(i) is complete.
-// Tensor memory: S buffers at columns 0 and 128, O at 256, P buffers (64 columns each) at 384, 448.
+// Warp roles: two softmax warpgroups (group g takes the tiles with local index i % 2 == g), two TMA
+// producer warps (Q_c and K; V), and two MMA-issuing warps, one for S and one for P.V: a single
+// thread's dependent scalar instructions cost several cycles each, and with the waits and commits of
+// both chains on one thread the issue, not the tensor pipe, set the pace (a lone chain of eight
+// 128x128x16 MMAs runs at the pipe's 64 cycles each once its descriptors are prepared; no
+// interleaving of chains is needed).
+// Tensor memory: three S/P buffers of 128 columns at 0, 128, 256 and O at 384.  Tile i lives in buffer
+// i % 3: S(i) arrives there, and its probabilities, rounded to bf16, overwrite the first 64 columns in
+// place (a thread stores the P of 32 keys only after the S of those columns is in its registers).  A
+// buffer is free again when the P.V that read it has completed; with three of them S(i+2) is ready
+// when its group has finished tile i, and a group never waits for the P.V of its own previous tile
+// (with two S buffers and a P buffer per group it did, for about a third of its time).
 #include <type_traits>
 
 #include "internal.h"
@@ -40,8 +44,9 @@ constexpr int kPvWarp = kGroups * 4 + 2;         // issues the P.V MMAs
 constexpr int kVProducerWarp = kGroups * 4 + 3;  // TMA: V tiles
 constexpr int kThreads = kGroups * 128 + 128;
 constexpr int kTmemCols = 512;
-constexpr uint32_t kColO = 256, kColP = 384;
-constexpr int kStages = 3;                 // K ring and V ring alike
+constexpr int kBufs = 3;                   // S/P buffers of 128 columns
+constexpr uint32_t kColO = kBufs * 128;
+constexpr int kStages = kBufs;             // K ring and V ring: slot t % 3 feeds buffer t % 3
 constexpr int kTileBytes = kKvTileBytes;   // 32 KB
 constexpr int kSmemBytes = (1 + 2 * kStages) * kTileBytes + 1024;  // Q_c block, K ring, V ring
 constexpr int kSms = 148;
@@ -65,7 +70,7 @@ __global__ void __launch_bounds__(kThreads, 1)
 calib_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__ CUtensorMap k_map,
                 const __grid_constant__ CUtensorMap v_map, const CalibArgs a) {
   extern __shared__ unsigned char smem_raw[];
-  __shared__ __align__(8) unsigned long long bars[24];
+  __shared__ __align__(8) unsigned long long bars[26];
   __shared__ uint32_t tmem_slot;
   __shared__ Ctl ctl;
 
@@ -86,15 +91,12 @@ calib_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
   unsigned char* const smem_al = smem_raw + (smem_base - smem_u32(smem_raw));
 
   const uint32_t bar0 = smem_u32(bars);
-  const uint32_t o_full = bar0, o_empty = bar0 + 8u, q_full = bar0 + 144u, q_empty = bar0 + 152u;
+  const uint32_t o_full = bar0, o_empty = bar0 + 8u, q_full = bar0 + 8u * 23, q_empty = bar0 + 8u * 24;
   auto full_k = [&](int s) { return bar0 + 8u * (2 + s); };
-  auto empty_k = [&](int s) { return bar0 + 8u * (5 + s); };
   auto full_v = [&](int s) { return bar0 + 8u * (8 + s); };
-  auto empty_v = [&](int s) { return bar0 + 8u * (11 + s); };
   auto s_full = [&](int b) { return bar0 + 8u * (14 + b); };
-  auto p_full = [&](int b) { return bar0 + 8u * (16 + b); };
-  auto s_free = [&](int b) { return bar0 + 8u * (20 + b); };    // S buffer b has been read into registers
-  auto p_empty = [&](int b) { return bar0 + 8u * (22 + b); };   // the P.V that read P buffer b has completed
+  auto p_full = [&](int b) { return bar0 + 8u * (17 + b); };
+  auto buf_free = [&](int b) { return bar0 + 8u * (20 + b); };  // the P.V that read buffer b has completed
 
   if (tid == 0) {
     ctl.abort = 0;
@@ -104,12 +106,11 @@ calib_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
     mbar_init(q_full, 1);
     mbar_init(q_empty, 1);
     for (int s = 0; s < kStages; ++s) {
-      mbar_init(full_k(s), 1); mbar_init(empty_k(s), 1);
-      mbar_init(full_v(s), 1); mbar_init(empty_v(s), 1);
+      mbar_init(full_k(s), 1);
+      mbar_init(full_v(s), 1);
     }
-    for (int b = 0; b < 2; ++b) {
-      mbar_init(s_full(b), 1); mbar_init(p_full(b), 128);
-      mbar_init(s_free(b), 128); mbar_init(p_empty(b), 1);
+    for (int b = 0; b < kBufs; ++b) {
+      mbar_init(s_full(b), 1); mbar_init(p_full(b), 128); mbar_init(buf_free(b), 1);
     }
     fence_mbar_init();
   }
@@ -130,8 +131,6 @@ calib_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
   // (the position inside the tile space is tracked incrementally: no division per tile)
   const int unit_begin = g_begin / a.n_tiles, tile_begin = g_begin - unit_begin * a.n_tiles;
   const int vu_begin = unit_begin * a.n_cblocks + cb;
-  auto seg_first = [&](int i, int tile) { return i == 0 || tile == 0; };
-  auto seg_last = [&](int i, int tile) { return i == nt - 1 || tile == a.n_tiles - 1; };
 
   if (warp == kProducerWarp) {
     // ------------------------------------------------------------ TMA producer of Q_c and K
@@ -143,7 +142,7 @@ calib_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
       int seg = 0, vu = vu_begin, tile = tile_begin, unit = unit_begin;
       for (int i = 0; i < nt; ++i, ++tile) {
         if (tile == a.n_tiles) { tile = 0; ++unit; vu += a.n_cblocks; }
-        if (seg_first(i, tile)) {
+        if (i == 0 || tile == 0) {
           // the Q_c block of the next virtual unit replaces the current one once its MMAs are done
           if (seg > 0 && !mbar_wait(&ctl, q_empty, (seg - 1) & 1, 20u | ((unsigned)i << 8))) break;
           const int g0 = (vu - unit * a.n_cblocks) * a.gpb;
@@ -153,7 +152,8 @@ calib_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
           ++seg;
         }
         const int s = i % kStages;
-        if (!mbar_wait(&ctl, empty_k(s), ((i / kStages) & 1) ^ 1, 21u | ((unsigned)i << 8))) break;
+        // slot s is free when S(i-3), which read it, is done: the barrier that hands S to the softmax group
+        if (!mbar_wait(&ctl, s_full(s), ((i / kStages) & 1) ^ 1, 21u | ((unsigned)i << 8))) break;
         mbar_arrive_expect_tx(full_k(s), kTileBytes);
         for (int half = 0; half < 2; ++half)
           tma_load_3d(k_base + s * kTileBytes + half * (kTileBytes / 2), &k_map, full_k(s), half * kHalfCols,
@@ -168,7 +168,8 @@ calib_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
       for (int i = 0; i < nt; ++i, ++tile) {
         if (tile == a.n_tiles) { tile = 0; ++unit; }
         const int s = i % kStages;
-        if (!mbar_wait(&ctl, empty_v(s), ((i / kStages) & 1) ^ 1, 22u | ((unsigned)i << 8))) break;
+        // slot s is free when the P.V of tile i-3 is done: the barrier that frees its S/P buffer
+        if (!mbar_wait(&ctl, buf_free(s), ((i / kStages) & 1) ^ 1, 22u | ((unsigned)i << 8))) break;
         mbar_arrive_expect_tx(full_v(s), kTileBytes);
         for (int half = 0; half < 2; ++half)
           tma_load_3d(v_base + s * kTileBytes + half * (kTileBytes / 2), &v_map, full_v(s), half * kHalfCols,
@@ -183,50 +184,44 @@ calib_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
     // for a single thread (measured: 2900 cycles a tile against 1024 of tensor-pipe time, the softmax
     // groups waiting for S half of the time).  The two chains touch different accumulators; what
     // orders them is the barriers, not the issue order.
-    // S(t) goes into buffer t % 2 as soon as S(t-2) has been read out of it (s_free), which is well
-    // before P(t-2) is complete.  S never runs ahead across a change of virtual unit: its Q_c block
-    // is only loaded once the current unit's S MMAs are done.
+    // S(t) goes into buffer t % 3 as soon as the P.V of tile t-3 has completed (buf_free).  S never
+    // runs ahead across a change of virtual unit: its Q_c block is only loaded once the current unit's
+    // S MMAs are done.
     if (lane == 0) {
       const uint32_t idesc = umma_idesc(128, 128, false, false);     // S: A = Q_c, B = K tile, K-major
       // Descriptors are built once per buffer and a k-step adds a constant to the address field: the
       // issuing thread's own instructions between two MMAs are what limits the issue rate.
       const uint64_t dq = smem_desc_sw128(q_base, 16u, 1024u);
       const uint64_t dk0 = smem_desc_sw128(k_base, 16u, 1024u);
-      int seg = 0;
-      bool ok = true;
-      // S(t): wait for its buffer and its K tile, eight k-steps, then tell the softmax group and
-      // the producer
-      auto issue_s = [&](int t) -> bool {
-        if (t >= 2 && !mbar_wait(&ctl, s_free(t & 1), ((t - 2) >> 1) & 1, 29u | ((unsigned)t << 8))) return false;
-        if (!mbar_wait(&ctl, full_k(t % kStages), (t / kStages) & 1, 24u | ((unsigned)t << 8))) return false;
+      // The loop is kept short on purpose: between two tiles this one thread runs dependent scalar
+      // instructions at several cycles each, and whatever it spends there the tensor pipe idles.
+      // b = t % 3 is the tile's buffer and its K slot, ph = (t / 3) & 1 their phase.
+      int seg = 0, tile = tile_begin, b = 0;
+      uint32_t ph = 0;
+      bool first = true;
+      for (int t = 0; t < nt; ++t) {
+        if (first) {
+          // new virtual unit: its Q_c block must have landed
+          if (!mbar_wait(&ctl, q_full, seg & 1, 23u | ((unsigned)t << 8))) break;
+          ++seg;
+        }
+        if (t >= kBufs && !mbar_wait(&ctl, buf_free(b), ph ^ 1u, 29u | ((unsigned)t << 8))) break;
+        if (!mbar_wait(&ctl, full_k(b), ph, 24u | ((unsigned)t << 8))) break;
         tc_fence_after_sync();
-        const uint32_t d = tmem_base + (uint32_t)((t & 1) * 128);
-        const uint64_t kd = desc_advance(dk0, (uint32_t)(t % kStages) * kTileBytes);
+        const uint32_t d = tmem_base + (uint32_t)(b * 128);
+        const uint64_t kd = desc_advance(dk0, (uint32_t)b * kTileBytes);
         umma_ss_imm<0>(d, dq, kd, idesc);
 #pragma unroll
         for (int kk = 1; kk < kD / 16; ++kk)
           umma_ss_imm<1>(d, desc_advance(dq, kmajor_step_bytes(kTileBytes / 2, kk)),
                          desc_advance(kd, kmajor_step_bytes(kTileBytes / 2, kk)), idesc);
-        umma_commit(s_full(t & 1));
-        umma_commit(empty_k(t % kStages));
-        return true;
-      };
-      int tile = tile_begin;
-      for (int i = 0; ok && i < nt; ++i, ++tile) {
-        if (tile == a.n_tiles) tile = 0;
-        const bool first = seg_first(i, tile), last = seg_last(i, tile);
-        if (first) {
-          // new virtual unit: its Q_c block must have landed; S(i) and S(i+1) open the unit
-          ok = mbar_wait(&ctl, q_full, seg & 1, 23u | ((unsigned)i << 8));
-          ++seg;
-          if (!ok) break;
-          ok = issue_s(i) && (last || issue_s(i + 1));
-          if (!ok) break;
-        }
-        // S(i+2) when that tile belongs to the same virtual unit
-        if (!last && !seg_last(i + 1, tile + 1)) ok = issue_s(i + 2);
+        umma_commit(s_full(b));   // to the softmax group, and to the K producer: the slot is free
+        ++tile;
+        first = tile == a.n_tiles;
+        if (first) tile = 0;
         // every S of the unit has been issued by its last tile: Q_c may be replaced once they are done
-        if (last) umma_commit(q_empty);
+        if (first || t == nt - 1) umma_commit(q_empty);
+        if (++b == kBufs) { b = 0; ph ^= 1u; }
       }
     }
   } else if (warp == kPvWarp) {
@@ -234,48 +229,49 @@ calib_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
     if (lane == 0) {
       const uint32_t idesc_o = umma_idesc(128, 128, false, true);    // O: A = P (TMEM), B = V tile, MN-major
       const uint32_t tmem_o = tmem_base + kColO;
-      const uint32_t tmem_p = tmem_base + kColP;
       // V tile with the keys as K, i.e. MN-major: blocks of 64 head-dim elements are half a tile
       // apart, groups of 8 keys 1024 bytes apart
       const uint64_t dv0 = smem_desc_sw128(v_base, kTileBytes / 2, 1024u);
       // P.V(i): A = P in tensor memory, 16 keys = 8 columns per step
-      auto pv_steps = [&](int i, auto first_tag) {
+      auto pv_steps = [&](int b, auto first_tag) {
         constexpr bool kFirst = decltype(first_tag)::value;
-        const uint64_t vd = desc_advance(dv0, (uint32_t)(i % kStages) * kTileBytes);
-        const uint32_t pa = tmem_p + (uint32_t)((i & 1) * 64);
+        const uint64_t vd = desc_advance(dv0, (uint32_t)b * kTileBytes);
+        const uint32_t pa = tmem_base + (uint32_t)(b * 128);
         if (kFirst) umma_ts_imm<0>(tmem_o, pa, vd, idesc_o);
         else umma_ts_imm<1>(tmem_o, pa, vd, idesc_o);
 #pragma unroll
         for (int kk = 1; kk < kTileKeys / 16; ++kk)
           umma_ts_imm<1>(tmem_o, pa + (uint32_t)(kk * 8), desc_advance(vd, (uint32_t)kk * 16u * kLineBytes), idesc_o);
       };
-      int seg = 0, tile = tile_begin;
-      for (int i = 0; i < nt; ++i, ++tile) {
-        if (tile == a.n_tiles) tile = 0;
-        const bool first = seg_first(i, tile), last = seg_last(i, tile);
+      int seg = 0, tile = tile_begin, b = 0;
+      uint32_t ph = 0;
+      bool first = true;
+      for (int i = 0; i < nt; ++i) {
         if (first) {
           // O of the previous unit must have been read out before the first P.V overwrites it
           if (seg > 0 && !mbar_wait(&ctl, o_empty, (seg - 1) & 1, 25u | ((unsigned)i << 8))) break;
           ++seg;
         }
-        if (!mbar_wait(&ctl, p_full(i & 1), (i >> 1) & 1, 26u | ((unsigned)i << 8))) break;
-        if (!mbar_wait(&ctl, full_v(i % kStages), (i / kStages) & 1, 27u | ((unsigned)i << 8))) break;
+        if (!mbar_wait(&ctl, p_full(b), ph, 26u | ((unsigned)i << 8))) break;
+        if (!mbar_wait(&ctl, full_v(b), ph, 27u | ((unsigned)i << 8))) break;
         tc_fence_after_sync();
-        if (first) pv_steps(i, std::true_type{});
-        else pv_steps(i, std::false_type{});
-        umma_commit(p_empty(i & 1));
-        umma_commit(empty_v(i % kStages));
-        if (last) umma_commit(o_full);
+        if (first) pv_steps(b, std::true_type{});
+        else pv_steps(b, std::false_type{});
+        umma_commit(buf_free(b));   // to the S issuer, and to the V producer: the slot is free
+        ++tile;
+        first = tile == a.n_tiles;
+        if (first) tile = 0;
+        if (first || i == nt - 1) umma_commit(o_full);
+        if (++b == kBufs) { b = 0; ph ^= 1u; }
       }
     }
   } else {
     // ------------------------------------------------------------ softmax threads (one row each)
     const int grp = warp >> 2, r = tid & 127;
     const uint32_t lane_bits = (uint32_t)((warp & 3) * 32) << 16;
-    const uint32_t taddr = tmem_base + lane_bits + (uint32_t)(grp * 128);  // this group's S buffer
-    const uint32_t paddr = tmem_base + lane_bits + kColP + (uint32_t)(grp * 64);  // and its P buffer
+    const uint32_t lane_addr = tmem_base + lane_bits;
     float l0 = 0.f, l1 = 0.f, nlse2 = -INFINITY;
-    int cur_vu = -1, seg = 0;
+    int seg = 0;
     bool ok = true, valid = false;
 
     // Read out O and the row sums of the virtual unit that just ended (each group half of O's
@@ -318,94 +314,108 @@ calib_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
     };
 
     const uint32_t* bm_all = a.bitmap;
-    // The four bitmap words of a tile are loaded RAW (nothing may touch a loaded value before the
-    // tile that uses it, or the thread waits for the load on the spot); the mask of the keys outside
-    // the candidates is worked out separately from the indices.
-    auto load_words = [&](int unit, int tile, uint32_t (&raw)[4], uint32_t (&msk)[4]) {
+    const int last_word = a.bitmap_words - 1;
+    // The four kept-key words of a tile (bit set = the key does not contribute) are loaded RAW one
+    // own tile ahead: nothing may touch a loaded value before the tile that uses it, or the thread
+    // waits for the load on the spot.  The index is clamped so that the load is always valid.
+    auto load_words = [&](int unit, int tile, uint32_t (&raw)[4]) {
       const uint32_t* bm = bm_all + (size_t)unit * a.bitmap_words;
+      const int w0 = tile * (kTileKeys / 32);
+#pragma unroll
+      for (int q = 0; q < 4; ++q) raw[q] = __ldg(bm + min(w0 + q, last_word));
+    };
+    // keys at or beyond n_cand do not contribute either; only a unit's last tile has any
+    auto tail_mask = [&](int tile, uint32_t (&w)[4]) {
       const int tbase = tile * kTileKeys;
 #pragma unroll
       for (int q = 0; q < 4; ++q) {
         const int kb = tbase + 32 * q;
-        raw[q] = __ldg(bm + min(kb >> 5, a.bitmap_words - 1));   // always a valid word; the mask decides
-        msk[q] = kb >= a.n_cand ? 0xffffffffu : (kb + 32 > a.n_cand ? 0xffffffffu << (a.n_cand - kb) : 0u);
+        w[q] |= kb >= a.n_cand ? 0xffffffffu : (kb + 32 > a.n_cand ? 0xffffffffu << (a.n_cand - kb) : 0u);
       }
     };
-    uint32_t next_raw[4] = {0u, 0u, 0u, 0u}, next_msk[4] = {0xffffffffu, 0xffffffffu, 0xffffffffu, 0xffffffffu};
-    {
-      // this group's first tile is local tile `grp`
+    // probabilities of 32 keys -> bf16 pairs -> columns [16 q, 16 q + 16) of the P buffer.  The
+    // kept-key word is the same for every row of the tile, so the test on it is uniform; most
+    // words have no kept key (the kept keys are a few per cent and come in runs).
+    auto soft32 = [&](uint32_t (&sv)[32], uint32_t paddr, uint32_t w) {
+#pragma unroll
+      for (int e = 0; e < 32; ++e)
+        sv[e] = __float_as_uint(ex2_approx(fmaf(__uint_as_float(sv[e]), a.scale2, nlse2)));
+      if (w != 0u) {
+#pragma unroll
+        for (int e = 0; e < 32; ++e)
+          if ((w >> e) & 1u) sv[e] = 0u;
+      }
+      uint32_t packed[16];
+#pragma unroll
+      for (int e = 0; e < 32; e += 2) {
+        l0 += __uint_as_float(sv[e]);
+        l1 += __uint_as_float(sv[e + 1]);
+        packed[e >> 1] = pack_bf16(__uint_as_float(sv[e]), __uint_as_float(sv[e + 1]));
+      }
+      tmem_st16(paddr, packed);
+    };
+
+    // The CTA's tile range is a sequence of segments (the tiles of one virtual unit); a group walks
+    // its own tiles only (local index of parity grp), and both groups open and close every segment,
+    // also one in which a group has no tile.  The bookkeeping between two tiles is kept short: it
+    // runs on one warp's dependent scalar instructions while the exponential unit idles.
+    uint32_t next_raw[4] = {0u, 0u, 0u, 0u};
+    if (grp < nt) {
       int t0 = tile_begin + grp, u0 = unit_begin;
       while (t0 >= a.n_tiles) { t0 -= a.n_tiles; ++u0; }
-      if (grp < nt) load_words(u0, t0, next_raw, next_msk);
+      load_words(u0, t0, next_raw);
     }
-    int vu = vu_begin, tile = tile_begin, unit = unit_begin;
-    for (int i = 0; i < nt; ++i, ++tile) {
-      if (tile == a.n_tiles) { tile = 0; ++unit; vu += a.n_cblocks; }
-      if (vu != cur_vu) {
-        if (cur_vu >= 0) {
-          ok = store_partial(cur_vu);
-          if (!ok) break;
+    int seg_first = 0, seg_tile0 = tile_begin, seg_unit = unit_begin, seg_vu = vu_begin;
+    while (seg_first < nt) {
+      const int seg_end = seg_first + min(nt - seg_first, a.n_tiles - seg_tile0);
+      l0 = l1 = 0.f;
+      load_q(seg_vu);
+      ++seg;
+#pragma unroll 1
+      for (int i = seg_first + ((seg_first ^ grp) & 1); i < seg_end; i += 2) {
+        const int tile = seg_tile0 + (i - seg_first);
+        uint32_t word[4] = {next_raw[0], next_raw[1], next_raw[2], next_raw[3]};
+        if (i + 2 < nt) {
+          int t2 = tile + 2, u2 = seg_unit;
+          while (t2 >= a.n_tiles) { t2 -= a.n_tiles; ++u2; }
+          load_words(u2, t2, next_raw);
         }
-        l0 = l1 = 0.f;
-        load_q(vu);
-        cur_vu = vu;
-        ++seg;
-      }
-      if ((i & 1) != grp) continue;
-      // kept-key bits of the tile's 128 keys (bit set = the key does not contribute).  The words of
-      // this group's NEXT tile are requested now and used a whole tile later: a load consumed in the
-      // tile that issued it stalled the group for an L2 round trip on every tile.
-      uint32_t word[4];
-#pragma unroll
-      for (int q = 0; q < 4; ++q) word[q] = next_raw[q] | next_msk[q];
-      {
-        int t2 = tile + 2, u2 = unit;
-        while (t2 >= a.n_tiles) { t2 -= a.n_tiles; ++u2; }
-        if (i + 2 < nt) load_words(u2, t2, next_raw, next_msk);
-      }
-      ok = mbar_wait(&ctl, s_full(grp), (i >> 1) & 1, 28u | ((unsigned)i << 8));
-      ok = __all_sync(0xffffffffu, ok);
-      if (!ok) break;
-      tc_fence_after_sync();
-      // probabilities of 32 keys -> bf16 pairs -> columns [16 q, 16 q + 16) of the P buffer
-      auto soft32 = [&](const uint32_t (&sv)[32], int q, uint32_t w) {
-        uint32_t packed[16];
-#pragma unroll
-        for (int e = 0; e < 32; e += 2) {
-          float p0 = ex2_approx(fmaf(__uint_as_float(sv[e]), a.scale2, nlse2));
-          float p1 = ex2_approx(fmaf(__uint_as_float(sv[e + 1]), a.scale2, nlse2));
-          if ((w >> e) & 1u) p0 = 0.f;
-          if ((w >> (e + 1)) & 1u) p1 = 0.f;
-          l0 += p0;
-          l1 += p1;
-          packed[e >> 1] = pack_bf16(p0, p1);
+        if (tile == a.n_tiles - 1) tail_mask(tile, word);
+        const int b = i % kBufs;
+        const uint32_t taddr = lane_addr + (uint32_t)(b * 128);   // S(i), then P(i) in its first 64 columns
+        ok = mbar_wait(&ctl, s_full(b), (i / kBufs) & 1, 28u | ((unsigned)i << 8));
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) break;
+        tc_fence_after_sync();
+        uint32_t ra[32], rb[32];
+        tmem_ld32_issue(taddr, ra);
+        tmem_ld_wait(ra);
+        tmem_ld32_issue(taddr + 32, rb);
+        // two rounds of (ra, rb); the loads of the second round are issued in the first.  P of the
+        // keys of columns [32 q, 32 q + 32) goes to columns [16 q, 16 q + 16): those have been read.
+#pragma unroll 1
+        for (int h = 0; h < 2; ++h) {
+          soft32(ra, taddr + (uint32_t)(32 * h), h ? word[2] : word[0]);
+          tmem_ld_wait(rb);
+          if (h == 0) tmem_ld32_issue(taddr + 64, ra);
+          soft32(rb, taddr + (uint32_t)(32 * h + 16), h ? word[3] : word[1]);
+          if (h == 0) {
+            tmem_ld_wait(ra);
+            tmem_ld32_issue(taddr + 96, rb);
+          }
         }
-        tmem_st16(paddr + (uint32_t)(16 * q), packed);
-      };
-      uint32_t ra[32], rb[32];
-      tmem_ld32_issue(taddr, ra);
-      tmem_ld_wait(ra);
-      tmem_ld32_issue(taddr + 32, rb);
-      // the P.V that read this P buffer two tiles ago must be done before it is overwritten
-      ok = mbar_wait(&ctl, p_empty(grp), ((i >> 1) & 1) ^ 1, 31u | ((unsigned)i << 8));
-      ok = __all_sync(0xffffffffu, ok);
+        tmem_st_wait();
+        tc_fence_before_sync();
+        mbar_arrive(p_full(b));
+      }
       if (!ok) break;
-      soft32(ra, 0, word[0]);
-      tmem_ld_wait(rb);
-      tmem_ld32_issue(taddr + 64, ra);
-      soft32(rb, 1, word[1]);
-      tmem_ld_wait(ra);
-      tmem_ld32_issue(taddr + 96, rb);
-      soft32(ra, 2, word[2]);
-      tmem_ld_wait(rb);
-      tc_fence_before_sync();
-      mbar_arrive(s_free(grp));   // S(i) is in registers: S(i+2) may overwrite the buffer
-      soft32(rb, 3, word[3]);
-      tmem_st_wait();
-      tc_fence_before_sync();
-      mbar_arrive(p_full(grp));
+      ok = store_partial(seg_vu);
+      if (!ok) break;
+      seg_first = seg_end;
+      seg_tile0 = 0;
+      ++seg_unit;
+      seg_vu += a.n_cblocks;
     }
-    if (ok && cur_vu >= 0) store_partial(cur_vu);
   }
 
   // ---------------------------------------------------------------- teardown (every path)
