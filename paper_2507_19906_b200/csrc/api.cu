@@ -94,7 +94,7 @@ CompressWs make_ws(const CompressGeom& g) {
     size_t parts;
     calib_tc_plan(g, &gpb, &n_cblocks, &tpc, &max_slots, &parts);
     w.calib_o = off; off = align_up(off + parts * 128 * kD * 4, 256);
-    w.calib_l = off; off = align_up(off + parts * 2 * 128 * 4, 256);
+    w.calib_l = off; off = align_up(off + parts * kCalibGroups * 128 * 4, 256);
   }
   w.total = off;
   return w;

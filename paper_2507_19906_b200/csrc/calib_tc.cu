@@ -37,12 +37,13 @@ namespace {
 
 using namespace tc;
 
-constexpr int kGroups = 2;
+constexpr int kGroups = kCalibGroups;  // softmax warpgroups: two pairs; a pair shares a tile, half of its keys each
 constexpr int kProducerWarp = kGroups * 4;       // TMA: Q_c blocks and K tiles
 constexpr int kMmaWarp = kGroups * 4 + 1;        // allocates TMEM, issues the S MMAs
 constexpr int kPvWarp = kGroups * 4 + 2;         // issues the P.V MMAs
 constexpr int kVProducerWarp = kGroups * 4 + 3;  // TMA: V tiles
 constexpr int kThreads = kGroups * 128 + 128;
+static_assert(kGroups == 4, "two pairs of softmax groups");
 constexpr int kTmemCols = 512;
 constexpr int kBufs = 3;                   // S/P buffers of 128 columns
 constexpr uint32_t kColO = kBufs * 128;
@@ -110,7 +111,7 @@ calib_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
       mbar_init(full_v(s), 1);
     }
     for (int b = 0; b < kBufs; ++b) {
-      mbar_init(s_full(b), 1); mbar_init(p_full(b), 128); mbar_init(buf_free(b), 1);
+      mbar_init(s_full(b), 1); mbar_init(p_full(b), 256); mbar_init(buf_free(b), 1);
     }
     fence_mbar_init();
   }
@@ -240,8 +241,9 @@ calib_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
         if (kFirst) umma_ts_imm<0>(tmem_o, pa, vd, idesc_o);
         else umma_ts_imm<1>(tmem_o, pa, vd, idesc_o);
 #pragma unroll
-        for (int kk = 1; kk < kTileKeys / 16; ++kk)
-          umma_ts_imm<1>(tmem_o, pa + (uint32_t)(kk * 8), desc_advance(vd, (uint32_t)kk * 16u * kLineBytes), idesc_o);
+        for (int kk = 1; kk < kTileKeys / 16; ++kk)   // the P of keys 64..127 sits at columns 64..95
+          umma_ts_imm<1>(tmem_o, pa + (uint32_t)((kk >> 2) * 64 + (kk & 3) * 8),
+                         desc_advance(vd, (uint32_t)kk * 16u * kLineBytes), idesc_o);
       };
       int seg = 0, tile = tile_begin, b = 0;
       uint32_t ph = 0;
@@ -268,13 +270,14 @@ calib_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
   } else {
     // ------------------------------------------------------------ softmax threads (one row each)
     const int grp = warp >> 2, r = tid & 127;
+    const int pair = grp >> 1, half = grp & 1;
     const uint32_t lane_bits = (uint32_t)((warp & 3) * 32) << 16;
     const uint32_t lane_addr = tmem_base + lane_bits;
     float l0 = 0.f, l1 = 0.f, nlse2 = -INFINITY;
     int seg = 0;
     bool ok = true, valid = false;
 
-    // Read out O and the row sums of the virtual unit that just ended (each group half of O's
+    // Read out O and the row sums of the virtual unit that just ended (each group a quarter of O's
     // columns).  o_full also tells that every MMA that read Q_c or P has completed.
     auto store_partial = [&](int vu) -> bool {
       bool w = mbar_wait(&ctl, o_full, (seg - 1) & 1, 30u);
@@ -284,8 +287,8 @@ calib_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
       const int slot = cta - ((vu / a.n_cblocks) * a.n_tiles) / a.tiles_per_cta;
       const size_t part = (size_t)vu * a.max_slots + slot;
       float* orow = a.o_part + (part * 128 + r) * kD;
-#pragma unroll 1
-      for (int c0 = grp * 64; c0 < grp * 64 + 64; c0 += 32) {
+      {
+        const int c0 = grp * 32;
         uint32_t ov[32];
         tmem_ld32(tmem_base + lane_bits + kColO + c0, ov);
         if (valid) {
@@ -315,25 +318,26 @@ calib_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
 
     const uint32_t* bm_all = a.bitmap;
     const int last_word = a.bitmap_words - 1;
-    // The four kept-key words of a tile (bit set = the key does not contribute) are loaded RAW one
-    // own tile ahead: nothing may touch a loaded value before the tile that uses it, or the thread
-    // waits for the load on the spot.  The index is clamped so that the load is always valid.
-    auto load_words = [&](int unit, int tile, uint32_t (&raw)[4]) {
+    // The two kept-key words of this group's 64 keys of a tile (bit set = the key does not
+    // contribute) are loaded RAW one own tile ahead: nothing may touch a loaded value before the tile
+    // that uses it, or the thread waits for the load on the spot.  The index is clamped so that the
+    // load is always valid.
+    auto load_words = [&](int unit, int tile, uint32_t (&raw)[2]) {
       const uint32_t* bm = bm_all + (size_t)unit * a.bitmap_words;
-      const int w0 = tile * (kTileKeys / 32);
+      const int w0 = tile * (kTileKeys / 32) + 2 * half;
 #pragma unroll
-      for (int q = 0; q < 4; ++q) raw[q] = __ldg(bm + min(w0 + q, last_word));
+      for (int q = 0; q < 2; ++q) raw[q] = __ldg(bm + min(w0 + q, last_word));
     };
     // keys at or beyond n_cand do not contribute either; only a unit's last tile has any
-    auto tail_mask = [&](int tile, uint32_t (&w)[4]) {
-      const int tbase = tile * kTileKeys;
+    auto tail_mask = [&](int tile, uint32_t (&w)[2]) {
+      const int tbase = tile * kTileKeys + 64 * half;
 #pragma unroll
-      for (int q = 0; q < 4; ++q) {
+      for (int q = 0; q < 2; ++q) {
         const int kb = tbase + 32 * q;
         w[q] |= kb >= a.n_cand ? 0xffffffffu : (kb + 32 > a.n_cand ? 0xffffffffu << (a.n_cand - kb) : 0u);
       }
     };
-    // probabilities of 32 keys -> bf16 pairs -> columns [16 q, 16 q + 16) of the P buffer.  The
+    // probabilities of 32 keys -> bf16 pairs -> 16 columns at paddr.  The
     // kept-key word is the same for every row of the tile, so the test on it is uniform; most
     // words have no kept key (the kept keys are a few per cent and come in runs).
     auto soft32 = [&](uint32_t (&sv)[32], uint32_t paddr, uint32_t w) {
@@ -355,13 +359,15 @@ calib_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
       tmem_st16(paddr, packed);
     };
 
-    // The CTA's tile range is a sequence of segments (the tiles of one virtual unit); a group walks
-    // its own tiles only (local index of parity grp), and both groups open and close every segment,
-    // also one in which a group has no tile.  The bookkeeping between two tiles is kept short: it
-    // runs on one warp's dependent scalar instructions while the exponential unit idles.
-    uint32_t next_raw[4] = {0u, 0u, 0u, 0u};
-    if (grp < nt) {
-      int t0 = tile_begin + grp, u0 = unit_begin;
+    // The CTA's tile range is a sequence of segments (the tiles of one virtual unit).  Pair p takes
+    // the tiles whose local index has parity p, each of its groups 64 of the tile's keys; every group
+    // opens and closes every segment, also one in which its pair has no tile.  Two pairs, half a tile
+    // apart, keep up to four warps per scheduler on the exponential unit: one warp per scheduler alone
+    // reaches less than half of that unit's rate (measured: a group alone took 2400 cycles for the
+    // 128 x 128 exponentials of a tile, 18 cycles per warp instruction against the unit's 8).
+    uint32_t next_raw[2] = {0u, 0u};
+    if (pair < nt) {
+      int t0 = tile_begin + pair, u0 = unit_begin;
       while (t0 >= a.n_tiles) { t0 -= a.n_tiles; ++u0; }
       load_words(u0, t0, next_raw);
     }
@@ -372,9 +378,9 @@ calib_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
       load_q(seg_vu);
       ++seg;
 #pragma unroll 1
-      for (int i = seg_first + ((seg_first ^ grp) & 1); i < seg_end; i += 2) {
+      for (int i = seg_first + ((seg_first ^ pair) & 1); i < seg_end; i += 2) {
         const int tile = seg_tile0 + (i - seg_first);
-        uint32_t word[4] = {next_raw[0], next_raw[1], next_raw[2], next_raw[3]};
+        uint32_t word[2] = {next_raw[0], next_raw[1]};
         if (i + 2 < nt) {
           int t2 = tile + 2, u2 = seg_unit;
           while (t2 >= a.n_tiles) { t2 -= a.n_tiles; ++u2; }
@@ -382,7 +388,9 @@ calib_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
         }
         if (tile == a.n_tiles - 1) tail_mask(tile, word);
         const int b = i % kBufs;
-        const uint32_t taddr = lane_addr + (uint32_t)(b * 128);   // S(i), then P(i) in its first 64 columns
+        // S(i) of this group's keys; their P goes to the first 32 of the same 64 columns, which this
+        // group alone reads, each 16 columns only after the S they held is in registers
+        const uint32_t taddr = lane_addr + (uint32_t)(b * 128 + half * 64);
         ok = mbar_wait(&ctl, s_full(b), (i / kBufs) & 1, 28u | ((unsigned)i << 8));
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) break;
@@ -390,20 +398,10 @@ calib_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
         uint32_t ra[32], rb[32];
         tmem_ld32_issue(taddr, ra);
         tmem_ld_wait(ra);
-        tmem_ld32_issue(taddr + 32, rb);
-        // two rounds of (ra, rb); the loads of the second round are issued in the first.  P of the
-        // keys of columns [32 q, 32 q + 32) goes to columns [16 q, 16 q + 16): those have been read.
-#pragma unroll 1
-        for (int h = 0; h < 2; ++h) {
-          soft32(ra, taddr + (uint32_t)(32 * h), h ? word[2] : word[0]);
-          tmem_ld_wait(rb);
-          if (h == 0) tmem_ld32_issue(taddr + 64, ra);
-          soft32(rb, taddr + (uint32_t)(32 * h + 16), h ? word[3] : word[1]);
-          if (h == 0) {
-            tmem_ld_wait(ra);
-            tmem_ld32_issue(taddr + 96, rb);
-          }
-        }
+        tmem_ld32_issue(taddr + 32, rb);   // arrives while the first 32 keys are worked on
+        soft32(ra, taddr, word[0]);
+        tmem_ld_wait(rb);
+        soft32(rb, taddr + 16, word[1]);
         tmem_st_wait();
         tc_fence_before_sync();
         mbar_arrive(p_full(b));

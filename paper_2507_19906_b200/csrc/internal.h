@@ -53,6 +53,7 @@ struct alignas(64) DecodeLayerMaps {
   CUtensorMap k64, v64, k16, v16;
 };
 
+constexpr int kCalibGroups = 4;  // softmax warpgroups of the calibration kernel: row-sum partials per slot
 constexpr int kDecodeMaxLayers = 32;
 constexpr int kDecodeMaxSplit = 64;
 constexpr int kDecodeTargetCtas = 148;  // one CTA of a launch on each of the 148 SMs
