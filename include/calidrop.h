@@ -12,10 +12,14 @@
  *                      calibration queries, threshold gate, and the merge of Eq. 1-2.
  *
  * Around them: calidrop_calibrate (the second half of calidrop_compress for a kept list chosen by
- * another eviction rule), calidrop_gather_evicted and calidrop_recalibrate (Algorithm 1 line 4 and
- * Algorithm 2 lines 3-8: the evicted rows compacted for offloading, and the recompute of a
- * calibration entry from them), calidrop_decode_batched (several layers in one launch) and
- * calidrop_decode_static (no caller workspace).
+ * another eviction rule), calidrop_select_streaming and calidrop_select_from_scores (the kept lists
+ * of two such rules: sinks plus recent rows, and top-k of caller-supplied accumulated scores),
+ * calidrop_gather_evicted, calidrop_offload_evicted, calidrop_reload_evicted and
+ * calidrop_recalibrate (Algorithm 1 line 4 and Algorithm 2 lines 3-8: the evicted rows compacted,
+ * moved to host memory and back beside the decode, and the recompute of a calibration entry from
+ * them), calidrop_decode_batched (several layers in one launch) and calidrop_decode_static (no
+ * caller workspace).  The field calib_size of the parameters is the calibration size of
+ * Section 4.4.
  *
  * Conventions
  *   - Unless a comment says HOST, every tensor pointer is a DEVICE pointer to a contiguous,

@@ -6,9 +6,9 @@
 // virtual unit is a (batch, kv-head) unit, or for the statistics one half of its window rows when
 // there are more than 256; its query rows stay resident in shared memory and are reloaded when
 // the CTA's range crosses into the next virtual unit.
-// Warp roles: two consumer warpgroups read the accumulators out of TMEM (one TMEM lane per
-// thread, group g owns accumulator buffer g), one warp is the TMA producer, one warp allocates TMEM
-// and issues the MMAs.  Every MMA has N = 256 where the shape allows it: with both operands in
+// Warp roles: four consumer warpgroups in two pairs read the accumulators out of TMEM (one TMEM
+// lane per thread; pair p drains accumulator buffer p, each of its groups half of the columns), one
+// warp is the TMA producer, one warp allocates TMEM and issues the MMAs.  Every MMA has N = 256 where the shape allows it: with both operands in
 // shared memory, narrower tiles are limited by operand fetch, not by the tensor pipe.
 //
 //   statistics (kVotes = false):  S = Q K^T, 128 query rows on the TMEM lanes, 256 keys per tile.
