@@ -266,14 +266,19 @@ int calidrop_compress(const calidrop_params* p, const void* Q_obs, const void* K
   e = select_cluster_supported(g) ? launch_pool_select_cluster(g, ws, wsp, kept_idx, st)
                                   : launch_pool_select(g, ws, wsp, kept_idx, st);
   if (e != cudaSuccess) return cuda_fail(e);
-  e = launch_gather(g, K, V, kept_idx, K_kept, V_kept, st);
-  if (e != cudaSuccess) return cuda_fail(e);
+  // the compaction of the retained rows rides on the calibration's second kernel when that runs
+  const bool calib_tc = tc_path && calib_tc_supported(g) && !(g.sized && g.n_calib == 0);
+  if (!calib_tc) {
+    e = launch_gather(g, K, V, kept_idx, K_kept, V_kept, st);
+    if (e != cudaSuccess) return cuda_fail(e);
+  }
+  const GatherArgs ga{(const uint4*)K, (const uint4*)V, kept_idx, (uint4*)K_kept, (uint4*)V_kept,
+                      g.L, g.n_kept, g.cap, g.units};
   if (g.sized && g.n_calib == 0)
     e = launch_calib_none(g, Q_obs, O_c, LSE_c, C_q, st);
   else
-    e = (tc_path && calib_tc_supported(g))
-            ? launch_calib_tc(g, ws, Q_obs, K, V, row_lse, wsp, O_c, LSE_c, C_q, st)
-            : launch_calib_direct(g, ws, Q_obs, K, V, wsp, O_c, LSE_c, C_q, st);
+    e = calib_tc ? launch_calib_tc(g, ws, Q_obs, K, V, row_lse, wsp, O_c, LSE_c, C_q, ga, st)
+                 : launch_calib_direct(g, ws, Q_obs, K, V, wsp, O_c, LSE_c, C_q, st);
   if (e != cudaSuccess) return cuda_fail(e);
   return CALIDROP_OK;
 }
@@ -309,11 +314,15 @@ int calidrop_calibrate(const calidrop_params* p, const void* Q_obs, const void* 
   }
   e = launch_bitmap_from_indices(g, ws, wsp, kept_idx, st);
   if (e != cudaSuccess) return cuda_fail(e);
-  e = launch_gather(g, K, V, kept_idx, K_kept, V_kept, st);
-  if (e != cudaSuccess) return cuda_fail(e);
-  e = (tc_path && calib_tc_supported(g))
-          ? launch_calib_tc(g, ws, Q_obs, K, V, row_lse, wsp, O_c, LSE_c, C_q, st)
-          : launch_calib_direct(g, ws, Q_obs, K, V, wsp, O_c, LSE_c, C_q, st);
+  const bool calib_tc = tc_path && calib_tc_supported(g);
+  if (!calib_tc) {
+    e = launch_gather(g, K, V, kept_idx, K_kept, V_kept, st);
+    if (e != cudaSuccess) return cuda_fail(e);
+  }
+  const GatherArgs ga{(const uint4*)K, (const uint4*)V, kept_idx, (uint4*)K_kept, (uint4*)V_kept,
+                      g.L, g.n_kept, g.cap, g.units};
+  e = calib_tc ? launch_calib_tc(g, ws, Q_obs, K, V, row_lse, wsp, O_c, LSE_c, C_q, ga, st)
+               : launch_calib_direct(g, ws, Q_obs, K, V, wsp, O_c, LSE_c, C_q, st);
   if (e != cudaSuccess) return cuda_fail(e);
   return CALIDROP_OK;
 }

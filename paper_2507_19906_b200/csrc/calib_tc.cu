@@ -427,15 +427,20 @@ calib_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
 
 // One warp per (batch, query head, calibration row): sum the partials of the CTAs that shared the
 // row's virtual unit, in order, then O_c = O / l, LSE_c = lse + log l (zeros and -inf when nothing
-// was evicted), C_q = the query.
-__global__ void __launch_bounds__(128)
+// was evicted), C_q = the query.  The blocks beyond the reduction's compact the retained rows.
+__global__ void __launch_bounds__(256)
 calib_reduce_kernel(const __nv_bfloat16* __restrict__ Q_obs, const float* __restrict__ row_lse,
                     const float* __restrict__ o_part, const float* __restrict__ l_part,
                     float* __restrict__ O_c, float* __restrict__ LSE_c, __nv_bfloat16* __restrict__ C_q, int B,
                     int Hq, int G, int W, int n_cal, int gpb, int n_cblocks, int n_tiles, int tiles_per_cta,
-                    int max_slots) {
+                    int max_slots, int reduce_blocks, const GatherArgs gather) {
+  if ((int)blockIdx.x >= reduce_blocks) {
+    const int gb = (int)blockIdx.x - reduce_blocks, per_unit = (gather.n_rows + 15) / 16;
+    gather_rows16(gather, gb % per_unit, gb / per_unit, threadIdx.x);
+    return;
+  }
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const int row = blockIdx.x * 4 + warp;  // (b, hq, c)
+  const int row = blockIdx.x * 8 + warp;  // (b, hq, c)
   if (row >= B * Hq * n_cal) return;
   const int c = row % n_cal, bhq = row / n_cal;
   const int b = bhq / Hq, hq = bhq % Hq;
@@ -490,7 +495,7 @@ void calib_tc_plan(const CompressGeom& g, int* gpb, int* n_cblocks, int* tiles_p
 
 cudaError_t launch_calib_tc(const CompressGeom& g, const CompressWs& ws, const void* Q_obs, const void* K,
                             const void* V, const float* row_lse, char* wsp, float* O_c, float* LSE_c, void* C_q,
-                            cudaStream_t st) {
+                            const GatherArgs& gather, cudaStream_t st) {
   CalibArgs a{};
   a.Hq = g.Hq; a.G = g.G; a.W = g.W; a.L = g.L; a.n_cand = g.n_cand; a.n_cal = g.n_cal;
   size_t parts;
@@ -527,9 +532,11 @@ cudaError_t launch_calib_tc(const CompressGeom& g, const CompressWs& ws, const v
   const int grid = (a.total_tiles + a.tiles_per_cta - 1) / a.tiles_per_cta * a.n_cblocks;
   calib_tc_kernel<<<grid, kThreads, kSmemBytes, st>>>(qm, km, vm, a);
   const int total = g.B * g.Hq * g.n_cal;
-  calib_reduce_kernel<<<(total + 3) / 4, 128, 0, st>>>((const __nv_bfloat16*)Q_obs, row_lse, a.o_part, a.l_part, O_c,
-                                                      LSE_c, (__nv_bfloat16*)C_q, g.B, g.Hq, g.G, g.W, g.n_cal,
-                                                      a.gpb, a.n_cblocks, a.n_tiles, a.tiles_per_cta, a.max_slots);
+  const int reduce_blocks = (total + 7) / 8;
+  const int gather_blocks = gather.idx ? gather.units * ((gather.n_rows + 15) / 16) : 0;
+  calib_reduce_kernel<<<reduce_blocks + gather_blocks, 256, 0, st>>>(
+      (const __nv_bfloat16*)Q_obs, row_lse, a.o_part, a.l_part, O_c, LSE_c, (__nv_bfloat16*)C_q, g.B, g.Hq, g.G, g.W,
+      g.n_cal, a.gpb, a.n_cblocks, a.n_tiles, a.tiles_per_cta, a.max_slots, reduce_blocks, gather);
   count_launch(2);
   return cudaGetLastError();
 }

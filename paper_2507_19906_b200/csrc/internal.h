@@ -101,9 +101,35 @@ cudaError_t launch_votes_tc(const CompressGeom& g, const CompressWs& ws, const v
 bool calib_tc_supported(const CompressGeom& g);
 void calib_tc_plan(const CompressGeom& g, int* gpb, int* n_cblocks, int* tiles_per_cta, int* max_slots,
                    size_t* parts);
+// The compaction of the retained rows (A5), as arguments: K_out[u, i, :] = K[u, idx[u, i], :], same
+// for V.  The calibration's second kernel carries it along (blocks of its own beside the reduction's)
+// when `idx` is not null: it only depends on the kept list, and as a kernel of its own between the
+// selection and the calibration its 10 us at copy bandwidth were exposed.
+struct GatherArgs {
+  const uint4* K;
+  const uint4* V;
+  const int32_t* idx;   // [units, n_rows]
+  uint4* K_out;         // [units, out_rows, 16]
+  uint4* V_out;
+  int L, n_rows, out_rows, units;
+};
 cudaError_t launch_calib_tc(const CompressGeom& g, const CompressWs& ws, const void* Q_obs, const void* K,
                             const void* V, const float* row_lse, char* wsp, float* O_c, float* LSE_c, void* C_q,
-                            cudaStream_t st);
+                            const GatherArgs& gather, cudaStream_t st);
+#ifdef __CUDACC__
+// Rows [16 bx, 16 bx + 16) of unit `unit`: 16 lanes x 16 bytes per row, 256 threads.
+__device__ __forceinline__ void gather_rows16(const GatherArgs& a, int bx, int unit, int tid) {
+  const int i = bx * 16 + (tid >> 4);
+  const int chunk = tid & 15;
+  if (i >= a.n_rows) return;
+  const int t = a.idx[(size_t)unit * a.n_rows + i];
+  if (t < 0 || t >= a.L) return;   // a caller's list may hold anything: rows outside the prompt are skipped
+  const size_t src = ((size_t)unit * a.L + t) * 16 + chunk;
+  const size_t dst = ((size_t)unit * a.out_rows + i) * 16 + chunk;
+  a.K_out[dst] = __ldg(a.K + src);
+  a.V_out[dst] = __ldg(a.V + src);
+}
+#endif
 // select.cu
 cudaError_t launch_pool_select(const CompressGeom& g, const CompressWs& ws, char* wsp,
                                int32_t* kept_idx, cudaStream_t st);

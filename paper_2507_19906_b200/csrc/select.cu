@@ -175,20 +175,8 @@ __global__ void bitmap_from_indices_kernel(const int32_t* __restrict__ kept_idx,
 }
 
 // K_kept[u, i, :] = K[u, kept_idx[u, i], :], same for V; 16 lanes x 16 bytes per row.
-__global__ void __launch_bounds__(256)
-gather_kernel(const uint4* __restrict__ K, const uint4* __restrict__ V,
-              const int32_t* __restrict__ kept_idx, uint4* __restrict__ K_kept,
-              uint4* __restrict__ V_kept, int L, int n_kept, int cap) {
-  const int unit = blockIdx.y;
-  const int i = blockIdx.x * 16 + (threadIdx.x >> 4);
-  const int chunk = threadIdx.x & 15;
-  if (i >= n_kept) return;
-  const int t = kept_idx[(size_t)unit * n_kept + i];
-  if (t < 0 || t >= L) return;   // a caller's list may hold anything: rows outside the prompt are skipped
-  const size_t src = ((size_t)unit * L + t) * 16 + chunk;
-  const size_t dst = ((size_t)unit * cap + i) * 16 + chunk;
-  K_kept[dst] = __ldg(K + src);
-  V_kept[dst] = __ldg(V + src);
+__global__ void __launch_bounds__(256) gather_kernel(const GatherArgs a) {
+  gather_rows16(a, blockIdx.x, blockIdx.y, threadIdx.x);
 }
 
 }  // namespace
@@ -310,8 +298,8 @@ cudaError_t launch_bitmap_from_indices(const CompressGeom& g, const CompressWs& 
 cudaError_t launch_gather_rows(const CompressGeom& g, const void* K, const void* V, const int32_t* idx, int n_rows,
                                int out_rows, void* K_out, void* V_out, cudaStream_t st) {
   dim3 grid((n_rows + 15) / 16, g.units);
-  gather_kernel<<<grid, 256, 0, st>>>((const uint4*)K, (const uint4*)V, idx, (uint4*)K_out, (uint4*)V_out, g.L,
-                                      n_rows, out_rows);
+  const GatherArgs a{(const uint4*)K, (const uint4*)V, idx, (uint4*)K_out, (uint4*)V_out, g.L, n_rows, out_rows, g.units};
+  gather_kernel<<<grid, 256, 0, st>>>(a);
   count_launch(1);
   return cudaGetLastError();
 }
