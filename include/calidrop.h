@@ -13,7 +13,8 @@
  *
  * Around them: calidrop_calibrate (the second half of calidrop_compress for a kept list chosen by
  * another eviction rule), calidrop_select_streaming and calidrop_select_from_scores (the kept lists
- * of two such rules: sinks plus recent rows, and top-k of caller-supplied accumulated scores),
+ * of two such rules: sinks plus recent rows, and top-k of accumulated scores, which
+ * calidrop_accumulated_scores computes when the prefill does not supply them),
  * calidrop_gather_evicted, calidrop_offload_evicted, calidrop_reload_evicted and
  * calidrop_recalibrate (Algorithm 1 line 4 and Algorithm 2 lines 3-8: the evicted rows compacted,
  * moved to host memory and back beside the decode, and the recompute of a calibration entry from
@@ -166,8 +167,8 @@ int calidrop_calibrate(const calidrop_params* p,
  * calidrop_select_from_scores: kept = the budget - tail rows of [0, L - tail) with the largest
  *   pooled score (zero-padded average pool of kernel `pool` of `p`, 1 for none; ties to the lowest
  *   index) and the last `tail` rows.  With the accumulated attention score of the prefill (its
- *   column sums over all queries, a by-product of the prefill attention that this library does not
- *   compute) and tail = budget / 2 this is H2O's rule; with the window votes and tail = window it is
+ *   column sums over all queries, a by-product of the prefill attention, or the output of
+ *   calidrop_accumulated_scores below) and tail = budget / 2 this is H2O's rule; with the window votes and tail = window it is
  *   the selection step of calidrop_compress.
  *     scores in [B, Hkv, L] f32, finite and non-negative (they are ordered by their bit patterns);
  *            entries at and beyond L - tail are not read
@@ -175,9 +176,24 @@ int calidrop_calibrate(const calidrop_params* p,
  *     workspace: a calidrop_compress workspace for `p` (the pooled scores and a bitmap go there)
  *   UNSUPPORTED beyond 262144 prompt rows.
  *   kept_idx out [B, Hkv, n_kept] i32, ascending.
+ * calidrop_accumulated_scores: H2O's importance measure (Section 4.1.2: the accumulated attention
+ *   score) for callers whose prefill does not hand it over:
+ *       scores[b, h, t] = sum over the G query heads of kv head h and over the prompt queries i >= t
+ *                         of softmax_i(q_i . k / sqrt(D))[t]      (causal attention, column sums)
+ *   in two tensor-core passes over Q and K (row statistics, then column sums; fp32 throughout, no
+ *   atomics: bit-reproducible).  It costs as much as the prefill attention itself, L^2 D flop per
+ *   head, and is therefore no part of calidrop_compress.
+ *     Q_full in  [B, Hq, L, D] bf16, every prompt query (its last `window` rows are Q_obs)
+ *     K      in  [B, Hkv, L, D] bf16
+ *     scores out [B, Hkv, L] f32
+ *     workspace: calidrop_accumulated_scores_workspace_bytes(p) bytes (the row statistics,
+ *            4 B Hq L), 256-byte aligned; WORKSPACE_TOO_SMALL otherwise
  */
 int calidrop_select_streaming(const calidrop_params* p, int32_t n_sink, int32_t* kept_idx, void* stream);
 int calidrop_select_from_scores(const calidrop_params* p, const float* scores, int32_t tail, int32_t* kept_idx,
+                                void* workspace, size_t workspace_bytes, void* stream);
+size_t calidrop_accumulated_scores_workspace_bytes(const calidrop_params* p);
+int calidrop_accumulated_scores(const calidrop_params* p, const void* Q_full, const void* K, float* scores,
                                 void* workspace, size_t workspace_bytes, void* stream);
 
 /*

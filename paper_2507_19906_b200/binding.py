@@ -26,6 +26,7 @@ EXPORTS = [
     "calidrop_compress_workspace_bytes", "calidrop_compress", "calidrop_calibrate", "calidrop_gather_evicted",
     "calidrop_recalibrate", "calidrop_offload_evicted", "calidrop_reload_evicted",
     "calidrop_select_streaming", "calidrop_select_from_scores",
+    "calidrop_accumulated_scores_workspace_bytes", "calidrop_accumulated_scores",
     "calidrop_compress_workspace_layout",
     "calidrop_decode_workspace_bytes", "calidrop_decode_workspace_init",
     "calidrop_decode_workspace_status_offset", "calidrop_decode",
@@ -85,6 +86,10 @@ def load():
         f.argtypes = [C.POINTER(Params), C.c_int32, vp, vp, vp, vp, vp, vp, vp]
     lib.calidrop_select_streaming.restype = C.c_int
     lib.calidrop_select_streaming.argtypes = [C.POINTER(Params), C.c_int32, vp, vp]
+    lib.calidrop_accumulated_scores_workspace_bytes.restype = C.c_size_t
+    lib.calidrop_accumulated_scores_workspace_bytes.argtypes = [C.POINTER(Params)]
+    lib.calidrop_accumulated_scores.restype = C.c_int
+    lib.calidrop_accumulated_scores.argtypes = [C.POINTER(Params), vp, vp, vp, vp, C.c_size_t, vp]
     lib.calidrop_select_from_scores.restype = C.c_int
     lib.calidrop_select_from_scores.argtypes = [C.POINTER(Params), vp, C.c_int32, vp, vp, C.c_size_t, vp]
     lib.calidrop_calibrate.restype = C.c_int
@@ -209,6 +214,18 @@ def calidrop_select_streaming(p, n_sink, kept_idx, check=True) -> int:
     rc = load().calidrop_select_streaming(C.byref(p), int(n_sink), _ptr(kept_idx), _stream())
     if check:
         _check(rc, "calidrop_select_streaming")
+    return rc
+
+
+def calidrop_accumulated_scores_workspace_bytes(p: Params) -> int:
+    return int(load().calidrop_accumulated_scores_workspace_bytes(C.byref(p)))
+
+
+def calidrop_accumulated_scores(p, Q_full, K, scores, workspace, check=True) -> int:
+    rc = load().calidrop_accumulated_scores(C.byref(p), _ptr(Q_full), _ptr(K), _ptr(scores), _ptr(workspace),
+                                            workspace.numel() * workspace.element_size(), _stream())
+    if check:
+        _check(rc, "calidrop_accumulated_scores")
     return rc
 
 

@@ -327,6 +327,27 @@ int calidrop_calibrate(const calidrop_params* p, const void* Q_obs, const void* 
   return CALIDROP_OK;
 }
 
+size_t calidrop_accumulated_scores_workspace_bytes(const calidrop_params* p) {
+  if (check_compress(p) != CALIDROP_OK) return 0;
+  return align_up((size_t)p->B * p->Hq * p->L * 4, 256);
+}
+
+int calidrop_accumulated_scores(const calidrop_params* p, const void* Q_full, const void* K, float* scores,
+                                void* workspace, size_t workspace_bytes, void* stream) {
+  int rc = check_compress(p);
+  if (rc != CALIDROP_OK) return rc;
+  const void* ptrs[] = {Q_full, K, scores, workspace};
+  for (const void* q : ptrs)
+    if (!q || !aligned16(q)) return CALIDROP_INVALID_ARG;
+  if (reinterpret_cast<uintptr_t>(workspace) & 255u) return CALIDROP_INVALID_ARG;
+  if (workspace_bytes < calidrop_accumulated_scores_workspace_bytes(p)) return CALIDROP_WORKSPACE_TOO_SMALL;
+  if (!device_supported()) return CALIDROP_UNSUPPORTED;
+  const CompressGeom g = make_geom(p);
+  cudaError_t e = launch_accum_scores(p->B, p->Hq, p->Hkv, p->L, g.scale2, Q_full, K, (float*)workspace, scores,
+                                      (cudaStream_t)stream);
+  return e == cudaSuccess ? CALIDROP_OK : cuda_fail(e);
+}
+
 int calidrop_select_streaming(const calidrop_params* p, int32_t n_sink, int32_t* kept_idx, void* stream) {
   int rc = check_compress(p);
   if (rc != CALIDROP_OK) return rc;

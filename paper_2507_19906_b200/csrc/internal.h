@@ -146,6 +146,9 @@ cudaError_t launch_gather_rows(const CompressGeom& g, const void* K, const void*
                                int out_rows, void* K_out, void* V_out, cudaStream_t st);
 cudaError_t launch_gather(const CompressGeom& g, const void* K, const void* V, const int32_t* kept_idx,
                           void* K_kept, void* V_kept, cudaStream_t st);
+// accum_scores.cu
+cudaError_t launch_accum_scores(int B, int Hq, int Hkv, int L, float scale2, const void* Q_full, const void* K,
+                                float* lse2, float* scores, cudaStream_t st);
 // decode.cu
 // Fills the TMA views of one layer; false when the driver refuses the encoding.
 bool make_decode_maps(const DecodeCommon& c, const DecodeLayerPtrs& L, DecodeLayerMaps* out);

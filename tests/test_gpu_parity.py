@@ -766,6 +766,53 @@ def test_streaming_and_h2o_kept_lists_from_the_library_feed_the_calibration(cuda
                                           check=False) == cd.INVALID_ARG
 
 
+@pytest.mark.parametrize("B,Hq,Hkv,L", [(1, 4, 2, 333), (2, 6, 2, 700), (1, 8, 1, 1100)])
+def test_h2o_accumulated_scores_from_the_library(cuda_lib, B, Hq, Hkv, L):
+    """H2O's importance measure (Section 4.1.2): the column sums of the causal attention of every prompt
+    query, per kv head, computed by the library from Q and K, against the oracle's definition; the kept
+    list that the library then selects from ITS scores equals the oracle's list from the oracle's scores
+    up to swaps of rows whose oracle scores are closer than the fp32 arithmetic resolves."""
+    cd = cuda_lib
+    G, W, budget = Hq // Hkv, 16, 128
+    rng = np.random.Generator(np.random.Philox(key=[41, L]))
+    Qf = wl.f32_to_bf16_bits(rng.standard_normal((B, Hq, L, 128)).astype(np.float32))
+    Kb = wl.f32_to_bf16_bits(rng.standard_normal((B, Hkv, L, 128)).astype(np.float32))
+    Kb[:, :, ::37] = wl.f32_to_bf16_bits(2.5 * wl.bf16_bits_to_f32(Kb[:, :, ::37]))   # some heavy hitters
+    p = cd.make_params(B=B, Hq=Hq, Hkv=Hkv, L=L, window=W, pool=1, budget=budget, n_cal=1, cap=budget + 2)
+    st = cd.alloc_layer_state(p)
+    ws = torch.empty((cd.calidrop_accumulated_scores_workspace_bytes(p),), dtype=torch.uint8, device="cuda")
+    scores = torch.full((B, Hkv, L), -1.0, dtype=torch.float32, device="cuda")
+    runs = []
+    for _ in range(2):                                  # twice: the result is reproducible bit for bit
+        cd.calidrop_accumulated_scores(p, to_dev(Qf), to_dev(Kb), scores, ws)
+        torch.cuda.synchronize()
+        runs.append(scores.cpu().numpy().copy())
+    np.testing.assert_array_equal(runs[0], runs[1])
+    got = runs[0]
+    ref = np.stack([np.stack([oracle.accumulated_attention(Qf[b, h * G:(h + 1) * G], Kb[b, h]) for h in range(Hkv)])
+                    for b in range(B)])
+    # every query's attention sums to one: the scores of a kv head sum to G * L
+    np.testing.assert_allclose(ref.sum(-1), G * L, rtol=1e-9)
+    np.testing.assert_allclose(got, ref, rtol=2e-5, atol=1e-6)
+    np.testing.assert_allclose(got.sum(-1, dtype=np.float64), G * L, rtol=1e-5)
+    cd.calidrop_select_from_scores(p, scores, budget // 2, st.kept_idx, st.ws_compress)
+    torch.cuda.synchronize()
+    kept = st.kept_idx.cpu().numpy()
+    for b in range(B):
+        for h in range(Hkv):
+            want = oracle.select_from_scores(ref[b, h].astype(np.float32), tail=budget // 2, budget=budget)
+            a, w = set(kept[b, h].tolist()), set(want.tolist())
+            assert len(a) == budget and np.all(np.diff(kept[b, h]) > 0)
+            if a != w:                                  # only near-ties of the oracle's scores may swap
+                thr = min(ref[b, h][t] for t in w if t < L - budget // 2)
+                for t in a ^ w:
+                    assert abs(ref[b, h][t] - thr) <= 2e-5 * thr, (b, h, t, ref[b, h][t], thr)
+    # argument checks
+    small = torch.empty((16,), dtype=torch.uint8, device="cuda")
+    assert cd.calidrop_accumulated_scores(p, to_dev(Qf), to_dev(Kb), scores, small, check=False) == cd.WORKSPACE_TOO_SMALL
+    assert cd.calidrop_accumulated_scores(p, None, to_dev(Kb), scores, ws, check=False) == cd.INVALID_ARG
+
+
 # ---------------------------------------------------------------- seeded random shapes
 def _random_shapes(n, seed):
     rng = np.random.Generator(np.random.Philox(key=[seed, 1]))
