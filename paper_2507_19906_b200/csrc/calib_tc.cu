@@ -127,6 +127,7 @@ calib_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
   __syncthreads();
   tc_fence_after_sync();
   const uint32_t tmem_base = tmem_slot;
+  pdl_wait();   // everything above ran beside the previous kernel's end; global memory from here on
 
   // first tile of a run of tiles of one virtual unit inside this CTA's range
   // (the position inside the tile space is tracked incrementally: no division per tile)
@@ -422,6 +423,7 @@ calib_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
   }
   tc_fence_before_sync();
   __syncthreads();
+  pdl_trigger();   // every warp is done: the next kernel's CTAs may set themselves up while this one winds down
   if (warp == kMmaWarp) tmem_dealloc(tmem_base, kTmemCols);
 }
 
@@ -434,6 +436,8 @@ calib_reduce_kernel(const __nv_bfloat16* __restrict__ Q_obs, const float* __rest
                     float* __restrict__ O_c, float* __restrict__ LSE_c, __nv_bfloat16* __restrict__ C_q, int B,
                     int Hq, int G, int W, int n_cal, int gpb, int n_cblocks, int n_tiles, int tiles_per_cta,
                     int max_slots, int reduce_blocks, const GatherArgs gather) {
+  pdl_trigger();
+  pdl_wait();
   if ((int)blockIdx.x >= reduce_blocks) {
     const int gb = (int)blockIdx.x - reduce_blocks, per_unit = (gather.n_rows + 15) / 16;
     gather_rows16(gather, gb % per_unit, gb / per_unit, threadIdx.x);
@@ -530,13 +534,16 @@ cudaError_t launch_calib_tc(const CompressGeom& g, const CompressWs& ws, const v
     if (dev >= 0 && dev < 64) attr_set[dev] = true;
   }
   const int grid = (a.total_tiles + a.tiles_per_cta - 1) / a.tiles_per_cta * a.n_cblocks;
-  calib_tc_kernel<<<grid, kThreads, kSmemBytes, st>>>(qm, km, vm, a);
+  e = launch_pdl(calib_tc_kernel, dim3(grid), dim3(kThreads), (size_t)kSmemBytes, st, qm, km, vm, a);
+  if (e != cudaSuccess) return e;
   const int total = g.B * g.Hq * g.n_cal;
   const int reduce_blocks = (total + 7) / 8;
   const int gather_blocks = gather.idx ? gather.units * ((gather.n_rows + 15) / 16) : 0;
-  calib_reduce_kernel<<<reduce_blocks + gather_blocks, 256, 0, st>>>(
-      (const __nv_bfloat16*)Q_obs, row_lse, a.o_part, a.l_part, O_c, LSE_c, (__nv_bfloat16*)C_q, g.B, g.Hq, g.G, g.W,
-      g.n_cal, a.gpb, a.n_cblocks, a.n_tiles, a.tiles_per_cta, a.max_slots, reduce_blocks, gather);
+  e = launch_pdl(calib_reduce_kernel, dim3(reduce_blocks + gather_blocks), dim3(256), 0, st,
+                 (const __nv_bfloat16*)Q_obs, row_lse, (const float*)a.o_part, (const float*)a.l_part, O_c, LSE_c,
+                 (__nv_bfloat16*)C_q, g.B, g.Hq, g.G, g.W, g.n_cal, a.gpb, a.n_cblocks, a.n_tiles, a.tiles_per_cta,
+                 a.max_slots, reduce_blocks, gather);
+  if (e != cudaSuccess) return e;
   count_launch(2);
   return cudaGetLastError();
 }

@@ -39,6 +39,15 @@ __device__ __forceinline__ float warp_sum(float v) {
   return v;
 }
 
+// Programmatic dependent launch.  The kernels of the compress step are launched with the
+// programmatic-serialisation attribute: a kernel may start (set up its barriers, tensor memory and
+// shared memory) while its predecessor in the stream still runs, and waits here before it touches
+// global memory.  pdl_trigger at a kernel's top lets its successor do the same; every thread of
+// every kernel launched this way calls pdl_wait, so a kernel that has completed implies that all
+// its predecessors have.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
   return static_cast<uint32_t>(__cvta_generic_to_shared(p));
 }

@@ -143,6 +143,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
   __syncthreads();
   tc_fence_after_sync();
   const uint32_t tmem_base = tmem_slot;
+  pdl_wait();   // everything above ran beside the previous kernel's end; global memory from here on
 
   if (warp == kProducerWarp) {
     // ------------------------------------------------------------ TMA producer
@@ -387,6 +388,11 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
   }
   tc_fence_before_sync();
   __syncthreads();
+  // Every warp of the CTA is done: the next kernel's CTAs may set themselves up while this one winds
+  // down.  (A trigger that any thread reaches earlier counts for the whole CTA: with the idle lanes of
+  // the producer and issuing warps passing it at the kernel's top, the successors' CTAs sat beside
+  // the running ones for the kernel's whole length and the compress step was 12 % slower.)
+  pdl_trigger();
   if (warp == kMmaWarp) tmem_dealloc(tmem_base, kTmemCols);
 }
 
@@ -395,6 +401,8 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
 __global__ void row_lse_from_parts_kernel(const float2* __restrict__ stat_part, float* __restrict__ row_lse,
                                           int rows, int GW, int vu_per_unit, int n_tiles, int tiles_per_cta,
                                           int max_slots) {
+  pdl_trigger();
+  pdl_wait();
   const int r = blockIdx.x * blockDim.x + threadIdx.x;
   if (r >= rows) return;
   const int unit = r / GW, row = r - unit * GW;
@@ -411,6 +419,8 @@ __global__ void row_lse_from_parts_kernel(const float2* __restrict__ stat_part, 
 }
 
 __global__ void add_votes_kernel(float* __restrict__ vote, const float* __restrict__ vote2, size_t n) {
+  pdl_trigger();
+  pdl_wait();
   const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (i < n) vote[i] += vote2[i];
 }
@@ -486,13 +496,13 @@ cudaError_t launch_row_stats_tc(const CompressGeom& g, const CompressWs& ws, con
   cudaError_t e = set_smem_limit<false>(smem);
   if (e != cudaSuccess) return e;
   const int grid = (a.total_tiles + a.tiles_per_cta - 1) / a.tiles_per_cta;
-  score_tc_kernel<false><<<grid, kThreads, smem, st>>>(qm, km, a);
+  e = launch_pdl(score_tc_kernel<false>, dim3(grid), dim3(kThreads), (size_t)smem, st, qm, km, a);
+  if (e != cudaSuccess) return e;
   const int rows = g.B * g.Hq * g.W;
-  row_lse_from_parts_kernel<<<(rows + 127) / 128, 128, 0, st>>>(a.stat_part, (float*)(wsp + ws.row_lse), rows, GW,
-                                                                a.vu_per_unit, a.n_tiles, a.tiles_per_cta,
-                                                                a.max_slots);
+  e = launch_pdl(row_lse_from_parts_kernel, dim3((rows + 127) / 128), dim3(128), 0, st, (const float2*)a.stat_part,
+                 (float*)(wsp + ws.row_lse), rows, GW, a.vu_per_unit, a.n_tiles, a.tiles_per_cta, a.max_slots);
   count_launch(2);
-  return cudaGetLastError();
+  return e != cudaSuccess ? e : cudaGetLastError();
 }
 
 // Votes of every candidate key, into ws.vote.
@@ -527,11 +537,13 @@ cudaError_t launch_votes_tc(const CompressGeom& g, const CompressWs& ws, const v
   cudaError_t e = set_smem_limit<true>(smem);
   if (e != cudaSuccess) return e;
   const int grid = (a.total_tiles + a.tiles_per_cta - 1) / a.tiles_per_cta;
-  score_tc_kernel<true><<<grid, kThreads, smem, st>>>(qm, km, a);
+  e = launch_pdl(score_tc_kernel<true>, dim3(grid), dim3(kThreads), (size_t)smem, st, qm, km, a);
+  if (e != cudaSuccess) return e;
   count_launch(1);
   if (a.n_blocks > 1) {
     const size_t n = (size_t)g.units * g.n_cand;
-    add_votes_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(a.vote, a.vote2, n);
+    e = launch_pdl(add_votes_kernel, dim3((unsigned)((n + 255) / 256)), dim3(256), 0, st, a.vote, (const float*)a.vote2, n);
+    if (e != cudaSuccess) return e;
     count_launch(1);
   }
   return cudaGetLastError();

@@ -38,6 +38,8 @@ pool_select_cluster_kernel(const float* __restrict__ vote, float* __restrict__ p
   __shared__ unsigned cnt[2][2];      // this CTA's counts of keys > T and == T, for the two thresholds
   __shared__ unsigned wsum[ROWS * kW][2];
 
+  pdl_trigger();
+  pdl_wait();
   cg::cluster_group cluster = cg::this_cluster();
   const int rank = (int)cluster.block_rank();
   const int unit = blockIdx.y;
@@ -230,14 +232,15 @@ pool_select_cluster_kernel(const float* __restrict__ vote, float* __restrict__ p
 template <int ROWS>
 void launch_rows(const CompressGeom& g, const CompressWs& ws, char* wsp, const float* scores, size_t stride,
                  int32_t* kept_idx, cudaStream_t st) {
+  // (the cluster shape is the kernel's own attribute; the launch adds programmatic serialisation)
   if (g.sized && g.n_calib > 0)
-    pool_select_cluster_kernel<ROWS, true><<<dim3(kClu, g.units), kT, 0, st>>>(
-        scores, (float*)(wsp + ws.pooled), (uint32_t*)(wsp + ws.bitmap), kept_idx, g.n_cand, g.L, g.pool, g.k_sel,
-        g.n_kept, g.bitmap_words, (uint32_t*)(wsp + ws.bitmap2), g.n_calib, stride);
+    launch_pdl(pool_select_cluster_kernel<ROWS, true>, dim3(kClu, g.units), dim3(kT), 0, st, scores,
+               (float*)(wsp + ws.pooled), (uint32_t*)(wsp + ws.bitmap), kept_idx, g.n_cand, g.L, g.pool, g.k_sel, g.n_kept,
+               g.bitmap_words, (uint32_t*)(wsp + ws.bitmap2), g.n_calib, stride);
   else
-    pool_select_cluster_kernel<ROWS, false><<<dim3(kClu, g.units), kT, 0, st>>>(
-        scores, (float*)(wsp + ws.pooled), (uint32_t*)(wsp + ws.bitmap), kept_idx, g.n_cand, g.L, g.pool, g.k_sel,
-        g.n_kept, g.bitmap_words, nullptr, 0, stride);
+    launch_pdl(pool_select_cluster_kernel<ROWS, false>, dim3(kClu, g.units), dim3(kT), 0, st, scores,
+               (float*)(wsp + ws.pooled), (uint32_t*)(wsp + ws.bitmap), kept_idx, g.n_cand, g.L, g.pool, g.k_sel, g.n_kept,
+               g.bitmap_words, (uint32_t*)nullptr, 0, stride);
 }
 
 }  // namespace
