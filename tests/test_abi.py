@@ -80,3 +80,28 @@ def test_null_arguments_are_rejected_before_any_cuda_call(lib):
     assert lib.calidrop_recalibrate(ctypes.byref(p), ptr, ptr, ptr, 10, 1, ptr, ptr, ptr, ptr, 1 << 20, None) == cd.INVALID_ARG
     assert lib.calidrop_recalibrate(ctypes.byref(p), ptr, ptr, ptr, 0, 0, ptr, ptr, ptr, ptr, 1 << 20, None) == cd.INVALID_ARG
     assert lib.calidrop_recalibrate(ctypes.byref(p), None, ptr, ptr, 10, 0, ptr, ptr, ptr, ptr, 1 << 20, None) == cd.INVALID_ARG
+
+
+def test_entry_points_of_the_other_eviction_rules_and_the_offload_validate_on_the_host(lib):
+    """The kept-list, accumulated-score and offload entry points refuse bad arguments before any CUDA call."""
+    p = cd.make_params(B=1, Hq=4, Hkv=2, L=300, window=8, pool=1, budget=40, n_cal=1, cap=40)
+    buf = (ctypes.c_char * 8192)()
+    ptr = ctypes.c_void_p((ctypes.addressof(buf) + 255) & ~255)     # an aligned host address: never dereferenced
+    pp = ctypes.byref(p)
+    # StreamingLLM's list: sinks must leave room for the window rows
+    assert lib.calidrop_select_streaming(pp, 40, ptr, None) == cd.INVALID_ARG
+    assert lib.calidrop_select_streaming(pp, -1, ptr, None) == cd.INVALID_ARG
+    assert lib.calidrop_select_streaming(pp, 4, None, None) == cd.INVALID_ARG
+    # H2O's list: window <= tail < budget
+    assert lib.calidrop_select_from_scores(pp, ptr, 7, ptr, ptr, 1 << 30, None) == cd.INVALID_ARG
+    assert lib.calidrop_select_from_scores(pp, ptr, 40, ptr, ptr, 1 << 30, None) == cd.INVALID_ARG
+    assert lib.calidrop_select_from_scores(pp, None, 20, ptr, ptr, 1 << 30, None) == cd.INVALID_ARG
+    assert lib.calidrop_select_from_scores(pp, ptr, 20, ptr, ptr, 16, None) == cd.WORKSPACE_TOO_SMALL
+    # accumulated scores: workspace = 4 B Hq L bytes, rounded up to 256
+    need = cd.calidrop_accumulated_scores_workspace_bytes(p)
+    assert need >= 4 * 1 * 4 * 300 and need % 256 == 0
+    assert lib.calidrop_accumulated_scores(pp, None, ptr, ptr, ptr, need, None) == cd.INVALID_ARG
+    assert lib.calidrop_accumulated_scores(pp, ptr, ptr, ptr, ptr, need - 256, None) == cd.WORKSPACE_TOO_SMALL
+    # calibration size below -1 is no setting
+    bad = cd.make_params(B=1, Hq=4, Hkv=2, L=300, window=8, pool=1, budget=40, n_cal=1, cap=40, calib_size=-2)
+    assert cd.calidrop_compress_workspace_bytes(bad) == 0
