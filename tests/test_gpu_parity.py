@@ -813,6 +813,54 @@ def test_h2o_accumulated_scores_from_the_library(cuda_lib, B, Hq, Hkv, L):
     assert cd.calidrop_accumulated_scores(p, None, to_dev(Kb), scores, ws, check=False) == cd.INVALID_ARG
 
 
+def test_calls_enqueued_back_to_back_give_the_results_of_calls_run_one_at_a_time(cuda_lib):
+    """The kernels of a compress call start beside the end of their predecessors (programmatic dependent
+    launch) and a decode launch prefetches ahead of its dependency wait: a stream of calls with no
+    synchronisation between them, on one shared workspace, must leave exactly what the same calls leave
+    when each is waited for."""
+    cd = cuda_lib
+    B, Hq, Hkv, L, W, pool, budget, n_cal = 2, 8, 2, 2300, 32, 7, 256, 32
+    cfgs = [wl.small_config(B=B, Hq=Hq, Hkv=Hkv, L=L, window=W, pool=pool, budget=budget, steps=3, n_heavy=24,
+                            seed=s) for s in (5, 6)]
+    inputs = [tuple(to_dev(x) for x in _inputs(c)) for c in cfgs]
+    T = 3
+    p = cd.make_params(B=B, Hq=Hq, Hkv=Hkv, L=L, window=W, pool=pool, budget=budget, n_cal=n_cal, cap=budget + T)
+    dec = [tuple(to_dev(x) for x in wl.gen_decode_inputs(c, wl.gen_q_obs(c), steps=T)) for c in cfgs]
+
+    def run(sync):
+        states = [cd.alloc_layer_state(p) for _ in range(2)]
+        for st in states:
+            st.ws_compress = states[0].ws_compress          # one workspace for every call
+        outs = []
+        for rnd in range(3):
+            for i, (st, (dQ, dK, dV)) in enumerate(zip(states, inputs)):
+                cd.calidrop_compress(p, dQ, dK, dV, None, st.kept_idx, st.K_kept, st.V_kept, st.O_c, st.LSE_c, st.C_q,
+                                     st.ws_compress)
+                if sync:
+                    torch.cuda.synchronize()
+                q, kn, vn = dec[i]
+                for t in range(T):
+                    o = torch.empty((B, Hq, 128), dtype=torch.bfloat16, device="cuda")
+                    cd.calidrop_decode(p, q[t], kn[t], vn[t], st.K_kept, st.V_kept, budget + t, st.O_c, st.LSE_c,
+                                       st.C_q, o, None, None, st.ws_decode)
+                    if sync:
+                        torch.cuda.synchronize()
+                    outs.append(o)
+        torch.cuda.synchronize()
+        lay = cd.calidrop_compress_workspace_layout(p)
+        assert int(states[0].ws_compress[lay.status_offset: lay.status_offset + 4].view(torch.int32).item()) == 0
+        return states, outs
+
+    ref_states, ref_outs = run(sync=True)
+    got_states, got_outs = run(sync=False)
+    for a, b in zip(ref_states, got_states):
+        assert torch.equal(a.kept_idx, b.kept_idx)
+        assert torch.equal(a.K_kept, b.K_kept) and torch.equal(a.V_kept, b.V_kept)
+        assert torch.equal(a.O_c, b.O_c) and torch.equal(a.LSE_c, b.LSE_c) and torch.equal(a.C_q, b.C_q)
+    for a, b in zip(ref_outs, got_outs):
+        assert torch.equal(a, b)
+
+
 # ---------------------------------------------------------------- seeded random shapes
 def _random_shapes(n, seed):
     rng = np.random.Generator(np.random.Philox(key=[seed, 1]))
